@@ -1,0 +1,188 @@
+/*
+ * CPU oracle, part 2: one full step of SketchedAMSGrad with gradient averaging (Algorithm 2), with the
+ * unsketching operator of Algorithm 3.  TEST INFRASTRUCTURE ONLY (see sk_oracle.h).
+ */
+#include "sk_oracle.h"
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+struct ora_state {
+    uint64_t d, k, seed, t, k_prev;
+    uint32_t n, r, c, log2g;
+    float lr, beta1, beta2, eps;
+    int v_keep, threads;
+    float *m, *e, *v, *vhat, *est, *tables, *sum;
+    uint32_t *I, *I_prev;
+    uint8_t* mask;
+    const uint32_t* h_idx;   /* injected hashes, or NULL: use the seeded family */
+    const int8_t* h_sgn;
+    uint64_t* row_key;
+};
+
+ora_state* ora_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, uint64_t seed,
+                      uint32_t log2g, float lr, float beta1, float beta2, float eps) {
+    if (d == 0 || n == 0 || r == 0 || r > 64 || c == 0 || k == 0 || k > d || log2g > 5) return NULL;
+    if ((c >> log2g) == 0 || d >= (1ULL << 32)) return NULL;
+    ora_state* s = (ora_state*)calloc(1, sizeof(ora_state));
+    s->d = d; s->n = n; s->r = r; s->c = c; s->k = k; s->seed = seed; s->log2g = log2g;
+    s->lr = lr; s->beta1 = beta1; s->beta2 = beta2; s->eps = eps;
+    s->threads = 1;
+    s->m = (float*)calloc((size_t)n * d, sizeof(float));        /* m_0 = 0 */
+    s->e = (float*)calloc((size_t)n * d, sizeof(float));        /* e_0 = 0 */
+    s->v = (float*)malloc((size_t)d * sizeof(float));
+    s->vhat = (float*)malloc((size_t)d * sizeof(float));
+    for (uint64_t j = 0; j < d; ++j) s->v[j] = s->vhat[j] = eps; /* v_0 = vhat_0 = eps */
+    s->est = (float*)calloc((size_t)d, sizeof(float));
+    s->tables = (float*)calloc((size_t)n * r * c, sizeof(float));
+    s->sum = (float*)calloc((size_t)r * c, sizeof(float));
+    s->I = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+    s->I_prev = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+    s->k_prev = 0;                                               /* I_0 = empty set */
+    s->mask = (uint8_t*)calloc((size_t)d, 1);
+    s->row_key = (uint64_t*)malloc((size_t)r * sizeof(uint64_t));
+    for (uint32_t j = 0; j < r; ++j) s->row_key[j] = ora_row_key(seed, j);
+    return s;
+}
+
+void ora_destroy(ora_state* s) {
+    if (!s) return;
+    free(s->m); free(s->e); free(s->v); free(s->vhat); free(s->est); free(s->tables); free(s->sum);
+    free(s->I); free(s->I_prev); free(s->mask); free(s->row_key); free(s);
+}
+
+void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn) { s->h_idx = idx; s->h_sgn = sgn; }
+
+void ora_set_option(ora_state* s, const char* key, int value) {
+    if (!strcmp(key, "v_keep")) s->v_keep = value;
+    else if (!strcmp(key, "threads")) s->threads = value > 0 ? value : 1;
+}
+
+void* ora_field(ora_state* s, const char* name) {
+    if (!strcmp(name, "m")) return s->m;
+    if (!strcmp(name, "e")) return s->e;
+    if (!strcmp(name, "v")) return s->v;
+    if (!strcmp(name, "vhat")) return s->vhat;
+    if (!strcmp(name, "est")) return s->est;
+    if (!strcmp(name, "tables")) return s->tables;
+    if (!strcmp(name, "sum")) return s->sum;
+    if (!strcmp(name, "I")) return s->I;
+    if (!strcmp(name, "I_prev")) return s->I_prev;
+    return NULL;
+}
+
+uint64_t ora_count(ora_state* s, const char* name) {
+    if (!strcmp(name, "I_prev")) return s->k_prev;
+    if (!strcmp(name, "I")) return s->t ? s->k : 0;
+    if (!strcmp(name, "t")) return s->t;
+    return 0;
+}
+
+/* bucket and sign of coordinate i in row j: injected arrays if present, else the seeded family */
+static inline void hash_at(const ora_state* s, uint32_t j, uint64_t i, uint32_t* b, int8_t* sg) {
+    if (s->h_idx) { *b = s->h_idx[j * s->d + i]; *sg = s->h_sgn[j * s->d + i]; return; }
+    uint64_t g = 1ULL << s->log2g, G = s->c / g;
+    uint64_t q = i >> s->log2g, o = i & (g - 1);
+    uint64_t u1 = ora_stream(s->row_key[j], 2 * q + 1);
+    uint64_t u2 = ora_stream(s->row_key[j], 2 * q + 2);
+    *b = (uint32_t)(g * (((u1 >> 32) * G) >> 32) + (o ^ ((u2 >> 32) & (g - 1))));
+    *sg = ((u1 >> o) & 1ULL) ? -1 : 1;
+}
+
+int ora_step(ora_state* s, const float* grads, float* x) {
+    const uint64_t d = s->d, k = s->k;
+    const uint32_t n = s->n, r = s->r, c = s->c;
+    const double b1 = (double)s->beta1, b2 = (double)s->beta2, lr = (double)s->lr;
+    const double rho = 1.0;   /* alpha_{t-1}/alpha_t with a constant step size (Theorem 2's alpha_t) */
+#ifdef _OPENMP
+    omp_set_num_threads(s->threads);
+#endif
+
+    /* Algorithm 2, worker side: m_t = beta1 m_{t-1} + (1-beta1) g_t */
+#pragma omp parallel for schedule(static)
+    for (uint64_t q = 0; q < (uint64_t)n * d; ++q)
+        s->m[q] = (float)(b1 * (double)s->m[q] + (1.0 - b1) * (double)grads[q]);
+
+    /* h_t = mean_w (g_t^(w)) restricted to I_{t-1} (zero elsewhere);
+       v_t = beta2 v_{t-1} + (1-beta2) h_t^2 ; vhat_t = max(vhat_{t-1}, v_t)   (master side) */
+    memset(s->mask, 0, (size_t)d);
+    for (uint64_t t = 0; t < s->k_prev; ++t) s->mask[s->I_prev[t]] = 1;
+#pragma omp parallel for schedule(static)
+    for (uint64_t j = 0; j < d; ++j) {
+        double h = 0.0;
+        if (s->mask[j]) {
+            for (uint32_t w = 0; w < n; ++w) h += (double)grads[(uint64_t)w * d + j];
+            h /= (double)n;
+        }
+        if (s->mask[j] || !s->v_keep) s->v[j] = (float)(b2 * (double)s->v[j] + (1.0 - b2) * h * h);
+        if (s->v[j] > s->vhat[j]) s->vhat[j] = s->v[j];
+    }
+
+    /* a_t^(w) = m_t^(w) + rho e_{t-1}^(w): the vector each worker sketches; kept in the e buffer */
+#pragma omp parallel for schedule(static)
+    for (uint64_t q = 0; q < (uint64_t)n * d; ++q)
+        s->e[q] = (float)((double)s->m[q] + rho * (double)s->e[q]);
+
+    /* S_t^(w) = S(a_t^(w)): one r x c table per worker, fp64 accumulation in increasing coordinate */
+#pragma omp parallel
+    {
+        double* acc = (double*)malloc((size_t)c * sizeof(double));
+#pragma omp for schedule(dynamic, 1)
+        for (uint64_t wj = 0; wj < (uint64_t)n * r; ++wj) {
+            uint32_t w = (uint32_t)(wj / r), j = (uint32_t)(wj % r);
+            const float* a = s->e + (uint64_t)w * d;
+            memset(acc, 0, (size_t)c * sizeof(double));
+            for (uint64_t i = 0; i < d; ++i) {
+                uint32_t b; int8_t sg;
+                hash_at(s, j, i, &b, &sg);
+                acc[b] += (double)sg * (double)a[i];
+            }
+            float* row = s->tables + ((uint64_t)w * r + j) * c;
+            for (uint32_t b = 0; b < c; ++b) row[b] = (float)acc[b];
+        }
+        free(acc);
+    }
+
+    /* S_t = (1/n) sum_w S_t^(w), workers added in the order 0,1,...,n-1 */
+#pragma omp parallel for schedule(static)
+    for (uint64_t q = 0; q < (uint64_t)r * c; ++q) {
+        double acc = 0.0;
+        for (uint32_t w = 0; w < n; ++w) acc += (double)s->tables[(uint64_t)w * r * c + q];
+        s->sum[q] = (float)(acc / (double)n);
+    }
+
+    /* U(S_t, vhat_t): est_i = median_j( s_j(i) S_t[j,h_j(i)] ) / sqrt(vhat_t,i) */
+#pragma omp parallel for schedule(static)
+    for (uint64_t i = 0; i < d; ++i) {
+        float q[64];
+        for (uint32_t j = 0; j < r; ++j) {
+            uint32_t b; int8_t sg;
+            hash_at(s, j, i, &b, &sg);
+            q[j] = (float)sg * s->sum[(uint64_t)j * c + b];
+        }
+        s->est[i] = (float)((double)ora_median(q, r) / sqrt((double)s->vhat[i]));
+    }
+
+    /* I_t = index set of Top-k of the estimates */
+    ora_topk(s->est, d, k, s->I);
+
+    /* Delta_t = (1/n) sum_w Delta_t^(w): exact coordinates of vhat^{-1/2} a_t^(w) on I_t;
+       x_{t+1} = x_t - alpha_t Delta_t ;  e_t^(w) = a_t^(w) with the coordinates of I_t removed */
+    for (uint64_t t = 0; t < k; ++t) {
+        uint64_t j = s->I[t];
+        double abar = 0.0;
+        for (uint32_t w = 0; w < n; ++w) abar += (double)s->e[(uint64_t)w * d + j];
+        abar /= (double)n;
+        double delta = abar / sqrt((double)s->vhat[j]);
+        x[j] = (float)((double)x[j] - lr * delta);
+        for (uint32_t w = 0; w < n; ++w) s->e[(uint64_t)w * d + j] = 0.0f;
+    }
+
+    memcpy(s->I_prev, s->I, (size_t)k * sizeof(uint32_t));
+    s->k_prev = k;
+    s->t += 1;
+    return 0;
+}

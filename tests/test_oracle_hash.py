@@ -1,0 +1,132 @@
+"""Pins for the oracle's hash and sign family (the bucket hashes h_j and sign hashes s_j of Section II-C).
+
+The paper names the hashes but fixes no family, so the family is this library's own definition; it is
+pinned by (a) the published known-answer vector of the splitmix64 generator it is built on, (b) an
+arbitrary-precision re-evaluation of the definition, (c) the structural and statistical properties a Count
+Sketch needs: range, sign domain, no collision inside a group, pair collisions at rate 1/c across groups,
+balanced signs, uniform buckets.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from conftest import GOLDEN
+
+M64 = (1 << 64) - 1
+GOLDEN_GAMMA = 0x9E3779B97F4A7C15
+
+
+def test_splitmix64_known_answers():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "splitmix64_kat.txt")) if l[0] != "#"]
+    assert len(rows) == 5
+    for s0, t, want in rows:
+        assert oracle.stream(int(s0), int(t)) == int(want)
+
+
+def _mix(z):
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & M64
+    return z ^ (z >> 31)
+
+
+def _family(seed, log2g, c, row, i):
+    """The family's definition evaluated with Python integers (no fixed-width arithmetic)."""
+    g = 1 << log2g
+    G = c // g
+    K = _mix((seed + (row + 1) * GOLDEN_GAMMA) & M64)
+    q, o = divmod(i, g)
+    u1 = _mix((K + (2 * q + 1) * GOLDEN_GAMMA) & M64)
+    u2 = _mix((K + (2 * q + 2) * GOLDEN_GAMMA) & M64)
+    B = ((u1 >> 32) * G) >> 32
+    p = (u2 >> 32) % g
+    return g * B + (o ^ p), (-1 if (u1 >> o) & 1 else 1)
+
+
+@pytest.mark.parametrize("log2g", [0, 1, 2, 3, 4, 5])
+@pytest.mark.parametrize("c", [2048, 100_000, 250_000, 401])
+def test_family_matches_bigint_definition(log2g, c):
+    if c >> log2g == 0:
+        pytest.skip("c < g")
+    rng = np.random.default_rng(7)
+    for seed in (0, 1, 0xDEADBEEFCAFEF00D):
+        for row in (0, 3, 9):
+            starts = [0, 1, 31, 33, int(rng.integers(0, 2**31)), 2**32 - 70]
+            for i0 in starts:
+                b, s = oracle.hash_family(seed, log2g, c, row, i0, 64)
+                for t in range(64):
+                    wb, ws = _family(seed, log2g, c, row, i0 + t)
+                    assert (int(b[t]), int(s[t])) == (wb, ws)
+
+
+@pytest.mark.parametrize("log2g", [0, 2, 5])
+def test_range_sign_domain_determinism(log2g):
+    c = 250_000
+    b, s = oracle.hash_family(0, log2g, c, 1, 0, 200_000)
+    b2, s2 = oracle.hash_family(0, log2g, c, 1, 0, 200_000)
+    assert np.array_equal(b, b2) and np.array_equal(s, s2)
+    assert b.max() < (c >> log2g) << log2g <= c
+    assert set(np.unique(s)) == {-1, 1}
+    # another row and another seed give different functions
+    b3, _ = oracle.hash_family(0, log2g, c, 2, 0, 200_000)
+    b4, _ = oracle.hash_family(1, log2g, c, 1, 0, 200_000)
+    assert (b != b3).mean() > 0.99 and (b != b4).mean() > 0.99
+
+
+@pytest.mark.parametrize("log2g", [1, 3, 5])
+def test_group_is_a_permutation_of_one_aligned_block(log2g):
+    g = 1 << log2g
+    c = 100_000
+    b, _ = oracle.hash_family(5, log2g, c, 0, 0, g * 4096)
+    blk = b.reshape(-1, g)
+    base = (blk[:, :1] // g) * g
+    assert np.all(blk // g * g == base)                       # one aligned block of g buckets per group
+    assert np.all(np.sort(blk - base, axis=1) == np.arange(g))  # every offset used exactly once
+    # xor structure: offset(o) ^ o is constant inside a group
+    x = (blk - base) ^ np.arange(g)
+    assert np.all(x == x[:, :1])
+    # the xor constant takes every value
+    assert len(np.unique(x[:, 0])) == g
+
+
+@pytest.mark.parametrize("log2g", [0, 3, 5])
+def test_bucket_uniformity_chi_square(log2g):
+    c, N = 2048, 2048 * 400
+    b, _ = oracle.hash_family(11, log2g, c, 2, 0, N)
+    cnt = np.bincount(b, minlength=c).astype(np.float64)
+    chi2 = ((cnt - N / c) ** 2 / (N / c)).sum()
+    # grouped buckets are filled in blocks of g, so compare at block level too; dof ~ c-1, sd ~ sqrt(2c)
+    if log2g == 0:
+        assert abs(chi2 - (c - 1)) < 6 * np.sqrt(2 * (c - 1))
+    G = c >> log2g
+    gcnt = cnt.reshape(G, -1).sum(1) / (1 << log2g)          # groups per block
+    ng = N >> log2g
+    chi2g = ((gcnt - ng / G) ** 2 / (ng / G)).sum()
+    assert abs(chi2g - (G - 1)) < 6 * np.sqrt(2 * (G - 1))
+
+
+@pytest.mark.parametrize("log2g", [0, 2, 5])
+def test_pair_collision_rate_and_sign_balance(log2g):
+    c, N = 4096, 60_000
+    g = 1 << log2g
+    b, s = oracle.hash_family(3, log2g, c, 0, 0, N)
+    assert abs(s.astype(np.float64).mean()) < 5 / np.sqrt(N)
+    # sign pairs inside a group and across groups are uncorrelated
+    assert abs((s[:-1].astype(np.float64) * s[1:]).mean()) < 5 / np.sqrt(N)
+    assert abs((s[:-g].astype(np.float64) * s[g:]).mean()) < 5 / np.sqrt(N)
+    # collisions: count pairs sharing a bucket
+    cnt = np.bincount(b, minlength=c).astype(np.float64)
+    pairs_same_bucket = (cnt * (cnt - 1) / 2).sum()
+    cross_pairs = N * (N - 1) / 2 - (N // g) * g * (g - 1) / 2
+    rate = pairs_same_bucket / cross_pairs
+    assert abs(rate * c - 1) < 0.02
+    # no two coordinates of one group share a bucket
+    blk = b[: (N // g) * g].reshape(-1, g)
+    assert all(len(np.unique(row)) == g for row in blk[:2000])
+
+
+def test_non_divisible_c_leaves_tail_buckets_unused():
+    c, log2g = 250_000, 5            # 250000 = 32*7812 + 16
+    b, _ = oracle.hash_family(0, log2g, c, 0, 0, 500_000)
+    assert b.max() < 7812 * 32

@@ -1,0 +1,190 @@
+"""Pins for the oracle's full step: Algorithm 2 (gradient averaging) with Algorithm 3's unsketch."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from conftest import GOLDEN
+
+HP = dict(lr=0.1, beta1=0.9, beta2=0.99, eps=1e-2)
+
+
+def _identity(d):
+    return np.arange(d, dtype=np.uint32)[None, :], np.ones((1, d), np.int8)
+
+
+def _golden():
+    out = {}
+    for line in open(os.path.join(GOLDEN, "amsgrad_ga_worked_examples.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        ex, t, q, j, val = line.split()
+        out.setdefault(ex, []).append((int(t), q, int(j), float(val)))
+    return out
+
+
+EXAMPLES = {
+    "A": dict(n=1, d=1, grads=[[1.0]]),
+    "B": dict(n=1, d=2, grads=[[1.0, 0.5]]),
+    "C": dict(n=2, d=2, grads=[[1.0, 0.5], [3.0, -0.5]]),
+    "D": dict(n=1, d=1, grads=[[1.0]], v_keep=True),
+}
+
+
+@pytest.mark.parametrize("ex", sorted(EXAMPLES))
+def test_worked_examples(ex):
+    cfg = EXAMPLES[ex]
+    n, d = cfg["n"], cfg["d"]
+    hi, hs = _identity(d)
+    o = oracle.Oracle(d, n, 1, d, 1, hash_idx=hi, hash_sgn=hs, v_keep=cfg.get("v_keep", False), **HP)
+    g = np.array(cfg["grads"], np.float32)
+    x = np.zeros(d, np.float32)
+    checks = _golden()[ex]
+    for t in range(1, max(c[0] for c in checks) + 1):
+        o.step(g, x)
+        for (tt, q, j, val) in checks:
+            if tt != t:
+                continue
+            if q == "x":
+                got = x[j]
+            elif q == "I":
+                got = o.field("I")[j]
+            elif q in ("e0", "e1"):
+                got = o.field("e")[int(q[1]), j]
+            elif q == "e":
+                got = o.field("e")[0, j]
+            else:
+                got = o.field(q)[j]
+            assert got == pytest.approx(val, rel=2e-6, abs=1e-9), (ex, t, q, j)
+
+
+def _run(d, n, r, c, k, steps, log2g, seed=0, identity=False, **kw):
+    rng = np.random.default_rng(seed + 100)
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.99, eps=1e-6)
+    hp.update(kw)
+    extra = {}
+    if identity:
+        hi, hs = _identity(d)
+        extra = dict(hash_idx=hi, hash_sgn=hs)
+        r, c = 1, d
+    o = oracle.Oracle(d, n, r, c, k, seed=seed, log2g=log2g, **hp, **extra)
+    x = rng.standard_normal(d).astype(np.float32)
+    hist = []
+    for t in range(steps):
+        g = (rng.standard_normal((n, d)) * rng.uniform(0.01, 1.0, d)).astype(np.float32)
+        prev = {f: o.field(f).copy() for f in ("m", "e", "v", "vhat")}
+        prev["I"] = o.field("I_prev").copy()
+        x0 = x.copy()
+        o.step(g, x)
+        hist.append(dict(g=g, prev=prev, x0=x0, x=x.copy(), I=o.field("I").copy(),
+                         **{f: o.field(f).copy() for f in ("m", "e", "v", "vhat", "est", "sum", "tables")}))
+    return o, hp, hist
+
+
+@pytest.mark.parametrize("log2g", [0, 4])
+def test_step_invariants(log2g):
+    d, n, r, c, k = 3000, 3, 5, 512, 100
+    o, hp, hist = _run(d, n, r, c, k, 6, log2g)
+    for t, h in enumerate(hist):
+        I, Iprev = h["I"], h["prev"]["I"]
+        assert len(I) == k and len(np.unique(I)) == k and np.all(np.diff(I.astype(np.int64)) > 0)
+        # vhat = max(vhat, v): never decreases, never below eps, changes only on I_{t-1} (proof of Lemma 3)
+        assert np.all(h["vhat"] >= h["prev"]["vhat"]) and np.all(h["vhat"] >= np.float32(hp["eps"]))
+        changed = np.flatnonzero(h["vhat"] != h["prev"]["vhat"])
+        assert np.isin(changed, Iprev).all()
+        assert np.all(h["vhat"] >= h["v"])
+        # off I_{t-1}, v decays by beta2 (Algorithm 2 with h_t zero there)
+        off = np.setdiff1d(np.arange(d), Iprev)
+        want = (np.float64(np.float32(hp["beta2"])) * h["prev"]["v"][off].astype(np.float64)).astype(np.float32)
+        assert np.array_equal(h["v"][off], want)
+        # m recurrence
+        b1 = np.float64(np.float32(hp["beta1"]))
+        wm = (b1 * h["prev"]["m"].astype(np.float64) + (1 - b1) * h["g"].astype(np.float64)).astype(np.float32)
+        assert np.array_equal(h["m"], wm)
+        # error feedback is a mask: e_t = a_t off I_t, 0 on I_t, so e_t + scatter(I_t, a_t[I_t]) = a_t exactly
+        a = (h["m"].astype(np.float64) + h["prev"]["e"].astype(np.float64)).astype(np.float32)
+        assert not h["e"][:, I].any()
+        rest = np.setdiff1d(np.arange(d), I)
+        assert np.array_equal(h["e"][:, rest], a[:, rest])
+        # aggregated sketch is the mean of worker sketches, and by linearity the sketch of the mean vector
+        np.testing.assert_allclose(h["sum"], h["tables"].astype(np.float64).mean(0), rtol=0, atol=1e-6)
+        idx = np.stack([oracle.hash_family(0, log2g, c, j, 0, d)[0] for j in range(r)])
+        sgn = np.stack([oracle.hash_family(0, log2g, c, j, 0, d)[1] for j in range(r)])
+        lin = oracle.sketch(a.astype(np.float64).mean(0).astype(np.float32), r, c, idx, sgn)
+        np.testing.assert_allclose(h["sum"], lin, rtol=0, atol=2e-6 * np.abs(lin).max())
+        # the update moves exactly the coordinates of I_t, by lr * mean_w a / sqrt(vhat)
+        moved = np.flatnonzero(h["x"] != h["x0"])
+        assert np.isin(moved, I).all()
+        delta = a.astype(np.float64).mean(0)[I] / np.sqrt(h["vhat"][I].astype(np.float64))
+        np.testing.assert_allclose(h["x"][I], h["x0"][I] - np.float64(np.float32(hp["lr"])) * delta, rtol=2e-7, atol=1e-7)
+        # I_t is the top-k of the stored estimates
+        assert np.array_equal(I, oracle.topk(h["est"], k))
+
+
+def test_lemma3_identity_and_contraction():
+    # Lemma 3: x_t - x~_t = alpha vhat_{t-1}^{-1/2} e_{t-1}, with x~_{t+1} = x~_t - alpha vhat_t^{-1/2} mean_w m_t.
+    # Also "Delta_t is some coordinates of Delta~_t": ||Delta~ - Delta|| <= ||Delta~||, and when I_t is the true
+    # top-k of Delta~_t (lossless sketch) the bound of Lemma 2 holds: <= sqrt(1-k/d) ||Delta~||.
+    d, n, k = 400, 4, 40
+    o, hp, hist = _run(d, n, 1, d, k, 12, 0, identity=True)
+    lr = np.float64(np.float32(hp["lr"]))
+    xt = hist[0]["x0"].astype(np.float64)
+    for h in hist:
+        vh = h["vhat"].astype(np.float64)
+        xt = xt - lr * h["m"].astype(np.float64).mean(0) / np.sqrt(vh)
+        ebar = h["e"].astype(np.float64).mean(0)
+        np.testing.assert_allclose(h["x"].astype(np.float64) - xt, lr * ebar / np.sqrt(vh), rtol=0, atol=5e-6)
+        a = h["m"].astype(np.float64) + h["prev"]["e"].astype(np.float64)
+        dtil = a.mean(0) / np.sqrt(vh)
+        dsel = np.zeros(d)
+        dsel[h["I"]] = dtil[h["I"]]
+        assert np.linalg.norm(dtil - dsel) <= np.sqrt(1 - k / d) * np.linalg.norm(dtil) * (1 + 1e-6)
+        true_topk = np.sort(np.argsort(-np.abs(dtil), kind="stable")[:k])
+        assert np.array_equal(h["I"], true_topk.astype(np.uint32))
+
+
+def test_no_compression_reduces_to_distributed_amsgrad():
+    # Section III-B: with no compressor (k = d, lossless sketch) Algorithm 2 is distributed AMSGrad on the mean
+    # gradient -- except that v first sees the gradient at t = 2, because I_0 is empty.
+    d, n = 50, 3
+    o, hp, hist = _run(d, n, 1, d, d, 8, 0, identity=True)
+    b1, b2, lr, eps = (np.float64(np.float32(hp[q])) for q in ("beta1", "beta2", "lr", "eps"))
+    m = np.zeros(d); v = np.full(d, eps); vh = v.copy(); x = hist[0]["x0"].astype(np.float64)
+    for t, h in enumerate(hist):
+        gbar = h["g"].astype(np.float64).mean(0)
+        m = b1 * m + (1 - b1) * gbar
+        v = b2 * v + (1 - b2) * (gbar ** 2 if t > 0 else 0.0)
+        vh = np.maximum(vh, v)
+        x = x - lr * m / np.sqrt(vh)
+        assert not h["e"].any()
+        np.testing.assert_allclose(h["x"], x, rtol=1e-5, atol=1e-6)
+        np.testing.assert_allclose(h["vhat"], vh, rtol=1e-5)
+
+
+def test_estimates_of_seeded_sketch_match_primitives():
+    # the step's on-the-fly hashing agrees with the explicit-array primitives pinned in test_oracle_sketch.py
+    d, n, r, c, k = 2000, 2, 5, 256, 50
+    o, hp, hist = _run(d, n, r, c, k, 2, 3, seed=4)
+    h = hist[-1]
+    idx = np.stack([oracle.hash_family(4, 3, c, j, 0, d)[0] for j in range(r)])
+    sgn = np.stack([oracle.hash_family(4, 3, c, j, 0, d)[1] for j in range(r)])
+    a = (h["m"].astype(np.float64) + h["prev"]["e"].astype(np.float64)).astype(np.float32)
+    for w in range(n):
+        assert np.array_equal(h["tables"][w], oracle.sketch(a[w], r, c, idx, sgn))
+    assert np.array_equal(h["est"], oracle.unsketch(h["sum"], d, idx, sgn, h["vhat"]))
+
+
+def test_threads_do_not_change_results():
+    d, n, r, c, k = 5000, 4, 5, 512, 64
+    rng = np.random.default_rng(0)
+    g = rng.standard_normal((2, n, d)).astype(np.float32)
+    outs = []
+    for th in (1, 4):
+        o = oracle.Oracle(d, n, r, c, k, seed=1, log2g=5, threads=th)
+        x = np.zeros(d, np.float32)
+        for t in range(2):
+            o.step(g[t], x)
+        outs.append((x.copy(), o.field("e").copy(), o.field("sum").copy(), o.field("I").copy()))
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
