@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the SketchedAMSGrad step: `python bench.py --gpus N --steps K --warmup W`.
+
+A step is one pass of the whole hot path (second moments on I_{t-1}, moments + Count Sketch of n workers,
+sum of sketches, unsketch + top-k, apply + error feedback) over one batch of synthetic gradients that is
+already resident in HBM.  The path does not shard (all n workers live on one GPU), so N > 1 runs N
+independent replicas, one process per GPU, and reports the aggregate (weak scaling).
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle on the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sketched_amsgrad_step_throughput"
+UNIT = "Gcoord/s"
+DEFAULT_WORKLOAD = "C3"      # d = 25.6M: the size the headline metric is quoted on
+
+# DRAM traffic of the dominant kernel (moments + sketch) from an ncu capture, in bytes per worker-coordinate,
+# valid only for the kernel source it was taken on (sha256 of sk_sketch.cu); otherwise reported as null.
+NCU_TRAFFIC = {"sha256": None, "bytes_per_worker_coord": None}
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out = self.proc.communicate(timeout=5)[0]
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        for line in out.splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [v for v in sm if v >= 0.5 * max(sm)] if sm else []
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _dist():
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return world, rank, local
+
+
+def reduce_max(value: float, world: int, device) -> float:
+    """Max over ranks (one number per rank); identity without a process group."""
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def reduce_sum(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def cpu_oracle_rate(w, scale: int, steps: int, threads: int):
+    """Times the CPU oracle, as it stands, on `steps` steps of the workload scaled down by `scale`."""
+    import oracle
+    from paper_2210_07454_b200 import synthetic
+    ws = synthetic.scaled(w, scale) if scale > 1 else w
+    src = synthetic.GradientSource(ws, device="cpu", cfg_id=int(w.name[1]) if w.name[1:2].isdigit() else 9)
+    lg = 5
+    while (1 << lg) > ws.c:
+        lg -= 1
+    o = oracle.Oracle(ws.d, ws.n, ws.r, ws.c, ws.k, seed=ws.seed, log2g=lg, lr=ws.lr, beta1=ws.beta1, beta2=ws.beta2,
+                      eps=ws.eps, threads=threads)
+    x = src.x0().numpy()
+    grads = [src.grads(t).numpy() for t in range(1, min(steps, 2) + 1)]
+    times = []
+    for t in range(steps):
+        t0 = time.perf_counter()
+        o.step(grads[t % len(grads)], x)
+        times.append(time.perf_counter() - t0)
+    sample = (f"{steps} step(s) of {w.name} scaled 1/{scale} (d={ws.d}, n={ws.n}, r={ws.r}, c={ws.c}, k={ws.k}), "
+              f"gcc -O2 OpenMP oracle")
+    return ws, times, sample
+
+
+def run_reference(args, w):
+    world, rank, _ = _dist()
+    if rank != 0:
+        return
+    threads = os.cpu_count() or 1
+    scale = args.ref_scale
+    total = args.steps + args.warmup
+    ws, times, sample = cpu_oracle_rate(w, scale, total, threads)
+    timed = times[args.warmup:]
+    ms = 1e3 * sum(timed) / len(timed)
+    value = ws.n * ws.d / (ms * 1e-3) / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k,
+                       "sampled_as": f"each step is one oracle step at 1/{scale} size"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--log2g", type=int, default=None)
+    ap.add_argument("--worker-chunk", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-scale", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stage-timing", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2210_07454_b200 import synthetic
+    w = synthetic.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    from paper_2210_07454_b200 import binding
+    world, rank, local = _dist()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg_id = int(w.name[1])
+    src = synthetic.GradientSource(w, device=dev, cfg_id=cfg_id)
+    opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
+                                  eps=w.eps, log2g=args.log2g)
+    opt.set_option("worker_chunk", args.worker_chunk)
+    # gradient buffers rotate so that no step finds its inputs in L2 (each set is far larger than L2 anyway)
+    free_b, _ = torch.cuda.mem_get_info()
+    set_bytes = 4 * w.n * w.d
+    nsets = int(max(2, min(4, (free_b * 0.5) // set_bytes)))
+    gsets = [src.grads(t + 1) for t in range(nsets)]
+    x = src.x0()
+    torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        opt.step(gsets[t % nsets], x)
+    opt.sync()
+    opt.timing()                                     # clear launch counters
+    opt.set_option("timing", 0 if args.no_stage_timing else 1)
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for t in range(args.steps):
+        opt.step(gsets[(args.warmup + t) % nsets], x)
+    ev1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    opt.sync()
+    ms_total = reduce_max(ev0.elapsed_time(ev1), world, dev)
+    nsteps, stage_ms, stage_launches = opt.timing()
+    opt.set_option("timing", 0)
+    launches = reduce_sum(float(sum(stage_launches)), world, dev)
+
+    ms_step = ms_total / args.steps
+    value = world * w.n * w.d / (ms_step * 1e-3) / 1e9
+    peak, peak_kind = _peaks()
+    b_alg = opt.algorithmic_bytes()
+
+    # dominant kernel: moments + sketch.  Algorithmic bytes per launch: 20 B per worker-coordinate streamed
+    # (read g, m, e; write m, e) plus the worker tables it fills (4 B per bucket).
+    k1_launches = max(1, stage_launches[2])
+    k1_bytes_step = 20 * w.n * w.d + 4 * w.n * w.r * w.c
+    roofline = None
+    if not args.no_stage_timing and stage_ms[2] > 0:
+        k1_ms = stage_ms[2] / k1_launches
+        k1_bytes = k1_bytes_step * args.steps / k1_launches
+        achieved = k1_bytes / (k1_ms * 1e-3) / 1e9
+        sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2210_07454_b200", "csrc", "sk_sketch.cu"), "rb").read()).hexdigest()
+        traffic = None
+        if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"]:
+            traffic = NCU_TRAFFIC["bytes_per_worker_coord"] * w.n * w.d * args.steps / k1_launches
+        roofline = {"bound": "hbm", "kernel": "k_moment_sketch_v4", "achieved": achieved, "peak": peak,
+                    "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+                    "ms_per_launch": k1_ms, "launches_per_step": k1_launches / args.steps,
+                    "algorithmic_bytes_per_launch": k1_bytes}
+
+    # end to end through the host entry point: pinned host gradients in, x back out, every step
+    e2e = None
+    if args.e2e_steps > 0:
+        hg = torch.empty((w.n, w.d), dtype=torch.float32, pin_memory=True)
+        hg.copy_(gsets[0])
+        hx = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
+        hx.copy_(x)
+        opt.step_host(hg, hx)                         # warm-up (allocates the staging buffers)
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            opt.step_host(hg, hx)
+        torch.cuda.synchronize()
+        dt = reduce_max(time.perf_counter() - t0, world, dev)
+        e2e = {"value": world * w.n * w.d * args.e2e_steps / dt / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": 4 * w.n * w.d + 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
+               "ms_per_step": 1e3 * dt / args.e2e_steps, "steps": args.e2e_steps}
+
+    if rank != 0:
+        return
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        threads = os.cpu_count() or 1
+        scale = 4
+        ws, times, sample = cpu_oracle_rate(w, scale, 3, threads)
+        cpu = {"value": ws.n * ws.d / (sum(times[1:]) / len(times[1:])) / 1e9, "unit": UNIT, "cores": threads,
+               "kind": "oracle", "sample": sample}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k,
+                       "recipe": w.recipe, "hash_group": 1 << opt.get_option("log2g"),
+                       "worker_chunk": opt.get_option("worker_chunk"), "replicas": world,
+                       "l2": f"inputs larger than L2: {nsets} rotating gradient sets of {set_bytes / 1e9:.2f} GB"},
+            "steps_per_s": 1e3 / ms_step,
+            "step_roofline": {"algorithmic_bytes": b_alg, "achieved_gbs": b_alg / (ms_step * 1e-3) / 1e9,
+                              "peak_gbs": peak, "peak_kind": f"of {peak_kind}",
+                              "frac": b_alg / (ms_step * 1e-3) / 1e9 / peak},
+            "roofline": roofline,
+            "stage_ms_per_step": {nm: stage_ms[q] / max(1, nsteps) for q, nm in enumerate(binding.STAGE_NAMES)},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,120 @@
+/*
+ * sketched_amsgrad.h -- C ABI of the B200 (sm_100a) library for one compressed optimiser step of
+ * SketchedAMSGrad with gradient averaging (Algorithm 2 of the paper), all n workers resident on one GPU.
+ *
+ * One step, in the paper's notation (w = worker, j = coordinate, constant step size so alpha_{t-1}/alpha_t = 1):
+ *   m_t^(w)   = beta1 m_{t-1}^(w) + (1-beta1) g_t^(w)                          (Algorithm 2, worker side)
+ *   h_t       = mean_w g_t^(w) on I_{t-1}, 0 elsewhere;  v_t = beta2 v_{t-1} + (1-beta2) h_t^2;
+ *   vhat_t    = max(vhat_{t-1}, v_t)                                            (Algorithm 2, master side)
+ *   a_t^(w)   = m_t^(w) + e_{t-1}^(w);   S_t^(w) = S(a_t^(w))                   (Count Sketch, Section II-C)
+ *   S_t       = (1/n) sum_w S_t^(w)       (workers added in the order 0..n-1)
+ *   est_j     = median_row( s_row(j) S_t[row, h_row(j)] ) / sqrt(vhat_t,j)      (Algorithm 3)
+ *   I_t       = indices of the k largest |est_j| (ties: smaller index)
+ *   x_j      -= lr * mean_w a_t^(w)_j / sqrt(vhat_t,j)   for j in I_t           (exact values, Section III-A)
+ *   e_t^(w)   = a_t^(w) off I_t, 0 on I_t                                       (error feedback)
+ * v_0 = vhat_0 = eps (an initial value, not a denominator term), m_0 = e_0 = 0, I_0 = empty.
+ *
+ * Conventions for every entry point:
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are ordinary memory.
+ *   - All arrays are dense fp32 / uint32 in C order.  The caller owns what it passes in; the handle owns all
+ *     optimiser state and scratch, allocated in sk_create and released in sk_destroy.
+ *   - Functions returning int give 0 on success or a negative SK_E* code; sk_last_error() then holds a
+ *     message (thread-local).  Nothing throws, nothing calls exit.  There is no CPU fallback: without a
+ *     CUDA device every call that needs one fails with SK_ECUDA.
+ *   - A handle is used from one thread at a time; kernels run asynchronously on the handle's stream
+ *     (the default stream unless sk_set_stream was called).
+ */
+#ifndef SKETCHED_AMSGRAD_H
+#define SKETCHED_AMSGRAD_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SK_OK        0
+#define SK_EINVAL   -1   /* bad argument (null, misaligned, out of range, unknown name) */
+#define SK_ECUDA    -2   /* a CUDA runtime call or launch failed; message in sk_last_error() */
+#define SK_ENOMEM   -3   /* device allocation failed */
+#define SK_ESTATE   -4   /* call not allowed in the handle's current state (e.g. hash option after first step) */
+#define SK_EDEVICE  -5   /* a kernel reported an internal inconsistency through the device status word */
+
+typedef struct sk_state sk_state;
+
+/* Algorithm 2's "Input/Set" lines.  d coordinates (1 <= d < 2^32), n workers, r x c sketch (1 <= r <= 16),
+ * k kept coordinates (1 <= k <= d), hash seed, step size lr, beta1, beta2 in [0,1), eps > 0.
+ * Allocates m,e (n*d), v,vhat (d), n+1 sketch tables and selection scratch (8*d bytes) on the current device
+ * and initialises them.  Returns NULL on failure (see sk_last_error()). */
+sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, uint64_t seed,
+                    float lr, float beta1, float beta2, float eps);
+
+/* One iteration of Algorithm 2 (the whole list above).  grads: device, n*d fp32, worker-major
+ * (grads[w*d + j]), read only.  x: device, d fp32, updated in place.  Both must be 4-byte aligned; the
+ * vectorised kernels are used when d % 4 == 0 and both are 16-byte aligned, scalar kernels otherwise.
+ * Asynchronous: returns after enqueueing on the handle's stream. */
+int sk_step(const float* grads, float* x, sk_state* state);
+
+/* Same step with HOST buffers: copies grads (n*d) to an internal device staging buffer and x (d) in,
+ * runs the step, copies x back, and synchronises the stream.  Pinned host memory makes the copies faster
+ * but is not required.  The staging buffers are allocated on first use and freed by sk_destroy. */
+int sk_step_host(const float* grads_host, float* x_host, sk_state* state);
+
+/* Releases everything sk_create and later calls allocated.  NULL is accepted. */
+void sk_destroy(sk_state* state);
+
+/* stream: a cudaStream_t cast to void* (NULL = default stream).  The handle does not own it. */
+int sk_set_stream(sk_state* state, void* stream);
+/* Waits for everything enqueued on the handle's stream and reports the device status word. */
+int sk_sync(sk_state* state);
+
+/* Options (integers):
+ *   "log2g"        hash group size g = 2^log2g, 0..5 (Section II-C fixes no hash family; see sk_hash).
+ *                  Only before the first step.  Default: the largest value <= 5 with 2^log2g <= c.
+ *   "worker_chunk" workers whose tables are accumulated concurrently by the sketch kernel (0 = automatic,
+ *                  sized so that the concurrently updated tables stay resident in L2).
+ *   "timing"       1 = record CUDA events around each stage (see sk_get_timing); 0 = off (default). */
+int sk_set_option(sk_state* state, const char* key, int64_t value);
+/* Also readable: "I_count" (entries "I" currently holds: 0 before the first step, else k unless sk_set installed
+ * fewer) and "vectorised" (1 when d % 4 == 0 and g >= 4, so aligned buffers take the 128-bit kernels). */
+int sk_get_option(const sk_state* state, const char* key, int64_t* value);
+
+/* The bucket hashes h_row and sign hashes s_row of Section II-C for coordinates i0 .. i0+count-1:
+ * idx_out[t] in [0,c), sign_out[t] in {+1,-1}; both DEVICE pointers.  Family (all arithmetic mod 2^64):
+ *   stream(s,t) = t-th output of splitmix64 started at s;  K_row = stream(seed, row+1);
+ *   q = i div g, o = i mod g, G = c div g;  u1 = stream(K_row, 2q+1), u2 = stream(K_row, 2q+2);
+ *   h_row(i) = g*floor((u1 div 2^32)*G / 2^32) + (o xor ((u2 div 2^32) mod g));
+ *   s_row(i) = +1 if bit o of u1 is clear, else -1. */
+int sk_hash(const sk_state* state, uint32_t row, uint64_t i0, uint64_t count,
+            uint32_t* idx_out, int8_t* sign_out);
+
+/* State access for checkpointing and for tests.  `buf` may be a host or a device pointer; `bytes` must equal
+ * the field's size.  Fields (fp32 unless noted):
+ *   "m","e"   n*d  per-worker momentum and error-feedback residual (after a step, "e" is e_t)
+ *   "v","vhat" d   second moments ("v" is brought up to date with the decay it is owed before export)
+ *   "tables"  n*r*c  the worker sketches S_t^(w) of the last step;  "sum"  r*c  the aggregate S_t
+ *   "est"     d    the estimates of the last step (recomputed on request from "sum" and "vhat"; get only)
+ *   "I"       k uint32  I_t of the last step, ascending (get);  set: installs I_{t-1} for the next step
+ *   "t"       1 uint64  number of steps taken
+ * Both calls synchronise the stream. */
+int sk_get(sk_state* state, const char* field, void* buf, uint64_t bytes);
+int sk_set(sk_state* state, const char* field, const void* buf, uint64_t bytes);
+
+/* Bytes one step must move by the method's own definition, used as the roofline numerator:
+ * 20*n*d (read g,m,e; write m,e) + 4*d (vhat) + 8*n*r*c + 4*r*c (worker tables written and read, aggregate
+ * written) + 12*n*k + 24*k (sparse gathers and updates on I_{t-1} and I_t). */
+uint64_t sk_algorithmic_bytes(const sk_state* state);
+
+/* Stage timing (option "timing" = 1).  Stages: 0 zero tables, 1 second moments on I_{t-1}, 2 moments+sketch,
+ * 3 sum of sketches, 4 unsketch+histogram, 5 unsketch+emit, 6 threshold refinement, 7 apply on I_t.
+ * Adds up the events of all steps since the last call into ms[0..7] (milliseconds) and launches[0..7]
+ * (kernel launches), then clears them.  Synchronises the stream.  Returns the number of steps covered, or <0. */
+#define SK_NUM_STAGES 8
+int sk_get_timing(sk_state* state, double* ms, uint64_t* launches);
+
+const char* sk_last_error(void);
+const char* sk_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

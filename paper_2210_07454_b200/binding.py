@@ -1,0 +1,160 @@
+"""ctypes binding of the C ABI in ``include/sketched_amsgrad.h``.
+
+Argument marshalling only: every step of the optimiser runs in the CUDA library.  There is no fallback; if the
+library has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsketched_amsgrad.so")
+
+EXPORTS = ["sk_create", "sk_step", "sk_step_host", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
+           "sk_get_option", "sk_hash", "sk_get", "sk_set", "sk_algorithmic_bytes", "sk_get_timing",
+           "sk_last_error", "sk_version"]
+NUM_STAGES = 8
+STAGE_NAMES = ["zero_tables", "second_moment", "moment_sketch", "sum_tables", "unsketch_hist",
+               "unsketch_emit", "refine", "apply"]
+
+_lib = None
+
+
+class SkError(RuntimeError):
+    pass
+
+
+def lib() -> C.CDLL:
+    """Loads the built library (build it with ``python -m paper_2210_07454_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise SkError(f"{LIB_PATH} is missing: build the CUDA library first (there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        u64, u32, f32, vp, i64 = C.c_uint64, C.c_uint32, C.c_float, C.c_void_p, C.c_int64
+        L.sk_create.restype = vp
+        L.sk_create.argtypes = [u64, u32, u32, u32, u64, u64, f32, f32, f32, f32]
+        L.sk_step.restype = C.c_int; L.sk_step.argtypes = [vp, vp, vp]
+        L.sk_step_host.restype = C.c_int; L.sk_step_host.argtypes = [vp, vp, vp]
+        L.sk_destroy.restype = None; L.sk_destroy.argtypes = [vp]
+        L.sk_set_stream.restype = C.c_int; L.sk_set_stream.argtypes = [vp, vp]
+        L.sk_sync.restype = C.c_int; L.sk_sync.argtypes = [vp]
+        L.sk_set_option.restype = C.c_int; L.sk_set_option.argtypes = [vp, C.c_char_p, i64]
+        L.sk_get_option.restype = C.c_int; L.sk_get_option.argtypes = [vp, C.c_char_p, C.POINTER(i64)]
+        L.sk_hash.restype = C.c_int; L.sk_hash.argtypes = [vp, u32, u64, u64, vp, vp]
+        L.sk_get.restype = C.c_int; L.sk_get.argtypes = [vp, C.c_char_p, vp, u64]
+        L.sk_set.restype = C.c_int; L.sk_set.argtypes = [vp, C.c_char_p, vp, u64]
+        L.sk_algorithmic_bytes.restype = u64; L.sk_algorithmic_bytes.argtypes = [vp]
+        L.sk_get_timing.restype = C.c_int
+        L.sk_get_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u64)]
+        L.sk_last_error.restype = C.c_char_p; L.sk_last_error.argtypes = []
+        L.sk_version.restype = C.c_char_p; L.sk_version.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc < 0:
+        raise SkError(f"error {rc}: {lib().sk_last_error().decode()}")
+
+
+def _ptr(t) -> int:
+    """Address of a torch tensor (device or host) or a numpy array."""
+    if isinstance(t, np.ndarray):
+        assert t.flags.c_contiguous
+        return t.ctypes.data
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _nbytes(t) -> int:
+    return t.nbytes if isinstance(t, np.ndarray) else t.numel() * t.element_size()
+
+
+class SketchedAMSGrad:
+    """Handle over ``sk_create`` / ``sk_step`` / ``sk_destroy`` and the auxiliary calls."""
+
+    _FIELD_SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "tables": "nrc", "sum": "rc"}
+
+    def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None):
+        self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
+        self._h = lib().sk_create(d, n, r, c, k, seed, lr, beta1, beta2, eps)
+        if not self._h:
+            raise SkError(f"sk_create failed: {lib().sk_last_error().decode()}")
+        if log2g is not None:
+            self.set_option("log2g", log2g)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().sk_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    # -- the hot path -----------------------------------------------------------------------------------
+    def step(self, grads, x) -> None:
+        """grads: CUDA float32 tensor of n*d elements (worker-major); x: CUDA float32 tensor of d, in place."""
+        _check(lib().sk_step(_ptr(grads), _ptr(x), self._h))
+
+    def step_host(self, grads, x) -> None:
+        """Same step with host buffers (numpy arrays or CPU tensors, ideally pinned); x is updated in place."""
+        _check(lib().sk_step_host(_ptr(grads), _ptr(x), self._h))
+
+    # -- auxiliaries ------------------------------------------------------------------------------------
+    def sync(self) -> None:
+        _check(lib().sk_sync(self._h))
+
+    def set_stream(self, cuda_stream_ptr: int) -> None:
+        _check(lib().sk_set_stream(self._h, cuda_stream_ptr))
+
+    def set_option(self, key: str, value: int) -> None:
+        _check(lib().sk_set_option(self._h, key.encode(), int(value)))
+
+    def get_option(self, key: str) -> int:
+        out = C.c_int64(0)
+        _check(lib().sk_get_option(self._h, key.encode(), C.byref(out)))
+        return int(out.value)
+
+    def hash(self, row: int, i0: int, count: int, idx_out, sign_out) -> None:
+        """Writes buckets (uint32 / int32 CUDA tensor) and signs (int8 CUDA tensor) of `count` coordinates."""
+        _check(lib().sk_hash(self._h, row, i0, count, _ptr(idx_out), _ptr(sign_out)))
+
+    def get(self, field: str, out=None):
+        """Copies a state field into `out` (numpy array or tensor) or into a new numpy array."""
+        if out is None:
+            if field == "I":
+                out = np.empty(self._count_I(), np.uint32)
+            elif field == "t":
+                out = np.empty(1, np.uint64)
+            else:
+                if field not in self._FIELD_SHAPES:
+                    raise SkError(f"unknown field '{field}'")
+                dims = {"n": self.n, "d": self.d, "r": self.r, "c": self.c}
+                out = np.empty(tuple(dims[ch] for ch in self._FIELD_SHAPES[field]), np.float32)
+        _check(lib().sk_get(self._h, field.encode(), _ptr(out) if _nbytes(out) else 0, _nbytes(out)))
+        return out
+
+    def _count_I(self) -> int:
+        return self.get_option("I_count")
+
+    def set(self, field: str, value) -> None:
+        _check(lib().sk_set(self._h, field.encode(), _ptr(value) if _nbytes(value) else 0, _nbytes(value)))
+
+    def algorithmic_bytes(self) -> int:
+        return int(lib().sk_algorithmic_bytes(self._h))
+
+    def timing(self):
+        """(steps, ms per stage, launches per stage) accumulated since the last call; clears the counters."""
+        ms = (C.c_double * NUM_STAGES)()
+        ln = (C.c_uint64 * NUM_STAGES)()
+        steps = lib().sk_get_timing(self._h, ms, ln)
+        _check(steps)
+        return steps, list(ms), [int(v) for v in ln]
+
+
+def version() -> str:
+    return lib().sk_version().decode()

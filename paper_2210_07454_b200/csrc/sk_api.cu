@@ -1,0 +1,372 @@
+// C ABI of the library (see include/sketched_amsgrad.h): handle life cycle, the step's launch sequence,
+// state export/import and stage timing.  Host code only; the kernels live in sk_sketch.cu / sk_select.cu.
+#include "../../include/sketched_amsgrad.h"
+#include "sk_internal.h"
+#include "sk_hash.cuh"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+namespace {
+
+thread_local std::string g_err;
+
+int fail(int code, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+#define SK_CUDA(expr)                                                                              \
+    do {                                                                                           \
+        cudaError_t err__ = (expr);                                                                \
+        if (err__ != cudaSuccess)                                                                  \
+            return fail(err__ == cudaErrorMemoryAllocation ? SK_ENOMEM : SK_ECUDA, "%s: %s", #expr, \
+                        cudaGetErrorString(err__));                                                \
+    } while (0)
+
+struct TimeRec { int stage; cudaEvent_t a, b; };
+
+}  // namespace
+
+struct sk_state {
+    sk::Params P{};
+    uint64_t seed = 0, t = 0;
+    float eps = 0;
+    uint32_t k_prev = 0;
+    int sm_count = 148;
+    size_t l2_bytes = 0;
+    int64_t worker_chunk = 0;
+    bool timing = false;
+    cudaStream_t stream = nullptr;
+    // device memory owned by the handle
+    float *m = nullptr, *e = nullptr, *v = nullptr, *vhat = nullptr, *tables = nullptr, *sum = nullptr;
+    uint32_t *vstamp = nullptr, *I = nullptr, *I_prev = nullptr, *hist = nullptr;
+    sk::Select* sel = nullptr;
+    sk::Cand* cand = nullptr;
+    float *stage_grads = nullptr, *stage_x = nullptr;
+    // timing
+    std::vector<TimeRec> recs;
+    std::vector<cudaEvent_t> free_events;
+    double ms[SK_NUM_STAGES] = {0};
+    uint64_t launches[SK_NUM_STAGES] = {0};
+    uint64_t timed_steps = 0;
+};
+
+namespace {
+
+void refresh_hash(sk_state* s) {
+    for (uint32_t j = 0; j < s->P.r; ++j) s->P.row_key[j] = sk::row_key(s->seed, j);
+    s->P.G = s->P.c >> s->P.log2g;
+}
+
+uint32_t chunk_of(const sk_state* s) {
+    if (s->worker_chunk > 0) return (uint32_t)std::min<int64_t>(s->worker_chunk, s->P.n);
+    // keep the tables that are being accumulated concurrently within a fraction of L2
+    const double budget = s->l2_bytes ? 0.38 * (double)s->l2_bytes : 48e6;
+    const double per_worker = (double)s->P.r * s->P.cs * 4.0;
+    uint32_t wc = (uint32_t)std::max(1.0, std::floor(budget / per_worker));
+    wc = std::min(wc, s->P.n);
+    const uint32_t chunks = (s->P.n + wc - 1) / wc;
+    return (s->P.n + chunks - 1) / chunks;
+}
+
+cudaEvent_t get_event(sk_state* s) {
+    if (!s->free_events.empty()) {
+        cudaEvent_t e = s->free_events.back();
+        s->free_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+int flush_timing(sk_state* s) {
+    if (s->recs.empty()) return SK_OK;
+    SK_CUDA(cudaStreamSynchronize(s->stream));
+    for (const TimeRec& r : s->recs) {
+        float ms = 0;
+        SK_CUDA(cudaEventElapsedTime(&ms, r.a, r.b));
+        s->ms[r.stage] += ms;
+        s->free_events.push_back(r.a);
+        s->free_events.push_back(r.b);
+    }
+    s->recs.clear();
+    return SK_OK;
+}
+
+struct StageTimer {   // brackets the launches of one stage with events when timing is on
+    sk_state* s; int stage; cudaEvent_t a = nullptr;
+    StageTimer(sk_state* s_, int stage_) : s(s_), stage(stage_) {
+        if (s->timing) { a = get_event(s); cudaEventRecord(a, s->stream); }
+    }
+    void done(int launches) {
+        s->launches[stage] += (uint64_t)launches;
+        if (s->timing) {
+            cudaEvent_t b = get_event(s);
+            cudaEventRecord(b, s->stream);
+            s->recs.push_back({stage, a, b});
+        }
+    }
+};
+
+int check_status(sk_state* s) {
+    sk::Select h{};
+    SK_CUDA(cudaMemcpyAsync(&h, s->sel, sizeof h, cudaMemcpyDeviceToHost, s->stream));
+    SK_CUDA(cudaStreamSynchronize(s->stream));
+    if (h.status) return fail(SK_EDEVICE, "device status word = %u (selection emitted %u of %u indices)", h.status,
+                              h.cnt_out, s->P.k);
+    return SK_OK;
+}
+
+int do_step(sk_state* s, const float* grads, float* x) {
+    const sk::Params& P = s->P;
+    const bool vec = (P.d % 4 == 0) && P.log2g >= 2 && ((uintptr_t)grads % 16 == 0) && ((uintptr_t)x % 16 == 0);
+    cudaStream_t st = s->stream;
+    const uint32_t t = (uint32_t)(s->t + 1);
+    if (s->timing && s->recs.size() > 4096) { int rc = flush_timing(s); if (rc) return rc; }
+
+    {   // v, vhat on I_{t-1}
+        StageTimer tm(s, 1);
+        tm.done(sk::launch_second_moment(P, grads, s->v, s->vhat, s->vstamp, s->I_prev, s->k_prev, t, st));
+    }
+    const uint32_t wc = chunk_of(s);
+    const uint64_t tfloats = (uint64_t)P.r * P.cs;
+    for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
+        const uint32_t nw = std::min(wc, P.n - w0);
+        {
+            StageTimer tm(s, 0);
+            tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats, st));
+        }
+        StageTimer tm(s, 2);
+        tm.done(sk::launch_moment_sketch(P, grads, s->m, s->e, s->tables, w0, nw, vec, s->sm_count, st));
+    }
+    {
+        StageTimer tm(s, 3);
+        tm.done(sk::launch_sum_tables(P, s->tables, s->sum, st));
+    }
+    {
+        StageTimer tm(s, 4);
+        int l = sk::launch_unsketch_hist(P, s->sum, s->vhat, s->hist, vec, s->sm_count, st);
+        l += sk::launch_pick_bin(P, s->hist, s->sel, st);
+        tm.done(l);
+    }
+    {
+        StageTimer tm(s, 5);
+        tm.done(sk::launch_unsketch_emit(P, s->sum, s->vhat, s->sel, s->I, s->cand, vec, s->sm_count, st));
+    }
+    {
+        StageTimer tm(s, 6);
+        tm.done(sk::launch_refine(P, s->sel, s->cand, s->I, st));
+    }
+    {
+        StageTimer tm(s, 7);
+        tm.done(sk::launch_apply(P, s->I, s->vhat, s->e, x, st));
+    }
+    SK_CUDA(cudaGetLastError());
+    std::swap(s->I, s->I_prev);      // I_prev now holds I_t
+    s->k_prev = P.k;
+    s->t += 1;
+    if (s->timing) s->timed_steps += 1;
+    return SK_OK;
+}
+
+enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_BAD };
+
+Field field_of(const char* name) {
+    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t"};
+    for (int q = 0; q < 9; ++q) if (!strcmp(name, names[q])) return (Field)q;
+    return F_BAD;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sk_last_error(void) { return g_err.c_str(); }
+const char* sk_version(void) { return "sketched-amsgrad-b200 0.1 (sm_100a)"; }
+
+sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, uint64_t seed, float lr,
+                    float beta1, float beta2, float eps) {
+    if (d < 1 || d >= (1ull << 32)) { fail(SK_EINVAL, "d must be in [1, 2^32)"); return nullptr; }
+    if (n < 1 || r < 1 || r > sk::kMaxRows || c < 1) { fail(SK_EINVAL, "need n >= 1, 1 <= r <= 16, c >= 1"); return nullptr; }
+    if (k < 1 || k > d) { fail(SK_EINVAL, "k must be in [1, d]"); return nullptr; }
+    if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f)) { fail(SK_EINVAL, "beta1, beta2 must be in [0,1)"); return nullptr; }
+    if (!(eps > 0.f) || !std::isfinite(eps) || !std::isfinite(lr)) { fail(SK_EINVAL, "eps must be > 0 and lr finite"); return nullptr; }
+    if ((uint64_t)r * (((uint64_t)c + 31) / 32 * 32) >= (1ull << 32)) { fail(SK_EINVAL, "r*c too large"); return nullptr; }
+
+    int dev = 0;
+    cudaDeviceProp prop{};
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        fail(SK_ECUDA, "no usable CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+        return nullptr;
+    }
+    sk_state* s = new sk_state();
+    s->sm_count = prop.multiProcessorCount;
+    s->l2_bytes = (size_t)prop.l2CacheSize;
+    s->seed = seed;
+    s->eps = eps;
+    sk::Params& P = s->P;
+    P.d = (uint32_t)d; P.n = n; P.r = r; P.c = c; P.k = (uint32_t)k;
+    P.cs = (c + 31u) / 32u * 32u;
+    P.beta1 = beta1; P.beta2 = beta2; P.lr = lr;
+    uint32_t lg = 5;
+    while ((1u << lg) > c) --lg;
+    P.log2g = lg;
+    refresh_hash(s);
+
+    const uint64_t nd = (uint64_t)n * d, tf = (uint64_t)r * P.cs;
+    bool ok = true;
+    auto alloc = [&](void** p, uint64_t bytes) {
+        if (ok && cudaMalloc(p, bytes ? bytes : 4) != cudaSuccess) {
+            ok = false;
+            fail(SK_ENOMEM, "cudaMalloc of %llu bytes failed: %s", (unsigned long long)bytes,
+                 cudaGetErrorString(cudaGetLastError()));
+        }
+    };
+    alloc((void**)&s->m, nd * 4); alloc((void**)&s->e, nd * 4);
+    alloc((void**)&s->v, d * 4); alloc((void**)&s->vhat, d * 4); alloc((void**)&s->vstamp, d * 4);
+    alloc((void**)&s->tables, (uint64_t)n * tf * 4); alloc((void**)&s->sum, tf * 4);
+    alloc((void**)&s->I, k * 4); alloc((void**)&s->I_prev, k * 4);
+    alloc((void**)&s->hist, sk::kHistBins * 4); alloc((void**)&s->sel, sizeof(sk::Select));
+    alloc((void**)&s->cand, d * sizeof(sk::Cand));
+    if (!ok) { sk_destroy(s); return nullptr; }
+    cudaMemset(s->m, 0, nd * 4); cudaMemset(s->e, 0, nd * 4);           // m_0 = e_0 = 0
+    cudaMemset(s->vstamp, 0, d * 4);
+    cudaMemset(s->tables, 0, (uint64_t)n * tf * 4); cudaMemset(s->sum, 0, tf * 4);
+    cudaMemset(s->hist, 0, sk::kHistBins * 4); cudaMemset(s->sel, 0, sizeof(sk::Select));
+    uint32_t eps_bits;
+    memcpy(&eps_bits, &eps, 4);
+    sk::launch_fill_u32((uint32_t*)s->v, d, eps_bits, nullptr);         // v_0 = vhat_0 = eps
+    sk::launch_fill_u32((uint32_t*)s->vhat, d, eps_bits, nullptr);
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        fail(SK_ECUDA, "initialisation failed: %s", cudaGetErrorString(cudaGetLastError()));
+        sk_destroy(s);
+        return nullptr;
+    }
+    return s;
+}
+
+void sk_destroy(sk_state* s) {
+    if (!s) return;
+    if (s->stream) cudaStreamSynchronize(s->stream); else cudaDeviceSynchronize();
+    for (void* p : {(void*)s->m, (void*)s->e, (void*)s->v, (void*)s->vhat, (void*)s->vstamp, (void*)s->tables,
+                    (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->sel, (void*)s->cand,
+                    (void*)s->stage_grads, (void*)s->stage_x})
+        if (p) cudaFree(p);
+    for (const TimeRec& r : s->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (cudaEvent_t e : s->free_events) cudaEventDestroy(e);
+    delete s;
+}
+
+int sk_step(const float* grads, float* x, sk_state* s) {
+    if (!s || !grads || !x) return fail(SK_EINVAL, "sk_step: null argument");
+    if (((uintptr_t)grads | (uintptr_t)x) % 4) return fail(SK_EINVAL, "sk_step: pointers must be 4-byte aligned");
+    return do_step(s, grads, x);
+}
+
+int sk_step_host(const float* grads_host, float* x_host, sk_state* s) {
+    if (!s || !grads_host || !x_host) return fail(SK_EINVAL, "sk_step_host: null argument");
+    const uint64_t nd = (uint64_t)s->P.n * s->P.d;
+    if (!s->stage_grads) {
+        SK_CUDA(cudaMalloc((void**)&s->stage_grads, nd * 4));
+        SK_CUDA(cudaMalloc((void**)&s->stage_x, (uint64_t)s->P.d * 4));
+    }
+    SK_CUDA(cudaMemcpyAsync(s->stage_grads, grads_host, nd * 4, cudaMemcpyHostToDevice, s->stream));
+    SK_CUDA(cudaMemcpyAsync(s->stage_x, x_host, (uint64_t)s->P.d * 4, cudaMemcpyHostToDevice, s->stream));
+    int rc = do_step(s, s->stage_grads, s->stage_x);
+    if (rc) return rc;
+    SK_CUDA(cudaMemcpyAsync(x_host, s->stage_x, (uint64_t)s->P.d * 4, cudaMemcpyDeviceToHost, s->stream));
+    SK_CUDA(cudaStreamSynchronize(s->stream));
+    return SK_OK;
+}
+
+int sk_set_stream(sk_state* s, void* stream) {
+    if (!s) return fail(SK_EINVAL, "null handle");
+    int rc = flush_timing(s);
+    if (rc) return rc;
+    SK_CUDA(cudaStreamSynchronize(s->stream));
+    s->stream = (cudaStream_t)stream;
+    return SK_OK;
+}
+
+int sk_sync(sk_state* s) {
+    if (!s) return fail(SK_EINVAL, "null handle");
+    return check_status(s);
+}
+
+int sk_set_option(sk_state* s, const char* key, int64_t value) {
+    if (!s || !key) return fail(SK_EINVAL, "null argument");
+    if (!strcmp(key, "log2g")) {
+        if (s->t != 0) return fail(SK_ESTATE, "log2g can only be changed before the first step");
+        if (value < 0 || value > 5 || (1u << value) > s->P.c) return fail(SK_EINVAL, "log2g must be in 0..5 with 2^log2g <= c");
+        s->P.log2g = (uint32_t)value;
+        refresh_hash(s);
+        return SK_OK;
+    }
+    if (!strcmp(key, "worker_chunk")) {
+        if (value < 0) return fail(SK_EINVAL, "worker_chunk must be >= 0");
+        s->worker_chunk = value;
+        return SK_OK;
+    }
+    if (!strcmp(key, "timing")) {
+        int rc = flush_timing(s);
+        if (rc) return rc;
+        s->timing = value != 0;
+        return SK_OK;
+    }
+    return fail(SK_EINVAL, "unknown option '%s'", key);
+}
+
+int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
+    if (!s || !key || !value) return fail(SK_EINVAL, "null argument");
+    if (!strcmp(key, "log2g")) *value = s->P.log2g;
+    else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
+    else if (!strcmp(key, "timing")) *value = s->timing;
+    else if (!strcmp(key, "I_count")) *value = s->k_prev;
+    else if (!strcmp(key, "vectorised")) *value = (s->P.d % 4 == 0) && s->P.log2g >= 2;
+    else return fail(SK_EINVAL, "unknown option '%s'", key);
+    return SK_OK;
+}
+
+int sk_hash(const sk_state* s, uint32_t row, uint64_t i0, uint64_t count, uint32_t* idx_out, int8_t* sign_out) {
+    if (!s || !idx_out || !sign_out) return fail(SK_EINVAL, "null argument");
+    if (row >= s->P.r || i0 + count > (1ull << 32)) return fail(SK_EINVAL, "row or coordinate range out of bounds");
+    if (count == 0) return SK_OK;
+    sk::launch_hash_export(s->P, row, i0, count, idx_out, sign_out, s->stream);
+    SK_CUDA(cudaGetLastError());
+    return SK_OK;
+}
+
+uint64_t sk_algorithmic_bytes(const sk_state* s) {
+    if (!s) return 0;
+    const uint64_t n = s->P.n, d = s->P.d, r = s->P.r, c = s->P.c, k = s->P.k;
+    return 20 * n * d + 4 * d + 8 * n * r * c + 4 * r * c + 12 * n * k + 24 * k;
+}
+
+int sk_get_timing(sk_state* s, double* ms, uint64_t* launches) {
+    if (!s || !ms || !launches) return fail(SK_EINVAL, "null argument");
+    int rc = flush_timing(s);
+    if (rc) return rc;
+    for (int q = 0; q < SK_NUM_STAGES; ++q) {
+        ms[q] = s->ms[q]; launches[q] = s->launches[q];
+        s->ms[q] = 0; s->launches[q] = 0;
+    }
+    const int steps = (int)s->timed_steps;
+    s->timed_steps = 0;
+    return steps;
+}
+
+}  // extern "C"
+
+#include "sk_api_state.inc"

@@ -1,0 +1,94 @@
+// Bucket and sign hashes of the Count Sketch (Section II-C names {h_j},{s_j}; the family is the library's own
+// and is documented with sk_hash in the public header).  Device-side evaluation only.
+#pragma once
+#include <cstdint>
+
+namespace sk {
+
+constexpr uint64_t kGolden = 0x9E3779B97F4A7C15ULL;
+
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+// t-th output (t >= 1) of splitmix64 started at state s
+__host__ __device__ __forceinline__ uint64_t stream(uint64_t s, uint64_t t) { return mix64(s + t * kGolden); }
+
+__host__ __device__ __forceinline__ uint64_t row_key(uint64_t seed, uint32_t row) {
+    return stream(seed, (uint64_t)row + 1);
+}
+
+// What one group of g = 2^log2g consecutive coordinates needs in one row.
+struct GroupHash {
+    uint32_t base;   // g * B : first bucket of the group's aligned block
+    uint32_t perm;   // xor permutation inside the block, in [0,g)
+    uint32_t signs;  // bit o set  <=>  coordinate with offset o carries sign -1
+};
+
+__device__ __forceinline__ GroupHash group_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t q) {
+    const uint64_t u1 = stream(key, 2ull * q + 1);
+    const uint64_t u2 = stream(key, 2ull * q + 2);
+    GroupHash h;
+    h.base = __umulhi((uint32_t)(u1 >> 32), G) << log2g;
+    h.perm = (uint32_t)(u2 >> 32) & ((1u << log2g) - 1u);
+    h.signs = (uint32_t)u1;
+    return h;
+}
+
+// Scalar form: bucket and sign (+1/-1) of coordinate i.
+__device__ __forceinline__ void coord_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t i,
+                                           uint32_t& bucket, float& sign) {
+    const uint32_t q = i >> log2g, o = i & ((1u << log2g) - 1u);
+    const GroupHash h = group_hash(key, log2g, G, q);
+    bucket = h.base + (o ^ h.perm);
+    sign = ((h.signs >> o) & 1u) ? -1.0f : 1.0f;
+}
+
+// Vector form for 4 consecutive coordinates i..i+3 (i % 4 == 0, g >= 4): they land in one aligned 16-byte
+// chunk of the row.  `off` is the element offset of that chunk inside the row; local coordinate l goes to
+// element (l xor p3) of the chunk; bit l of `sgn` is its sign.
+struct Quad {
+    uint32_t off;
+    uint32_t p3sgn;  // bits 0..1: p3 ; bits 2..5: sign bits of local coordinates 0..3
+};
+
+__device__ __forceinline__ Quad quad_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t i) {
+    const uint32_t q = i >> log2g, o = i & ((1u << log2g) - 1u);
+    const GroupHash h = group_hash(key, log2g, G, q);
+    Quad r;
+    r.off = h.base + ((o ^ h.perm) & ~3u);
+    r.p3sgn = (h.perm & 3u) | (((h.signs >> o) & 0xFu) << 2);
+    return r;
+}
+
+__device__ __forceinline__ float flip(float a, uint32_t bit) {  // a * (bit ? -1 : +1)
+    return __uint_as_float(__float_as_uint(a) ^ (bit << 31));
+}
+
+// signed and permuted: out element e = s(l) * a_l with l = e xor p3
+__device__ __forceinline__ float4 quad_scatter(const Quad h, float4 a) {
+    const uint32_t s = h.p3sgn >> 2;
+    a.x = flip(a.x, s & 1u);
+    a.y = flip(a.y, (s >> 1) & 1u);
+    a.z = flip(a.z, (s >> 2) & 1u);
+    a.w = flip(a.w, (s >> 3) & 1u);
+    if (h.p3sgn & 1u) { float t = a.x; a.x = a.y; a.y = t; t = a.z; a.z = a.w; a.w = t; }
+    if (h.p3sgn & 2u) { float t = a.x; a.x = a.z; a.z = t; t = a.y; a.y = a.w; a.w = t; }
+    return a;
+}
+
+// inverse: given the chunk's 4 values, return s(l) * chunk[l xor p3] for l = 0..3 (xor is an involution)
+__device__ __forceinline__ float4 quad_gather(const Quad h, float4 cch) {
+    if (h.p3sgn & 1u) { float t = cch.x; cch.x = cch.y; cch.y = t; t = cch.z; cch.z = cch.w; cch.w = t; }
+    if (h.p3sgn & 2u) { float t = cch.x; cch.x = cch.z; cch.z = t; t = cch.y; cch.y = cch.w; cch.w = t; }
+    const uint32_t s = h.p3sgn >> 2;
+    cch.x = flip(cch.x, s & 1u);
+    cch.y = flip(cch.y, (s >> 1) & 1u);
+    cch.z = flip(cch.z, (s >> 2) & 1u);
+    cch.w = flip(cch.w, (s >> 3) & 1u);
+    return cch;
+}
+
+}  // namespace sk

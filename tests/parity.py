@@ -1,0 +1,103 @@
+"""Helpers for the GPU-vs-oracle parity tests: tolerance rule, state transfer, stage-by-stage comparison."""
+from __future__ import annotations
+
+import numpy as np
+
+REL = 1e-5      # "within 1e-5 relative (fp32, atomic order)"
+
+
+def close(got, ref, what, groups_axis=None, rel=REL, scale=None):
+    """|got - ref| <= rel * max(|ref|, RMS) with RMS the root mean square of `ref` over its natural group
+    (the whole array, or each slice along `groups_axis`).  A bucket or a mean is a signed sum that can cancel
+    to nearly zero for any summation order, so the bound is relative to the group's scale, not to the element."""
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    if groups_axis is None:
+        rms = np.sqrt(np.mean(ref * ref)) if ref.size else 0.0
+    else:
+        axes = tuple(a for a in range(ref.ndim) if a != groups_axis)
+        rms = np.sqrt(np.mean(ref * ref, axis=axes, keepdims=True))
+    bound = rel * np.maximum(np.abs(ref), rms)
+    if scale is not None:                      # an additional per-element error scale inherited from an input
+        bound = np.maximum(bound, rel * np.asarray(scale, np.float64))
+    err = np.abs(got - ref)
+    bad = err > bound
+    if bad.any():
+        q = np.unravel_index(np.argmax(err / np.maximum(bound, 1e-300)), err.shape)
+        raise AssertionError(f"{what}: {bad.sum()} of {bad.size} outside tolerance; worst at {q}: "
+                             f"got {got[q]!r} ref {ref[q]!r} err {err[q]:.3e} bound {np.broadcast_to(bound, err.shape)[q]:.3e}")
+
+
+def est_scale(S_ref, vhat_ref):
+    """An estimate is one bucket of the aggregated sketch divided by sqrt(vhat): it inherits the bucket's absolute
+    error bound, rel * RMS(row), magnified by vhat^{-1/2}."""
+    S = np.asarray(S_ref, np.float64)
+    row_rms = np.sqrt(np.mean(S * S, axis=1)).max()
+    return row_rms / np.sqrt(np.asarray(vhat_ref, np.float64))
+
+
+def index_sets_agree(I_gpu, I_ref, est_ref, k, what="I", rel=REL, scale=None):
+    """The sets must be equal except for indices whose reference magnitude lies within the tolerance band of the
+    k-th largest magnitude tau.  Returns the symmetric difference (to be excluded from x/e comparisons)."""
+    I_gpu = np.asarray(I_gpu, np.int64)
+    I_ref = np.asarray(I_ref, np.int64)
+    assert len(I_gpu) == k == len(I_ref), (what, len(I_gpu), len(I_ref), k)
+    assert len(np.unique(I_gpu)) == k, f"{what}: repeated indices"
+    diff = np.setxor1d(I_gpu, I_ref)
+    if diff.size:
+        mag = np.abs(np.asarray(est_ref, np.float64))
+        tau = mag[I_ref].min()
+        rms = np.sqrt(np.mean(mag * mag))
+        band = rel * max(tau, rms) * np.ones(diff.size)
+        if scale is not None:
+            band = np.maximum(band, rel * np.asarray(scale, np.float64)[diff])
+        off = np.abs(mag[diff] - tau)
+        # both the differing element and the threshold element carry an error of up to one band
+        assert (off <= 2 * band).all(), (f"{what}: {diff.size} indices differ and {np.sum(off > 2 * band)} of them "
+                                         f"are outside the band (tau={tau:.6e}, worst {off.max():.3e})")
+    return diff
+
+
+def force_state(gpu, ora):
+    """Teacher forcing: install the oracle's state (m, e, v, vhat, I_{t-1}, t) in the GPU handle."""
+    t = np.array([ora.t], np.uint64)
+    gpu.set("t", t)
+    for f in ("m", "e", "v", "vhat"):
+        gpu.set(f, np.ascontiguousarray(ora.field(f)))
+    gpu.set("I", np.ascontiguousarray(ora.field("I_prev")))
+
+
+def compare_step(gpu, ora, x_gpu, x_ref, x_before, lr, check_tables=True, x_gpu_before=None):
+    """Compares every stage output of the step both sides just took from the same state and gradients."""
+    d, n, k = ora.d, ora.n, ora.k
+    if check_tables:
+        close(gpu.get("tables"), ora.field("tables"), "worker sketches", groups_axis=1)
+    close(gpu.get("sum"), ora.field("sum"), "aggregated sketch", groups_axis=0)
+    close(gpu.get("vhat"), ora.field("vhat"), "vhat")
+    close(gpu.get("v"), ora.field("v"), "v")
+    est_ref = ora.field("est")
+    sc = est_scale(ora.field("sum"), ora.field("vhat"))
+    close(gpu.get("est"), est_ref, "estimates", scale=sc)
+    I_gpu = gpu.get("I")
+    assert np.all(np.diff(I_gpu.astype(np.int64)) > 0)
+    diff = index_sets_agree(I_gpu, ora.field("I"), est_ref, k, scale=sc)
+    keep = np.ones(d, bool)
+    keep[diff] = False
+    close(gpu.get("m"), ora.field("m"), "m", groups_axis=0)
+    e_gpu, e_ref = gpu.get("e"), ora.field("e")
+    close(e_gpu[:, keep], e_ref[:, keep], "e", groups_axis=0)
+    assert not e_gpu[:, I_gpu].any(), "e must be zero on I_t"
+    # x: compare the CHANGE against lr * RMS(Delta) scale
+    dx_gpu = np.asarray(x_gpu, np.float64) - (x_before if x_gpu_before is None else np.asarray(x_gpu_before, np.float64))
+    dx_ref = np.asarray(x_ref, np.float64) - x_before
+    sel = np.asarray(ora.field("I"), np.int64)
+    rms = np.sqrt(np.mean(dx_ref[sel] ** 2)) if sel.size else 0.0
+    err = np.abs(dx_gpu - dx_ref)[keep]
+    # x itself is rounded to fp32 on both sides: allow one ulp of |x| on top of the relative bound on the change
+    bound = REL * np.maximum(np.abs(dx_ref[keep]), rms) + 1.2e-7 * np.abs(np.asarray(x_ref, np.float64)[keep])
+    assert (err <= bound).all(), f"x: {np.sum(err > bound)} coordinates outside tolerance, worst {err.max():.3e}"
+    untouched = np.setdiff1d(np.arange(d), I_gpu)
+    own_before = x_before.astype(np.float32) if x_gpu_before is None else np.asarray(x_gpu_before)
+    assert np.array_equal(np.asarray(x_gpu)[untouched], own_before[untouched])
+    return diff

@@ -1,0 +1,260 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+import oracle
+from parity import close, compare_step, force_state, index_sets_agree
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _binding():
+    from paper_2210_07454_b200 import binding
+    return binding
+
+
+def _source(w, device="cuda", cfg_id=None):
+    from paper_2210_07454_b200.synthetic import GradientSource
+    return GradientSource(w, device=device, cfg_id=cfg_id)
+
+
+def _workload(base, **over):
+    from paper_2210_07454_b200 import synthetic
+    w = synthetic.WORKLOADS[base]
+    if over:
+        w = synthetic.Workload(**{**w.__dict__, **over})
+    return w
+
+
+def _pair(w, log2g=None, threads=8):
+    b = _binding()
+    gpu = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
+                            eps=w.eps, log2g=log2g)
+    lg = gpu.get_option("log2g")
+    ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=lg, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
+                        eps=w.eps, threads=threads)
+    return gpu, ora
+
+
+# ------------------------------------------------------------------------------------------------ hash
+@pytest.mark.parametrize("log2g", [0, 1, 2, 3, 4, 5])
+@pytest.mark.parametrize("c", [2048, 250_000, 401])
+def test_hash_bit_exact(log2g, c):
+    b = _binding()
+    d, r = 300_000, 7
+    gpu = b.SketchedAMSGrad(d, 1, r, c, 1, seed=12345, log2g=log2g)
+    idx = torch.empty(d, dtype=torch.int32, device="cuda")
+    sgn = torch.empty(d, dtype=torch.int8, device="cuda")
+    for row in range(r):
+        gpu.hash(row, 0, d, idx, sgn)
+        gpu.sync()
+        wb, ws = oracle.hash_family(12345, log2g, c, row, 0, d)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), wb)
+        assert np.array_equal(sgn.cpu().numpy(), ws)
+    # far end of the coordinate range
+    gpu.hash(3, 2**32 - 1000, 1000, idx, sgn)
+    gpu.sync()
+    wb, ws = oracle.hash_family(12345, log2g, c, 3, 2**32 - 1000, 1000)
+    assert np.array_equal(idx[:1000].cpu().numpy().view(np.uint32), wb)
+    assert np.array_equal(sgn[:1000].cpu().numpy(), ws)
+
+
+# ------------------------------------------------------------------------------------------------ steps
+def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True):
+    gpu, ora = _pair(w, log2g)
+    src = _source(w, cfg_id=cfg_id)
+    x_gpu = src.x0()
+    x_ref = x_gpu.cpu().numpy().copy()
+    diverged_at = None
+    for t in range(1, steps + 1):
+        g = src.grads(t)
+        g_host = g.cpu().numpy()
+        if teacher and t > 1:
+            force_state(gpu, ora)
+            x_gpu.copy_(torch.from_numpy(x_ref))
+        x_before = x_ref.astype(np.float64).copy()
+        x_gpu_before = x_gpu.cpu().numpy().copy()
+        gpu.step(g, x_gpu)
+        gpu.sync()
+        ora.step(g_host, x_ref)
+        diff = compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, check_tables=check_tables,
+                            x_gpu_before=x_gpu_before)
+        if diff.size and diverged_at is None:
+            diverged_at = t
+            if not teacher:
+                break
+    return diverged_at
+
+
+def test_c1_ten_steps_teacher_forced():
+    _run_steps(_workload("C1"), 10)
+
+
+def test_c1_free_running():
+    # without teacher forcing the trajectories may legitimately split once an in-band index flips;
+    # until then every stage must agree (compare_step raises otherwise)
+    _run_steps(_workload("C1"), 10, teacher=False)
+
+
+@pytest.mark.parametrize("log2g", [0, 1, 2, 3, 4])
+def test_c1_other_group_sizes(log2g):
+    _run_steps(_workload("C1"), 3, log2g=log2g)
+
+
+EDGE = {
+    "k1": dict(d=4096, n=2, r=3, c=512, k=1),
+    "k_eq_d": dict(d=2048, n=2, r=3, c=4096, k=2048),
+    "r1_n1": dict(d=8192, n=1, r=1, c=1024, k=100),
+    "d_odd": dict(d=10_007, n=3, r=5, c=1000, k=333),          # scalar kernels: d % 4 != 0, c % 32 != 0
+    "c_odd": dict(d=20_000, n=3, r=5, c=401, k=200),
+    "r_even": dict(d=30_000, n=2, r=10, c=2048, k=300),        # lower median
+    "r16": dict(d=12_000, n=2, r=16, c=1024, k=120),           # run-time row count
+    "r9": dict(d=12_000, n=2, r=9, c=1024, k=120),
+    "n_odd_tail": dict(d=50_000, n=5, r=5, c=4096, k=500),     # odd worker count: the pair loop's tail
+    "tiny": dict(d=4, n=1, r=1, c=32, k=2),
+    "ragged_tile": dict(d=1024 * 37 + 12, n=4, r=7, c=3000, k=700),
+}
+
+
+@pytest.mark.parametrize("case", sorted(EDGE))
+def test_edge_cases(case):
+    w = _workload("C1", name="E", steps=3, recipe="planted", **EDGE[case])
+    _run_steps(w, 3, cfg_id=7)
+
+
+def test_worker_chunking_matches_single_pass():
+    w = _workload("C1", name="E", d=40_000, n=6, r=5, c=2048, k=400)
+    b = _binding()
+    src = _source(w, cfg_id=6)
+    outs = []
+    for chunk in (0, 1, 4):
+        gpu = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=3)
+        gpu.set_option("worker_chunk", chunk)
+        x = src.x0()
+        for t in (1, 2):
+            gpu.step(src.grads(t), x)
+        gpu.sync()
+        outs.append((gpu.get("tables"), gpu.get("I"), x.cpu().numpy()))
+    for o in outs[1:]:
+        close(o[0], outs[0][0], "tables under chunking", groups_axis=1)
+
+
+def test_integer_inputs_are_bit_exact():
+    # small-integer gradients and beta1 = 0 make every sum exact in fp32, whatever the order of the atomic adds:
+    # a lost or doubled update would show as a wrong integer
+    d, n, r, c, k = 200_000, 4, 5, 4096, 1000
+    b = _binding()
+    gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0)
+    ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=gpu.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
+                        threads=8)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    x = torch.zeros(d, device="cuda")
+    x_ref = np.zeros(d, np.float32)
+    g = torch.randint(-8, 9, (n, d), generator=gen, device="cuda").float()
+    gpu.step(g, x)
+    gpu.sync()
+    ora.step(g.cpu().numpy(), x_ref)
+    assert np.array_equal(gpu.get("tables"), ora.field("tables"))
+    assert np.array_equal(gpu.get("m"), ora.field("m"))
+    # n = 4: the mean of four integer tables is exact too
+    assert np.array_equal(gpu.get("sum"), ora.field("sum"))
+    assert np.array_equal(gpu.get("est"), ora.field("est"))
+    assert np.array_equal(gpu.get("I"), ora.field("I"))       # ties are everywhere here: smaller index must win
+    assert np.array_equal(gpu.get("e"), ora.field("e"))
+    assert np.array_equal(x.cpu().numpy(), x_ref)
+
+
+def test_all_zero_gradients_select_lowest_indices():
+    d, n, r, c, k = 50_000, 2, 5, 1024, 77
+    b = _binding()
+    gpu = b.SketchedAMSGrad(d, n, r, c, k)
+    x = torch.ones(d, device="cuda")
+    gpu.step(torch.zeros((n, d), device="cuda"), x)
+    gpu.sync()
+    assert np.array_equal(gpu.get("I"), np.arange(k, dtype=np.uint32))
+    assert torch.equal(x, torch.ones(d, device="cuda"))
+
+
+def test_lazy_v_decay_is_bit_exact_over_steps():
+    w = _workload("C1", name="E", d=30_000, n=2, r=5, c=2048, k=300, steps=8)
+    gpu, ora = _pair(w)
+    src = _source(w, cfg_id=5)
+    x = src.x0()
+    x_ref = x.cpu().numpy().copy()
+    ever = np.zeros(w.d, bool)
+    for t in range(1, 9):
+        g = src.grads(t)
+        prev = ora.field("I_prev").copy()
+        gpu.step(g, x)
+        ora.step(g.cpu().numpy(), x_ref)
+        if np.setxor1d(gpu.get("I"), ora.field("I")).size:
+            break
+        ever[prev] = True
+        # a coordinate that has never been selected has only decayed: one fp32 multiply per step on both sides
+        assert np.array_equal(gpu.get("v")[~ever], ora.field("v")[~ever])
+        # v is a sum of non-negative terms: no cancellation, so the bound is relative to each element
+        np.testing.assert_allclose(gpu.get("v"), ora.field("v"), rtol=1e-5, atol=0)
+        close(gpu.get("vhat"), ora.field("vhat"), "vhat")
+
+
+def test_checkpoint_roundtrip():
+    w = _workload("C1", name="E", d=20_000, n=3, r=5, c=2048, k=200)
+    b = _binding()
+    src = _source(w, cfg_id=4)
+    a = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=1)
+    xa = src.x0()
+    for t in (1, 2, 3):
+        a.step(src.grads(t), xa)
+    a.sync()
+    c2 = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=1)
+    c2.set("t", a.get("t"))
+    for f in ("m", "e", "v", "vhat", "I"):
+        c2.set(f, a.get(f))
+    xb = xa.clone()
+    a.step(src.grads(4), xa)
+    c2.step(src.grads(4), xb)
+    a.sync(); c2.sync()
+    assert np.array_equal(a.get("I"), c2.get("I"))
+    close(xb.cpu().numpy(), xa.cpu().numpy(), "x after resume")
+    close(c2.get("e"), a.get("e"), "e after resume", groups_axis=0)
+    assert np.array_equal(c2.get("v"), a.get("v"))
+
+
+def test_host_step_matches_device_step():
+    w = _workload("C1", name="E", d=16_384, n=2, r=5, c=1024, k=100)
+    b = _binding()
+    src = _source(w, cfg_id=3)
+    a = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k)
+    h = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k)
+    xa = src.x0()
+    xh = xa.cpu().numpy().copy()
+    for t in (1, 2):
+        g = src.grads(t)
+        a.step(g, xa)
+        h.step_host(g.cpu().numpy(), xh)
+    a.sync()
+    assert np.array_equal(a.get("I"), h.get("I"))
+    close(xh, xa.cpu().numpy(), "x via host entry point")
+
+
+def test_argument_errors():
+    b = _binding()
+    with pytest.raises(b.SkError):
+        b.SketchedAMSGrad(100, 1, 5, 64, 101)          # k > d
+    with pytest.raises(b.SkError):
+        b.SketchedAMSGrad(100, 1, 17, 64, 10)          # r > 16
+    with pytest.raises(b.SkError):
+        b.SketchedAMSGrad(100, 1, 5, 64, 10, eps=0.0)
+    s = b.SketchedAMSGrad(100, 1, 5, 64, 10)
+    with pytest.raises(b.SkError):
+        s.set_option("log2g", 7)
+    with pytest.raises(b.SkError):
+        s.get("nope")
+    with pytest.raises(b.SkError):
+        s.set("I", np.array([100], np.uint32))          # index >= d
+    x = torch.zeros(100, device="cuda")
+    s.step(torch.zeros((1, 100), device="cuda"), x)
+    with pytest.raises(b.SkError):
+        s.set_option("log2g", 2)                        # hash family is fixed after the first step
