@@ -168,8 +168,11 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--log2g", type=int, default=None)
     ap.add_argument("--worker-chunk", type=int, default=0)
+    ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-scale", type=int, default=16)
+    ap.add_argument("--scale", type=int, default=1, help="run the workload at 1/SCALE size (profiling captures)")
+    ap.add_argument("--grad-sets", type=int, default=0, help="rotating gradient sets (0 = as many as fit, 2..4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-timing", action="store_true")
     args = ap.parse_args()
@@ -177,6 +180,9 @@ def main():
 
     from paper_2210_07454_b200 import synthetic
     w = synthetic.WORKLOADS[args.workload]
+    cfg_id = int(w.name[1])
+    if args.scale > 1:
+        w = synthetic.scaled(w, args.scale)
     if args.impl == "reference":
         return run_reference(args, w)
 
@@ -190,15 +196,16 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg_id = int(w.name[1])
     src = synthetic.GradientSource(w, device=dev, cfg_id=cfg_id)
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
                                   eps=w.eps, log2g=args.log2g)
     opt.set_option("worker_chunk", args.worker_chunk)
+    if args.sketch_ctas:
+        opt.set_option("sketch_ctas_per_sm", args.sketch_ctas)
     # gradient buffers rotate so that no step finds its inputs in L2 (each set is far larger than L2 anyway)
     free_b, _ = torch.cuda.mem_get_info()
     set_bytes = 4 * w.n * w.d
-    nsets = int(max(2, min(4, (free_b * 0.5) // set_bytes)))
+    nsets = args.grad_sets if args.grad_sets > 0 else int(max(2, min(4, (free_b * 0.5) // set_bytes)))
     gsets = [src.grads(t + 1) for t in range(nsets)]
     x = src.x0()
     torch.cuda.synchronize()

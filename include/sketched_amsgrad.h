@@ -81,9 +81,9 @@ int sk_get_option(const sk_state* state, const char* key, int64_t* value);
 /* The bucket hashes h_row and sign hashes s_row of Section II-C for coordinates i0 .. i0+count-1:
  * idx_out[t] in [0,c), sign_out[t] in {+1,-1}; both DEVICE pointers.  Family (all arithmetic mod 2^64):
  *   stream(s,t) = t-th output of splitmix64 started at s;  K_row = stream(seed, row+1);
- *   q = i div g, o = i mod g, G = c div g;  u1 = stream(K_row, 2q+1), u2 = stream(K_row, 2q+2);
- *   h_row(i) = g*floor((u1 div 2^32)*G / 2^32) + (o xor ((u2 div 2^32) mod g));
- *   s_row(i) = +1 if bit o of u1 is clear, else -1. */
+ *   q = i div g, o = i mod g, G = c div g;  u = stream(K_row, q+1), hi = u div 2^32, lo = u mod 2^32;
+ *   x = hi*G;  h_row(i) = g*(x div 2^32) + (o xor p), p = the leading log2(g) bits of (x mod 2^32);
+ *   s_row(i) = +1 if bit o of lo is clear, else -1. */
 int sk_hash(const sk_state* state, uint32_t row, uint64_t i0, uint64_t count,
             uint32_t* idx_out, int8_t* sign_out);
 

@@ -15,11 +15,13 @@
  *   stream(s,t): t-th output of splitmix64 started at state s, = mix64(s + t*GOLDEN)
  *   K_j        = stream(seed, j+1)                                   row key
  *   g = 2^b consecutive coordinates form a group: q = i div g, o = i mod g, G = floor(c/g)
- *   u1 = stream(K_j, 2q+1), u2 = stream(K_j, 2q+2)
- *   B  = floor( (u1 div 2^32) * G / 2^32 )                           bucket group, in [0,G)
- *   p  = (u2 div 2^32) mod g                                         xor-permutation inside the group
+ *   u  = stream(K_j, q+1);  hi = u div 2^32, lo = u mod 2^32;  x = hi * G  (a 64-bit product)
+ *   B  = x div 2^32                                                  bucket group, in [0,G)
+ *   p  = (x mod 2^32) div 2^(32-b)                                   xor-permutation inside the group: the
+ *                                                                    leading b bits of the remainder of the
+ *                                                                    range reduction (p = 0 when g = 1)
  *   h_j(i) = g*B + (o xor p)
- *   s_j(i) = +1 if bit o of (u1 mod 2^32) is 0, else -1
+ *   s_j(i) = +1 if bit o of lo is 0, else -1
  *
  * Two coordinates of one group never share a bucket; two coordinates of different groups share one
  * with probability 1/(G*g).  With g = 1 this is an ordinary per-coordinate hash.
@@ -43,12 +45,13 @@ void ora_hash_one(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint6
     uint64_t q = i >> log2g;
     uint64_t o = i & (g - 1);
     uint64_t K = ora_row_key(seed, row);
-    uint64_t u1 = ora_stream(K, 2 * q + 1);
-    uint64_t u2 = ora_stream(K, 2 * q + 2);
-    uint64_t B = ((u1 >> 32) * G) >> 32;
-    uint64_t p = (u2 >> 32) & (g - 1);
+    uint64_t u = ora_stream(K, q + 1);
+    uint64_t hi = u >> 32, lo = u & 0xFFFFFFFFULL;
+    uint64_t x = hi * G;
+    uint64_t B = x >> 32;
+    uint64_t p = log2g ? ((x & 0xFFFFFFFFULL) >> (32 - log2g)) : 0;
     *bucket = (uint32_t)(g * B + (o ^ p));
-    *sign = ((u1 >> o) & 1ULL) ? -1 : 1;
+    *sign = ((lo >> o) & 1ULL) ? -1 : 1;
 }
 
 void ora_hash(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint64_t i0, uint64_t count,

@@ -86,10 +86,11 @@ static inline void hash_at(const ora_state* s, uint32_t j, uint64_t i, uint32_t*
     if (s->h_idx) { *b = s->h_idx[j * s->d + i]; *sg = s->h_sgn[j * s->d + i]; return; }
     uint64_t g = 1ULL << s->log2g, G = s->c / g;
     uint64_t q = i >> s->log2g, o = i & (g - 1);
-    uint64_t u1 = ora_stream(s->row_key[j], 2 * q + 1);
-    uint64_t u2 = ora_stream(s->row_key[j], 2 * q + 2);
-    *b = (uint32_t)(g * (((u1 >> 32) * G) >> 32) + (o ^ ((u2 >> 32) & (g - 1))));
-    *sg = ((u1 >> o) & 1ULL) ? -1 : 1;
+    uint64_t u = ora_stream(s->row_key[j], q + 1);
+    uint64_t x = (u >> 32) * G;
+    uint64_t p = s->log2g ? ((x & 0xFFFFFFFFULL) >> (32 - s->log2g)) : 0;
+    *b = (uint32_t)(g * (x >> 32) + (o ^ p));
+    *sg = (((u & 0xFFFFFFFFULL) >> o) & 1ULL) ? -1 : 1;
 }
 
 int ora_step(ora_state* s, const float* grads, float* x) {

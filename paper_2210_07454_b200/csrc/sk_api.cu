@@ -46,13 +46,17 @@ struct sk_state {
     int sm_count = 148;
     size_t l2_bytes = 0;
     int64_t worker_chunk = 0;
+    int64_t sketch_ctas_per_sm = 64;
     bool timing = false;
     cudaStream_t stream = nullptr;
     // device memory owned by the handle
     float *m = nullptr, *e = nullptr, *v = nullptr, *vhat = nullptr, *tables = nullptr, *sum = nullptr;
-    uint32_t *vstamp = nullptr, *I = nullptr, *I_prev = nullptr, *hist = nullptr;
+    uint32_t *vstamp = nullptr, *I = nullptr, *I_prev = nullptr, *hist = nullptr, *hist2 = nullptr;
+    uint32_t *keys = nullptr, *bitmap = nullptr;
+    float* gsum = nullptr;
+    uint64_t bitmap_bytes = 0;
     sk::Select* sel = nullptr;
-    sk::Cand* cand = nullptr;
+    sk::Cand *cand = nullptr, *cand2 = nullptr;
     float *stage_grads = nullptr, *stage_x = nullptr;
     // timing
     std::vector<TimeRec> recs;
@@ -136,20 +140,24 @@ int do_step(sk_state* s, const float* grads, float* x) {
     const uint32_t t = (uint32_t)(s->t + 1);
     if (s->timing && s->recs.size() > 4096) { int rc = flush_timing(s); if (rc) return rc; }
 
-    {   // v, vhat on I_{t-1}
-        StageTimer tm(s, 1);
-        tm.done(sk::launch_second_moment(P, grads, s->v, s->vhat, s->vstamp, s->I_prev, s->k_prev, t, st));
-    }
+    sk::MomentArgs A{};
+    A.grads = grads; A.m = s->m; A.e = s->e; A.tables = s->tables; A.gsum = s->gsum;
+    A.v = s->v; A.vhat = s->vhat; A.vstamp = s->vstamp; A.bitmap = s->bitmap;
+    A.step = t; A.members = s->k_prev ? 1u : 0u;
     const uint32_t wc = chunk_of(s);
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
         const uint32_t nw = std::min(wc, P.n - w0);
         {
             StageTimer tm(s, 0);
-            tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats, st));
+            tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats * 4, st));
         }
-        StageTimer tm(s, 2);
-        tm.done(sk::launch_moment_sketch(P, grads, s->m, s->e, s->tables, w0, nw, vec, s->sm_count, st));
+        StageTimer tm(s, 2);     // moments + sketch; also leaves the gradient sums on I_{t-1} in gsum
+        tm.done(sk::launch_moment_sketch(P, A, w0, nw, vec, s->sm_count * (int)s->sketch_ctas_per_sm, st));
+    }
+    {   // v, vhat on I_{t-1} from those sums
+        StageTimer tm(s, 1);
+        tm.done(sk::launch_second_moment(P, A, s->I_prev, s->k_prev, st));
     }
     {
         StageTimer tm(s, 3);
@@ -157,21 +165,23 @@ int do_step(sk_state* s, const float* grads, float* x) {
     }
     {
         StageTimer tm(s, 4);
-        int l = sk::launch_unsketch_hist(P, s->sum, s->vhat, s->hist, vec, s->sm_count, st);
-        l += sk::launch_pick_bin(P, s->hist, s->sel, st);
+        int l = sk::launch_unsketch_hist(P, s->sum, s->vhat, s->keys, s->hist, vec, s->sm_count, st);
+        l += sk::launch_pick_bin(P, s->hist, s->sel, 0, st);
         tm.done(l);
     }
     {
         StageTimer tm(s, 5);
-        tm.done(sk::launch_unsketch_emit(P, s->sum, s->vhat, s->sel, s->I, s->cand, vec, s->sm_count, st));
+        tm.done(sk::launch_emit(P, s->keys, s->sel, s->I, s->cand, s->hist2, s->sm_count, st));
     }
     {
         StageTimer tm(s, 6);
-        tm.done(sk::launch_refine(P, s->sel, s->cand, s->I, st));
+        tm.done(sk::launch_refine(P, s->sel, s->cand, s->cand2, s->hist2, s->I, s->sm_count, st));
     }
     {
-        StageTimer tm(s, 7);
-        tm.done(sk::launch_apply(P, s->I, s->vhat, s->e, x, st));
+        StageTimer tm(s, 7);     // the bitmap of I_{t-1} has served its purpose: clear it, then apply marks I_t
+        int l = sk::launch_zero(s->bitmap, s->bitmap_bytes, st);
+        l += sk::launch_apply(P, s->I, s->vhat, s->e, x, s->bitmap, st);
+        tm.done(l);
     }
     SK_CUDA(cudaGetLastError());
     std::swap(s->I, s->I_prev);      // I_prev now holds I_t
@@ -239,12 +249,19 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     alloc((void**)&s->tables, (uint64_t)n * tf * 4); alloc((void**)&s->sum, tf * 4);
     alloc((void**)&s->I, k * 4); alloc((void**)&s->I_prev, k * 4);
     alloc((void**)&s->hist, sk::kHistBins * 4); alloc((void**)&s->sel, sizeof(sk::Select));
-    alloc((void**)&s->cand, d * sizeof(sk::Cand));
+    alloc((void**)&s->hist2, sk::kHistBins * 4);
+    alloc((void**)&s->cand, d * sizeof(sk::Cand)); alloc((void**)&s->cand2, d * sizeof(sk::Cand));
+    const uint64_t d_pad = (d + 3) / 4 * 4;
+    s->bitmap_bytes = ((d + 31) / 32 * 4 + 15) / 16 * 16;
+    alloc((void**)&s->keys, d_pad * 4); alloc((void**)&s->gsum, d_pad * 4);
+    alloc((void**)&s->bitmap, s->bitmap_bytes);
     if (!ok) { sk_destroy(s); return nullptr; }
+    cudaMemset(s->bitmap, 0, s->bitmap_bytes);                          // I_0 is empty
     cudaMemset(s->m, 0, nd * 4); cudaMemset(s->e, 0, nd * 4);           // m_0 = e_0 = 0
     cudaMemset(s->vstamp, 0, d * 4);
     cudaMemset(s->tables, 0, (uint64_t)n * tf * 4); cudaMemset(s->sum, 0, tf * 4);
-    cudaMemset(s->hist, 0, sk::kHistBins * 4); cudaMemset(s->sel, 0, sizeof(sk::Select));
+    cudaMemset(s->hist, 0, sk::kHistBins * 4); cudaMemset(s->hist2, 0, sk::kHistBins * 4);
+    cudaMemset(s->sel, 0, sizeof(sk::Select));
     uint32_t eps_bits;
     memcpy(&eps_bits, &eps, 4);
     sk::launch_fill_u32((uint32_t*)s->v, d, eps_bits, nullptr);         // v_0 = vhat_0 = eps
@@ -261,7 +278,8 @@ void sk_destroy(sk_state* s) {
     if (!s) return;
     if (s->stream) cudaStreamSynchronize(s->stream); else cudaDeviceSynchronize();
     for (void* p : {(void*)s->m, (void*)s->e, (void*)s->v, (void*)s->vhat, (void*)s->vstamp, (void*)s->tables,
-                    (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->sel, (void*)s->cand,
+                    (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->hist2, (void*)s->sel, (void*)s->cand, (void*)s->cand2,
+                    (void*)s->keys, (void*)s->gsum, (void*)s->bitmap,
                     (void*)s->stage_grads, (void*)s->stage_x})
         if (p) cudaFree(p);
     for (const TimeRec& r : s->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -319,6 +337,11 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         s->worker_chunk = value;
         return SK_OK;
     }
+    if (!strcmp(key, "sketch_ctas_per_sm")) {
+        if (value < 1 || value > 4096) return fail(SK_EINVAL, "sketch_ctas_per_sm must be in 1..4096");
+        s->sketch_ctas_per_sm = value;
+        return SK_OK;
+    }
     if (!strcmp(key, "timing")) {
         int rc = flush_timing(s);
         if (rc) return rc;
@@ -333,6 +356,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     if (!strcmp(key, "log2g")) *value = s->P.log2g;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
+    else if (!strcmp(key, "sketch_ctas_per_sm")) *value = s->sketch_ctas_per_sm;
     else if (!strcmp(key, "I_count")) *value = s->k_prev;
     else if (!strcmp(key, "vectorised")) *value = (s->P.d % 4 == 0) && s->P.log2g >= 2;
     else return fail(SK_EINVAL, "unknown option '%s'", key);

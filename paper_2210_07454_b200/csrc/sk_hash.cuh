@@ -27,14 +27,19 @@ struct GroupHash {
     uint32_t signs;  // bit o set  <=>  coordinate with offset o carries sign -1
 };
 
-__device__ __forceinline__ GroupHash group_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t q) {
-    const uint64_t u1 = stream(key, 2ull * q + 1);
-    const uint64_t u2 = stream(key, 2ull * q + 2);
+// from one 64-bit draw u: high word -> bucket group by multiply-high range reduction, the leading bits of the
+// remainder -> xor permutation, low word -> sign bits
+__device__ __forceinline__ GroupHash group_from_draw(uint64_t u, uint32_t log2g, uint32_t G) {
+    const uint32_t hi = (uint32_t)(u >> 32);
     GroupHash h;
-    h.base = __umulhi((uint32_t)(u1 >> 32), G) << log2g;
-    h.perm = (uint32_t)(u2 >> 32) & ((1u << log2g) - 1u);
-    h.signs = (uint32_t)u1;
+    h.base = __umulhi(hi, G) << log2g;
+    h.perm = log2g ? ((hi * G) >> (32u - log2g)) : 0u;
+    h.signs = (uint32_t)u;
     return h;
+}
+
+__device__ __forceinline__ GroupHash group_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t q) {
+    return group_from_draw(stream(key, (uint64_t)q + 1), log2g, G);
 }
 
 // Scalar form: bucket and sign (+1/-1) of coordinate i.
@@ -61,6 +66,49 @@ __device__ __forceinline__ Quad quad_hash(uint64_t key, uint32_t log2g, uint32_t
     r.off = h.base + ((o ^ h.perm) & ~3u);
     r.p3sgn = (h.perm & 3u) | (((h.signs >> o) & 0xFu) << 2);
     return r;
+}
+
+__device__ __forceinline__ Quad quad_from_draw(uint64_t u, uint32_t log2g, uint32_t G, uint32_t i) {
+    const uint32_t o = i & ((1u << log2g) - 1u);
+    const GroupHash h = group_from_draw(u, log2g, G);
+    Quad r;
+    r.off = h.base + ((o ^ h.perm) & ~3u);
+    r.p3sgn = (h.perm & 3u) | (((h.signs >> o) & 0xFu) << 2);
+    return r;
+}
+
+// Hashes of coordinate quad t (coordinates 4t..4t+3) in rows 0..r-1.  With g = 32 the eight lanes that share a
+// group split the rows between them (one 64-bit draw per lane and round) and exchange the draws by shuffle, so
+// ALL 32 LANES OF THE WARP MUST CALL THIS TOGETHER (callers clamp t for lanes past the end).
+template <int RMAX>
+__device__ __forceinline__ void quad_hashes(const uint64_t* __restrict__ row_key /* param space */, uint32_t r,
+                                            uint32_t log2g, uint32_t G, uint32_t t, Quad (&h)[RMAX]) {
+    if (log2g == 5) {
+        const uint32_t lane = threadIdx.x & 31u, li = lane & 7u, q = t >> 3;
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)RMAX; k += 8) {
+            if (k < r) {
+                uint64_t key = 0;
+#pragma unroll
+                for (uint32_t j = 0; j < 8; ++j)
+                    if (k + j < (uint32_t)RMAX && j == li) key = row_key[k + j];
+                const uint64_t u = (k + li < r) ? stream(key, (uint64_t)q + 1) : 0ull;
+                const uint32_t hi = (uint32_t)(u >> 32), lo = (uint32_t)u;
+#pragma unroll
+                for (uint32_t j = 0; j < 8; ++j)
+                    if (k + j < (uint32_t)RMAX && k + j < r) {
+                        const uint32_t src = (lane & ~7u) + j;
+                        const uint32_t ohi = __shfl_sync(0xFFFFFFFFu, hi, src);
+                        const uint32_t olo = __shfl_sync(0xFFFFFFFFu, lo, src);
+                        h[k + j] = quad_from_draw(((uint64_t)ohi << 32) | olo, 5, G, t << 2);
+                    }
+            }
+        }
+    } else {
+#pragma unroll
+        for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+            if (row < r) h[row] = quad_hash(row_key[row], log2g, G, t << 2);
+    }
 }
 
 __device__ __forceinline__ float flip(float a, uint32_t bit) {  // a * (bit ? -1 : +1)

@@ -26,32 +26,51 @@ struct Select {
     uint32_t need;       // how many candidates of the threshold bin are still to be taken
     uint32_t cnt_out;    // indices emitted so far
     uint32_t cnt_cand;   // candidates collected
-    uint32_t status;     // 0 ok; bit 0: emitted count != k; bit 1: candidate overflow
-    uint32_t pad[3];
+    uint32_t status;     // 0 ok; bit 0: emitted count != k
+    uint32_t bin2;       // second-level threshold bin (key bits 18..7) inside `bin`
+    uint32_t need2;      // how many of the candidates sharing the threshold's first 24 key bits are to be taken
+    uint32_t cnt_cand2;  // candidates sharing the threshold's first 24 key bits
 };
 
 struct Cand { uint32_t key, idx; };
 
+// Pointers of the moment + sketch kernel (all device memory).
+struct MomentArgs {
+    const float* grads;
+    float *m, *e, *tables;
+    float* gsum;             // running gradient sums on I_{t-1} when the workers are processed in several launches
+    float *v, *vhat;
+    uint32_t* vstamp;        // step at which v[j] was last brought up to date
+    const uint32_t* bitmap;  // membership of I_{t-1}: bit j of word j/32
+    uint32_t step;           // t (1-based)
+    uint32_t members;        // 0 when I_{t-1} is empty
+};
+
 // Launchers.  Each enqueues on `st` and returns the number of kernels it launched.
-int launch_zero(float* p, uint64_t nfloats, cudaStream_t st);
-int launch_second_moment(const Params& P, const float* grads, float* v, float* vhat, uint32_t* vstamp,
-                         const uint32_t* I_prev, uint32_t k_prev, uint32_t t, cudaStream_t st);
-int launch_moment_sketch(const Params& P, const float* grads, float* m, float* e, float* tables,
-                         uint32_t w0, uint32_t nw, bool vec, int sm_count, cudaStream_t st);
+int launch_zero(void* p, uint64_t bytes, cudaStream_t st);
+int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st);
+int launch_set_bits(const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st);
+int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,
+                         cudaStream_t st);
+int launch_second_moment(const Params& P, const MomentArgs& A, const uint32_t* I_prev, uint32_t k_prev,
+                         cudaStream_t st);
 int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStream_t st);
-int launch_unsketch_hist(const Params& P, const float* sum, const float* vhat, uint32_t* hist, bool vec,
-                         int sm_count, cudaStream_t st);
-int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, cudaStream_t st);
-int launch_unsketch_emit(const Params& P, const float* sum, const float* vhat, Select* sel, uint32_t* I_out,
-                         Cand* cand, bool vec, int sm_count, cudaStream_t st);
-int launch_refine(const Params& P, Select* sel, const Cand* cand, uint32_t* I_out, cudaStream_t st);
-int launch_apply(const Params& P, const uint32_t* I, const float* vhat, float* e, float* x, cudaStream_t st);
+int launch_unsketch_hist(const Params& P, const float* sum, const float* vhat, uint32_t* keys, uint32_t* hist,
+                         bool vec, int sm_count, cudaStream_t st);
+int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cudaStream_t st);
+int launch_emit(const Params& P, const uint32_t* keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2,
+                int sm_count, cudaStream_t st);
+int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
+                  int sm_count, cudaStream_t st);
+int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, float* x, uint32_t* bitmap,
+                 cudaStream_t st);
 // helpers for state export / import
 int launch_estimates(const Params& P, const float* sum, const float* vhat, float* est, cudaStream_t st);
 int launch_hash_export(const Params& P, uint32_t row, uint64_t i0, uint64_t count, uint32_t* idx, int8_t* sgn,
                        cudaStream_t st);
 int launch_v_materialize(const Params& P, const float* v, const uint32_t* vstamp, uint32_t t, float* out,
                          cudaStream_t st);
-int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st);
+int launch_masked_copy(const Params& P, const float* e, const uint32_t* bitmap, uint32_t workers, float* out,
+                       cudaStream_t st);
 
 }  // namespace sk

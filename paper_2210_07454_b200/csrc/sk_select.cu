@@ -2,9 +2,12 @@
 // vhat^{-1/2} (Algorithm 3), select the k largest magnitudes (Algorithm 2, "Top-k"), and apply the update with
 // the exact worker means on I_t together with the error-feedback reset.
 //
-// Selection never stores the d estimates: they are recomputed from the L2-resident aggregate sketch in two
-// streaming passes (histogram of the top key bits, then emit-above-threshold + collect-threshold-bin), and
-// the small candidate list of the threshold bin is resolved exactly by one thread block.
+// Selection: (A) one pass over the coordinates computes every ranking key from the L2-resident aggregate sketch,
+// stores it (4 bytes per coordinate) and histograms key bits 30..19; (B) one pass over the stored keys emits the
+// indices above the threshold bin, collects the threshold bin's candidates and histograms their next 12 key
+// bits; (C) the candidates are split once more and (D) the handful that share the first 24 key bits with the
+// threshold are resolved exactly by one block.
+// key = bit pattern of |estimate| (monotone for finite non-negative floats); ties go to the smaller index.
 #include "sk_internal.h"
 #include "sk_hash.cuh"
 
@@ -14,17 +17,33 @@ namespace {
 
 constexpr int kThreads = 256;
 
-// lower median of r values held in registers: ascending compare-exchange sort, element (r-1)/2
+// ---- median of r values held in registers (lower median for even r) ----------------------------------------
+__device__ __forceinline__ float med3(float x, float y, float z) {
+    return fmaxf(fminf(x, y), fminf(fmaxf(x, y), z));
+}
+
 template <int R>
 __device__ __forceinline__ float median_fixed(float (&q)[R]) {
+    if constexpr (R == 1) return q[0];
+    else if constexpr (R == 2) return fminf(q[0], q[1]);
+    else if constexpr (R == 3) return med3(q[0], q[1], q[2]);
+    else if constexpr (R == 5) {
+        // the median of five is the median of: the larger of the two pair-minima, the smaller of the two
+        // pair-maxima, and the fifth element
+        const float f = fmaxf(fminf(q[0], q[1]), fminf(q[2], q[3]));
+        const float g = fminf(fmaxf(q[0], q[1]), fmaxf(q[2], q[3]));
+        return med3(q[4], f, g);
+    } else {
+        // bubble passes until position (R-1)/2 is final
 #pragma unroll
-    for (int a = 0; a < R - 1; ++a)
+        for (int a = 0; a < R - (R - 1) / 2; ++a)
 #pragma unroll
-        for (int b = 0; b < R - 1 - a; ++b) {
-            const float lo = fminf(q[b], q[b + 1]), hi = fmaxf(q[b], q[b + 1]);
-            q[b] = lo; q[b + 1] = hi;
-        }
-    return q[(R - 1) / 2];
+            for (int b = 0; b < R - 1 - a; ++b) {
+                const float lo = fminf(q[b], q[b + 1]), hi = fmaxf(q[b], q[b + 1]);
+                q[b] = lo; q[b + 1] = hi;
+            }
+        return q[(R - 1) / 2];
+    }
 }
 
 __device__ __forceinline__ float median_any(float* q, uint32_t r) {
@@ -37,111 +56,130 @@ __device__ __forceinline__ float median_any(float* q, uint32_t r) {
     return q[(r - 1) / 2];
 }
 
+// est = med / sqrt(vhat), both operations correctly rounded (this is the value the selection is defined on)
 __device__ __forceinline__ float scale_est(float med, float vhat) { return __fdiv_rn(med, __fsqrt_rn(vhat)); }
+__device__ __forceinline__ uint32_t key_of(float est) { return __float_as_uint(est) & 0x7FFFFFFFu; }
 
-// estimates of the 4 coordinates 4t..4t+3 (vector form, g >= 4)
+// Ranking key of a coordinate: the bit pattern of |med * rsqrt(vhat)|.  The hardware reciprocal square root is
+// within 2 ulp, so the key is within a few ulp (< 4e-7 relative) of the correctly rounded estimate -- two orders
+// of magnitude inside the tolerance within which the selected set is defined -- and it is a deterministic
+// function of (med, vhat), which is all the selection needs.  Denormal vhat takes the exact path.
+__device__ __forceinline__ uint32_t key_rank(float med, float vhat) {
+    return key_of(vhat > 1e-30f ? med * rsqrtf(vhat) : scale_est(med, vhat));
+}
+
+// medians of the 4 coordinates 4t..4t+3 (vector form, g >= 4).  All lanes of the warp call this together.
 template <int R>
-__device__ __forceinline__ float4 estimate4(const Params& P, const float* __restrict__ sum, uint32_t t,
-                                            float4 vh) {
+__device__ __forceinline__ float4 medians4(const Params& P, const float* __restrict__ sum, uint32_t t) {
+    constexpr int RMAX = R > 0 ? R : (int)kMaxRows;
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
-    float qx[R > 0 ? R : (int)kMaxRows], qy[R > 0 ? R : (int)kMaxRows];
-    float qz[R > 0 ? R : (int)kMaxRows], qw[R > 0 ? R : (int)kMaxRows];
+    Quad h[RMAX];
+    quad_hashes<RMAX>(P.row_key, r, P.log2g, P.G, t, h);
+    float qx[RMAX], qy[RMAX], qz[RMAX], qw[RMAX];
 #pragma unroll
-    for (uint32_t row = 0; row < r; ++row) {
-        const Quad h = quad_hash(P.row_key[row], P.log2g, P.G, t << 2);
-        float4 cch = __ldg((const float4*)(sum + (uint64_t)row * P.cs + h.off));
-        cch = quad_gather(h, cch);
-        qx[row] = cch.x; qy[row] = cch.y; qz[row] = cch.z; qw[row] = cch.w;
-    }
-    float4 est;
+    for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+        if (row < r) {
+            float4 cch = __ldg((const float4*)(sum + (uint64_t)row * P.cs + h[row].off));
+            cch = quad_gather(h[row], cch);
+            qx[row] = cch.x; qy[row] = cch.y; qz[row] = cch.z; qw[row] = cch.w;
+        }
+    float4 med;
     if constexpr (R > 0) {
-        est.x = median_fixed(qx); est.y = median_fixed(qy); est.z = median_fixed(qz); est.w = median_fixed(qw);
+        med.x = median_fixed(qx); med.y = median_fixed(qy); med.z = median_fixed(qz); med.w = median_fixed(qw);
     } else {
-        est.x = median_any(qx, r); est.y = median_any(qy, r); est.z = median_any(qz, r); est.w = median_any(qw, r);
+        med.x = median_any(qx, r); med.y = median_any(qy, r); med.z = median_any(qz, r); med.w = median_any(qw, r);
     }
-    est.x = scale_est(est.x, vh.x); est.y = scale_est(est.y, vh.y);
-    est.z = scale_est(est.z, vh.z); est.w = scale_est(est.w, vh.w);
-    return est;
+    return med;
 }
 
 // scalar form, any group size / alignment
-__device__ __forceinline__ float estimate1(const Params& P, const float* __restrict__ sum, uint32_t j, float vh) {
+__device__ __forceinline__ float median1(const Params& P, const float* __restrict__ sum, uint32_t j) {
     float q[kMaxRows];
     for (uint32_t row = 0; row < P.r; ++row) {
         uint32_t b; float s;
         coord_hash(P.row_key[row], P.log2g, P.G, j, b, s);
         q[row] = s * __ldg(sum + (uint64_t)row * P.cs + b);
     }
-    return scale_est(median_any(q, P.r), vh);
+    return median_any(q, P.r);
 }
 
-__device__ __forceinline__ uint32_t key_of(float est) { return __float_as_uint(est) & 0x7FFFFFFFu; }
-
-// ---- pass A: histogram of key bits 30..19 ------------------------------------------------------------
+// ---- pass A: ranking keys of all coordinates (stored) + histogram of key bits 30..19 -----------------------------
 template <int R, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_unsketch_hist(const __grid_constant__ Params P, const float* __restrict__ sum, const float* __restrict__ vhat,
-                uint32_t* hist) {
+                uint32_t* keys, uint32_t* hist) {
     __shared__ uint32_t sh[kHistBins];
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh[b] = 0;
     __syncthreads();
-    if (VEC) {
-        const uint32_t d4 = P.d >> 2;
-        for (uint32_t t = blockIdx.x * kThreads + threadIdx.x; t < d4; t += gridDim.x * kThreads) {
-            const float4 est = estimate4<R>(P, sum, t, __ldcs((const float4*)vhat + t));
-            atomicAdd(&sh[key_of(est.x) >> kHistShift], 1u);
-            atomicAdd(&sh[key_of(est.y) >> kHistShift], 1u);
-            atomicAdd(&sh[key_of(est.z) >> kHistShift], 1u);
-            atomicAdd(&sh[key_of(est.w) >> kHistShift], 1u);
+    const uint32_t items = VEC ? (P.d >> 2) : P.d;
+    const uint32_t trips = (items + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
+    for (uint32_t it = 0; it < trips; ++it) {                // uniform trip count: warps stay whole
+        const uint32_t t = (it * gridDim.x + blockIdx.x) * kThreads + threadIdx.x;
+        const bool live = t < items;
+        const uint32_t tc = live ? t : items - 1;
+        if (VEC) {
+            const float4 med = medians4<R>(P, sum, tc);
+            if (live) {
+                const float4 vh = __ldcs((const float4*)vhat + t);
+                uint4 k4;
+                k4.x = key_rank(med.x, vh.x); k4.y = key_rank(med.y, vh.y);
+                k4.z = key_rank(med.z, vh.z); k4.w = key_rank(med.w, vh.w);
+                ((uint4*)keys)[t] = k4;
+                atomicAdd(&sh[k4.x >> kHistShift], 1u); atomicAdd(&sh[k4.y >> kHistShift], 1u);
+                atomicAdd(&sh[k4.z >> kHistShift], 1u); atomicAdd(&sh[k4.w >> kHistShift], 1u);
+            }
+        } else if (live) {
+            const uint32_t key = key_rank(median1(P, sum, t), vhat[t]);
+            keys[t] = key;
+            atomicAdd(&sh[key >> kHistShift], 1u);
         }
-    } else {
-        for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads)
-            atomicAdd(&sh[key_of(estimate1(P, sum, j, vhat[j])) >> kHistShift], 1u);
     }
     __syncthreads();
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
         if (sh[b]) atomicAdd(&hist[b], sh[b]);
 }
 
-// ---- threshold bin: largest b with count(bins >= b) >= k; clears the histogram for the next step ----------
-__global__ void __launch_bounds__(1024) k_pick_bin(uint32_t k, uint32_t* hist, Select* sel) {
+// ---- threshold bin of a 4096-bin histogram: largest b with count(bins >= b) >= need ------------------------
+// level 0: need = k, result -> sel->bin/need, counters reset.  level 1: need = sel->need, result -> bin2/need2.
+__global__ void __launch_bounds__(1024) k_pick_bin(uint32_t k, uint32_t* hist, Select* sel, int level) {
     __shared__ uint32_t part[1024];
     constexpr uint32_t per = kHistBins / 1024;
+    const uint32_t need = level == 0 ? k : sel->need;
     uint32_t mine[per];
     uint32_t s = 0;
-    // thread i owns bins in DESCENDING order: its first bin is kHistBins-1 - i*per
-    const uint32_t top = kHistBins - 1 - threadIdx.x * per;
+    const uint32_t top = kHistBins - 1 - threadIdx.x * per;   // thread i owns `per` bins in descending order
 #pragma unroll
     for (uint32_t q = 0; q < per; ++q) { mine[q] = hist[top - q]; hist[top - q] = 0; s += mine[q]; }
     part[threadIdx.x] = s;
     __syncthreads();
-    for (uint32_t off = 1; off < 1024; off <<= 1) {       // inclusive scan over threads (descending bins)
+    for (uint32_t off = 1; off < 1024; off <<= 1) {
         const uint32_t add = threadIdx.x >= off ? part[threadIdx.x - off] : 0;
         __syncthreads();
         part[threadIdx.x] += add;
         __syncthreads();
     }
-    uint32_t above = part[threadIdx.x] - s;               // keys in bins above this thread's first bin
+    uint32_t above = part[threadIdx.x] - s;
 #pragma unroll
     for (uint32_t q = 0; q < per; ++q) {
-        if (above < k && above + mine[q] >= k) {
-            sel->bin = top - q;
-            sel->need = k - above;
-            sel->cnt_out = 0;
-            sel->cnt_cand = 0;
+        if (above < need && above + mine[q] >= need) {
+            if (level == 0) {
+                sel->bin = top - q; sel->need = need - above;
+                sel->cnt_out = 0; sel->cnt_cand = 0; sel->cnt_cand2 = 0;
+            } else {
+                sel->bin2 = top - q; sel->need2 = need - above;
+            }
         }
         above += mine[q];
     }
 }
 
-// ---- pass B: emit indices above the threshold bin, collect the threshold bin's candidates -----------------
-// Block-aggregated appends: one atomic per block-iteration and list.
-__device__ __forceinline__ void block_append(uint32_t n_out, uint32_t n_cand, uint32_t* cnt_out, uint32_t* cnt_cand,
-                                             uint32_t& base_out, uint32_t& base_cand) {
+// Block-aggregated appends to two lists: one atomic per block-iteration and list.
+__device__ __forceinline__ void block_append(uint32_t n_a, uint32_t n_b, uint32_t* cnt_a, uint32_t* cnt_b,
+                                             uint32_t& base_a, uint32_t& base_b) {
     __shared__ uint32_t warp_tot[kThreads / 32];
     __shared__ uint32_t block_base[2];
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    uint32_t packed = n_out | (n_cand << 16);              // each <= 4 per thread, <= 1024 per block
+    const uint32_t packed = n_a | (n_b << 16);              // each <= 4 per thread, <= 1024 per block
     uint32_t incl = packed;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -158,33 +196,37 @@ __device__ __forceinline__ void block_append(uint32_t n_out, uint32_t n_cand, ui
         total += wtot;
     }
     if (threadIdx.x == 0) {
-        block_base[0] = (total & 0xFFFFu) ? atomicAdd(cnt_out, total & 0xFFFFu) : 0u;
-        block_base[1] = (total >> 16) ? atomicAdd(cnt_cand, total >> 16) : 0u;
+        block_base[0] = (total & 0xFFFFu) ? atomicAdd(cnt_a, total & 0xFFFFu) : 0u;
+        block_base[1] = (total >> 16) ? atomicAdd(cnt_b, total >> 16) : 0u;
     }
     __syncthreads();
     const uint32_t excl = before + incl - packed;
-    base_out = block_base[0] + (excl & 0xFFFFu);
-    base_cand = block_base[1] + (excl >> 16);
-    __syncthreads();                                       // shared scratch is reused by the next iteration
+    base_a = block_base[0] + (excl & 0xFFFFu);
+    base_b = block_base[1] + (excl >> 16);
+    __syncthreads();                                        // the shared scratch is reused by the next call
 }
 
-template <int R, bool VEC>
+// ---- pass B over the stored keys: emit above the threshold bin, collect the threshold bin, histogram its next
+// 12 key bits ---------------------------------------------------------------------------------------------------
+template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
-k_unsketch_emit(const __grid_constant__ Params P, const float* __restrict__ sum, const float* __restrict__ vhat,
-                Select* sel, uint32_t* I_out, Cand* cand) {
+k_emit(uint32_t d, const uint32_t* __restrict__ keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2) {
+    __shared__ uint32_t sh2[kHistBins];
+    for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh2[b] = 0;
+    __syncthreads();
     const uint32_t bin = sel->bin;
-    const uint32_t items = VEC ? (P.d >> 2) : P.d;
+    const uint32_t items = VEC ? (d >> 2) : d;
     const uint32_t trips = (items + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
-    for (uint32_t it = 0; it < trips; ++it) {               // uniform trip count: the block scans need all threads
+    for (uint32_t it = 0; it < trips; ++it) {
         const uint32_t t = (it * gridDim.x + blockIdx.x) * kThreads + threadIdx.x;
-        uint32_t keys[4], idx0 = VEC ? (t << 2) : t, nk = 0;
+        uint32_t kq[4], idx0 = VEC ? (t << 2) : t, nk = 0;
         if (t < items) {
             if (VEC) {
-                const float4 est = estimate4<R>(P, sum, t, __ldcs((const float4*)vhat + t));
-                keys[0] = key_of(est.x); keys[1] = key_of(est.y); keys[2] = key_of(est.z); keys[3] = key_of(est.w);
+                const uint4 k4 = __ldcs((const uint4*)keys + t);
+                kq[0] = k4.x; kq[1] = k4.y; kq[2] = k4.z; kq[3] = k4.w;
                 nk = 4;
             } else {
-                keys[0] = key_of(estimate1(P, sum, t, vhat[t]));
+                kq[0] = keys[t];
                 nk = 1;
             }
         }
@@ -192,45 +234,72 @@ k_unsketch_emit(const __grid_constant__ Params P, const float* __restrict__ sum,
 #pragma unroll
         for (uint32_t q = 0; q < 4; ++q)
             if (q < nk) {
-                const uint32_t b = keys[q] >> kHistShift;
+                const uint32_t b = kq[q] >> kHistShift;
+                if (b == bin) { atomicAdd(&sh2[(kq[q] >> 7) & (kHistBins - 1u)], 1u); ++n_cand; }
                 n_out += b > bin;
-                n_cand += b == bin;
             }
         uint32_t po, pc;
         block_append(n_out, n_cand, &sel->cnt_out, &sel->cnt_cand, po, pc);
 #pragma unroll
         for (uint32_t q = 0; q < 4; ++q)
             if (q < nk) {
-                const uint32_t b = keys[q] >> kHistShift;
+                const uint32_t b = kq[q] >> kHistShift;
                 if (b > bin) I_out[po++] = idx0 + q;
-                else if (b == bin) { cand[pc].key = keys[q]; cand[pc].idx = idx0 + q; ++pc; }
+                else if (b == bin) { cand[pc].key = kq[q]; cand[pc].idx = idx0 + q; ++pc; }
             }
+    }
+    __syncthreads();
+    for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
+        if (sh2[b]) atomicAdd(&hist2[b], sh2[b]);
+}
+
+// ---- pass C over the candidates: first 24 key bits above the threshold -> emit, equal -> second list ----------
+__global__ void __launch_bounds__(kThreads)
+k_split_candidates(Select* sel, const Cand* __restrict__ cand, uint32_t* I_out, Cand* cand2) {
+    const uint32_t ncand = sel->cnt_cand;
+    const uint32_t thr = (sel->bin << kHistBits) | sel->bin2;          // leading 24 bits of the threshold key
+    const uint32_t trips = (ncand + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
+    for (uint32_t it = 0; it < trips; ++it) {
+        const uint32_t q = (it * gridDim.x + blockIdx.x) * kThreads + threadIdx.x;
+        Cand cnd{0u, 0u};
+        uint32_t n_out = 0, n_eq = 0;
+        if (q < ncand) {
+            cnd = cand[q];
+            const uint32_t lead = cnd.key >> 7;
+            n_out = lead > thr;
+            n_eq = lead == thr;
+        }
+        uint32_t po, pc;
+        block_append(n_out, n_eq, &sel->cnt_out, &sel->cnt_cand2, po, pc);
+        if (n_out) I_out[po] = cnd.idx;
+        if (n_eq) cand2[pc] = cnd;
     }
 }
 
-// ---- refinement: of the candidates in the threshold bin take the `need` largest (key, then smaller index) ----
-// Radix select, one block, on the 51-bit composite (key bits 18..0 , ~idx): all composites are distinct, so the
-// selection is exact and ties in the key go to the smaller index.
-__global__ void __launch_bounds__(1024) k_refine(uint32_t k, Select* sel, const Cand* __restrict__ cand,
-                                                 uint32_t* I_out) {
+// ---- pass D: of the second list take the `need2` largest by (last 7 key bits, then smaller index) -------------
+// Radix select by one block on the 39-bit composite (key & 127, ~idx): all composites are distinct, so the
+// selection is exact and equal keys go to the smaller index.
+__global__ void __launch_bounds__(1024) k_resolve(uint32_t k, Select* sel, const Cand* __restrict__ cand2,
+                                                  uint32_t* I_out) {
     constexpr uint32_t W = 11, BINS = 1u << W;
     __shared__ uint32_t hist[BINS];
     __shared__ uint32_t s_bin, s_need, s_done, s_pos;
     __shared__ uint32_t s_wtot[32];
-    const uint32_t ncand = sel->cnt_cand;
-    uint32_t need = sel->need;
-    const uint64_t lowmask = (1ull << kHistShift) - 1;
+    const uint32_t ncand = sel->cnt_cand2;
+    uint32_t need = sel->need2;
     uint64_t prefix = 0;        // composite >> shift must equal prefix for an element to be still undecided
-    int shift = 51;
+    int shift = 39;
     bool exact = false;         // true once every element with composite >= threshold is known to be wanted
+    bool first = true;
     while (shift > 0 && !exact) {
-        const int w = shift >= (int)W ? (int)W : shift;
+        const int w = first ? 7 : (shift >= (int)W ? (int)W : shift);   // the key bits first, then the index
+        first = false;
         shift -= w;
         for (uint32_t b = threadIdx.x; b < BINS; b += blockDim.x) hist[b] = 0;
         __syncthreads();
         for (uint32_t q = threadIdx.x; q < ncand; q += blockDim.x) {
-            const Cand cnd = cand[q];
-            const uint64_t comp = ((uint64_t)(cnd.key & lowmask) << 32) | (uint32_t)~cnd.idx;
+            const Cand cnd = cand2[q];
+            const uint64_t comp = ((uint64_t)(cnd.key & 127u) << 32) | (uint32_t)~cnd.idx;
             if ((comp >> (shift + w)) == prefix) atomicAdd(&hist[(comp >> shift) & ((1u << w) - 1u)], 1u);
         }
         __syncthreads();
@@ -264,17 +333,13 @@ __global__ void __launch_bounds__(1024) k_refine(uint32_t k, Select* sel, const 
     __syncthreads();
     for (uint32_t q0 = 0; q0 < ncand; q0 += blockDim.x) {
         const uint32_t q = q0 + threadIdx.x;
-        bool take = false;
-        uint32_t idx = 0;
         if (q < ncand) {
-            const Cand cnd = cand[q];
-            idx = cnd.idx;
-            const uint64_t comp = ((uint64_t)(cnd.key & lowmask) << 32) | (uint32_t)~cnd.idx;
-            take = comp >= threshold;
-        }
-        if (take) {
-            const uint32_t pos = atomicAdd(&s_pos, 1u);
-            if (pos < k) I_out[pos] = idx;
+            const Cand cnd = cand2[q];
+            const uint64_t comp = ((uint64_t)(cnd.key & 127u) << 32) | (uint32_t)~cnd.idx;
+            if (comp >= threshold) {
+                const uint32_t pos = atomicAdd(&s_pos, 1u);
+                if (pos < k) I_out[pos] = cnd.idx;
+            }
         }
     }
     __syncthreads();
@@ -284,27 +349,35 @@ __global__ void __launch_bounds__(1024) k_refine(uint32_t k, Select* sel, const 
     }
 }
 
-// ---- apply on I_t: x_j -= lr * mean_w a^(w)_j / sqrt(vhat_j) ; e^(w)_j = 0 ----------------------------------
+// ---- apply on I_t: x_j -= lr * mean_w a^(w)_j / sqrt(vhat_j).  The error-feedback reset e^(w)_j = 0 is recorded
+// as a bit in the membership bitmap of I_t, which the next step's moment kernel honours. -----------------------
 __global__ void __launch_bounds__(kThreads)
-k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const float* __restrict__ vhat, float* e,
-        float* x) {
+k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const float* __restrict__ vhat,
+        const float* __restrict__ e, float* x, uint32_t* bitmap) {
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
     if (q >= P.k) return;
     const uint32_t j = I[q];
     float abar = 0.0f;
-#pragma unroll 4
-    for (uint32_t w = 0; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
+    uint32_t w = 0;
+    for (; w + 8 <= P.n; w += 8) {                           // eight independent gathers in flight, added in order
+        float a[8];
+#pragma unroll
+        for (uint32_t u = 0; u < 8; ++u) a[u] = e[(uint64_t)(w + u) * P.d + j];
+#pragma unroll
+        for (uint32_t u = 0; u < 8; ++u) abar += a[u];
+    }
+    for (; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
     abar = abar / (float)P.n;
     const float delta = scale_est(abar, vhat[j]);
     x[j] = x[j] - P.lr * delta;
-    for (uint32_t w = 0; w < P.n; ++w) e[(uint64_t)w * P.d + j] = 0.0f;
+    atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
 }
 
 __global__ void __launch_bounds__(kThreads)
 k_estimates(const __grid_constant__ Params P, const float* __restrict__ sum, const float* __restrict__ vhat,
             float* est) {
     for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads)
-        est[j] = estimate1(P, sum, j, vhat[j]);
+        est[j] = scale_est(median1(P, sum, j), vhat[j]);
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -340,40 +413,40 @@ inline int grid_for(uint64_t items, int sm_count, int per_sm) {
         default: KERNEL<0, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                           \
     }
 
-int launch_unsketch_hist(const Params& P, const float* sum, const float* vhat, uint32_t* hist, bool vec,
-                         int sm_count, cudaStream_t st) {
+int launch_unsketch_hist(const Params& P, const float* sum, const float* vhat, uint32_t* keys, uint32_t* hist,
+                         bool vec, int sm_count, cudaStream_t st) {
     if (!vec) {
-        k_unsketch_hist<0, false><<<grid_for(P.d, sm_count, 4), kThreads, 0, st>>>(P, sum, vhat, hist);
+        k_unsketch_hist<0, false><<<grid_for(P.d, sm_count, 6), kThreads, 0, st>>>(P, sum, vhat, keys, hist);
         return 1;
     }
-    const int grid = grid_for(P.d >> 2, sm_count, 4);
-    SK_ROWS_SWITCH(k_unsketch_hist, P, sum, vhat, hist)
+    const int grid = grid_for(P.d >> 2, sm_count, 6);
+    SK_ROWS_SWITCH(k_unsketch_hist, P, sum, vhat, keys, hist)
     return 1;
 }
 
-int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, cudaStream_t st) {
-    k_pick_bin<<<1, 1024, 0, st>>>(P.k, hist, sel);
+int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cudaStream_t st) {
+    k_pick_bin<<<1, 1024, 0, st>>>(P.k, hist, sel, level);
     return 1;
 }
 
-int launch_unsketch_emit(const Params& P, const float* sum, const float* vhat, Select* sel, uint32_t* I_out,
-                         Cand* cand, bool vec, int sm_count, cudaStream_t st) {
-    if (!vec) {
-        k_unsketch_emit<0, false><<<grid_for(P.d, sm_count, 4), kThreads, 0, st>>>(P, sum, vhat, sel, I_out, cand);
-        return 1;
-    }
-    const int grid = grid_for(P.d >> 2, sm_count, 4);
-    SK_ROWS_SWITCH(k_unsketch_emit, P, sum, vhat, sel, I_out, cand)
+int launch_emit(const Params& P, const uint32_t* keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2,
+                int sm_count, cudaStream_t st) {
+    if (P.d % 4 == 0) k_emit<true><<<grid_for(P.d >> 2, sm_count, 8), kThreads, 0, st>>>(P.d, keys, sel, I_out, cand, hist2);
+    else k_emit<false><<<grid_for(P.d, sm_count, 8), kThreads, 0, st>>>(P.d, keys, sel, I_out, cand, hist2);
     return 1;
 }
 
-int launch_refine(const Params& P, Select* sel, const Cand* cand, uint32_t* I_out, cudaStream_t st) {
-    k_refine<<<1, 1024, 0, st>>>(P.k, sel, cand, I_out);
-    return 1;
+int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
+                  int sm_count, cudaStream_t st) {
+    k_pick_bin<<<1, 1024, 0, st>>>(P.k, hist2, sel, 1);
+    k_split_candidates<<<sm_count, kThreads, 0, st>>>(sel, cand, I_out, cand2);
+    k_resolve<<<1, 1024, 0, st>>>(P.k, sel, cand2, I_out);
+    return 3;
 }
 
-int launch_apply(const Params& P, const uint32_t* I, const float* vhat, float* e, float* x, cudaStream_t st) {
-    k_apply<<<(P.k + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, I, vhat, e, x);
+int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, float* x, uint32_t* bitmap,
+                 cudaStream_t st) {
+    k_apply<<<(P.k + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, I, vhat, e, x, bitmap);
     return 1;
 }
 

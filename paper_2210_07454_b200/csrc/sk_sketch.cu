@@ -1,5 +1,6 @@
-// Dense half of the step: second moments on I_{t-1}, momentum + error-feedback accumulate + Count Sketch of
-// every worker's vector (Algorithm 2, worker side; Section II-C), and the fixed-order sum of the n sketches.
+// Dense half of the step: momentum + error-feedback accumulate + Count Sketch of every worker's vector
+// (Algorithm 2, worker side; Section II-C) fused with the master's second-moment update on I_{t-1}, and the
+// fixed-order sum of the n sketches.
 #include "sk_internal.h"
 #include "sk_hash.cuh"
 
@@ -26,6 +27,11 @@ __global__ void __launch_bounds__(kThreads) k_fill_u32(uint32_t* p, uint64_t n, 
         p[t] = value;
 }
 
+__global__ void __launch_bounds__(kThreads) k_set_bits(const uint32_t* __restrict__ I, uint32_t count, uint32_t* bitmap) {
+    const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
+    if (q < count) atomicOr(&bitmap[I[q] >> 5], 1u << (I[q] & 31u));
+}
+
 // v is kept lazily: vstamp[j] is the step at which v[j] was last brought up to date.  A coordinate outside
 // I_{t-1} only decays, v <- beta2 v (Algorithm 2's v update with h_t = 0 there), and vhat = max(vhat, v) cannot
 // change, so the decays are applied one fp32 multiply per owed step when the coordinate is next touched --
@@ -35,22 +41,15 @@ __device__ __forceinline__ float decay_owed(float v, float beta2, uint32_t owed)
     return v;
 }
 
-// For j in I_{t-1}: h = mean_w g^(w)_j ; v_j = beta2 v_j + (1-beta2) h^2 ; vhat_j = max(vhat_j, v_j).
-__global__ void __launch_bounds__(kThreads)
-k_second_moment(const __grid_constant__ Params P, const float* __restrict__ grads, float* v, float* vhat,
-                uint32_t* vstamp, const uint32_t* __restrict__ I_prev, uint32_t k_prev, uint32_t t) {
-    const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
-    if (q >= k_prev) return;
-    const uint32_t j = I_prev[q];
-    float h = 0.0f;
-#pragma unroll 4
-    for (uint32_t w = 0; w < P.n; ++w) h += __ldg(grads + (uint64_t)w * P.d + j);
-    h = h / (float)P.n;
-    float vj = decay_owed(v[j], P.beta2, t - 1u - vstamp[j]);
+// Master side of Algorithm 2 for one coordinate of I_{t-1}, given the sum of the workers' gradients there:
+// h = sum / n ; v = beta2 v + (1-beta2) h^2 ; vhat = max(vhat, v).
+__device__ __forceinline__ void second_moment(const Params& P, const MomentArgs& A, uint32_t j, float gsum) {
+    const float h = gsum / (float)P.n;
+    float vj = decay_owed(A.v[j], P.beta2, A.step - 1u - A.vstamp[j]);
     vj = fmaf(P.beta2, vj, (1.0f - P.beta2) * h * h);
-    v[j] = vj;
-    vstamp[j] = t;
-    if (vj > vhat[j]) vhat[j] = vj;
+    A.v[j] = vj;
+    A.vstamp[j] = A.step;
+    if (vj > A.vhat[j]) A.vhat[j] = vj;
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -60,83 +59,121 @@ k_v_materialize(const __grid_constant__ Params P, const float* __restrict__ v,
         out[j] = decay_owed(v[j], P.beta2, t - vstamp[j]);
 }
 
-// m = beta1 m + (1-beta1) g ; a = m + e (kept in the e buffer) ; S^(w)[row, h_row(j)] += s_row(j) a_j.
+// e as Algorithm 2 defines it: the buffer keeps a_t everywhere and the bitmap of I_t marks the zeros
+__global__ void __launch_bounds__(kThreads)
+k_masked_copy(const float* __restrict__ e, const uint32_t* __restrict__ bitmap, uint32_t d, uint64_t total, float* out) {
+    for (uint64_t q = blockIdx.x * (uint64_t)kThreads + threadIdx.x; q < total; q += (uint64_t)gridDim.x * kThreads) {
+        const uint32_t j = (uint32_t)(q % d);
+        out[q] = ((bitmap[j >> 5] >> (j & 31u)) & 1u) ? 0.0f : e[q];
+    }
+}
+
+#define SK_MOMENT(mm, aa, gg, mask)                                                     \
+    mm.x = fmaf(b1, mm.x, omb1 * gg.x); mm.y = fmaf(b1, mm.y, omb1 * gg.y);             \
+    mm.z = fmaf(b1, mm.z, omb1 * gg.z); mm.w = fmaf(b1, mm.w, omb1 * gg.w);             \
+    aa.x = mm.x + ((mask & 1u) ? 0.0f : aa.x); aa.y = mm.y + ((mask & 2u) ? 0.0f : aa.y); \
+    aa.z = mm.z + ((mask & 4u) ? 0.0f : aa.z); aa.w = mm.w + ((mask & 8u) ? 0.0f : aa.w);
+
+// m = beta1 m + (1-beta1) g ; a = m + e (kept in the e buffer; e counts as 0 on I_{t-1}) ;
+// S^(w)[row, h_row(j)] += s_row(j) a_j ; and on I_{t-1} the gradient sum that feeds v and vhat.
 // Vector form: one thread owns 4 consecutive coordinates and walks the workers w0..w0+nw-1, so the hashes are
 // evaluated once per coordinate quad and reused for every worker (all workers share h and s, or the sketches
 // could not be added).  R > 0: rows known at compile time; R == 0: any r <= kMaxRows.
 template <int R>
-__global__ void __launch_bounds__(kThreads)
-k_moment_sketch_v4(const __grid_constant__ Params P, const float4* __restrict__ grads, float4* m, float4* e,
-                   float* tables, uint32_t w0, uint32_t nw) {
+__global__ void __launch_bounds__(kThreads, 3)
+k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
+    const float4* __restrict__ grads = (const float4*)A.grads;
+    float4* m = (float4*)A.m;
+    float4* e = (float4*)A.e;
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
     const uint32_t d4 = P.d >> 2;
     const float b1 = P.beta1, omb1 = 1.0f - P.beta1;
     const uint64_t tstride = (uint64_t)P.r * P.cs;
-    for (uint32_t t = blockIdx.x * kThreads + threadIdx.x; t < d4; t += gridDim.x * kThreads) {
-        Quad h[R > 0 ? R : (int)kMaxRows];
-#pragma unroll
-        for (uint32_t row = 0; row < r; ++row) h[row] = quad_hash(P.row_key[row], P.log2g, P.G, t << 2);
+    constexpr int RMAX = R > 0 ? R : (int)kMaxRows;
+    const uint32_t trips = (d4 + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
+    for (uint32_t it = 0; it < trips; ++it) {            // uniform trip count: the hash exchange needs whole warps
+        const uint32_t t = (it * gridDim.x + blockIdx.x) * kThreads + threadIdx.x;
+        Quad h[RMAX];
+        quad_hashes<RMAX>(P.row_key, r, P.log2g, P.G, t < d4 ? t : d4 - 1, h);
+        if (t >= d4) continue;
+        const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
+        float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);     // running gradient sum in worker order (used on I_{t-1})
+        if (mask && w0 > 0) gs = ((const float4*)A.gsum)[t];
         uint32_t w = w0;
         const uint32_t wend = w0 + nw;
-        for (; w + 2 <= wend; w += 2) {          // two workers per trip: six 16-byte loads in flight
+        for (; w + 2 <= wend; w += 2) {                  // two workers per trip: six 16-byte loads in flight
             const uint64_t q0 = (uint64_t)w * d4 + t, q1 = q0 + d4;
             const float4 g0 = __ldcs(grads + q0), g1 = __ldcs(grads + q1);
             float4 m0 = __ldcs(m + q0), m1 = __ldcs(m + q1);
             float4 a0 = __ldcs(e + q0), a1 = __ldcs(e + q1);
-            m0.x = fmaf(b1, m0.x, omb1 * g0.x); m0.y = fmaf(b1, m0.y, omb1 * g0.y);
-            m0.z = fmaf(b1, m0.z, omb1 * g0.z); m0.w = fmaf(b1, m0.w, omb1 * g0.w);
-            m1.x = fmaf(b1, m1.x, omb1 * g1.x); m1.y = fmaf(b1, m1.y, omb1 * g1.y);
-            m1.z = fmaf(b1, m1.z, omb1 * g1.z); m1.w = fmaf(b1, m1.w, omb1 * g1.w);
-            a0.x += m0.x; a0.y += m0.y; a0.z += m0.z; a0.w += m0.w;
-            a1.x += m1.x; a1.y += m1.y; a1.z += m1.z; a1.w += m1.w;
+            SK_MOMENT(m0, a0, g0, mask)
+            SK_MOMENT(m1, a1, g1, mask)
+            gs.x = (gs.x + g0.x) + g1.x; gs.y = (gs.y + g0.y) + g1.y;
+            gs.z = (gs.z + g0.z) + g1.z; gs.w = (gs.w + g0.w) + g1.w;
             __stcs(m + q0, m0); __stcs(m + q1, m1);
             __stcs(e + q0, a0); __stcs(e + q1, a1);
-            float* t0 = tables + (uint64_t)w * tstride;
+            float* t0 = A.tables + (uint64_t)w * tstride;
             float* t1 = t0 + tstride;
 #pragma unroll
-            for (uint32_t row = 0; row < r; ++row) {
-                red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
-                red_add_v4(t1 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a1));
-            }
+            for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+                if (row < r) {
+                    red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+                    red_add_v4(t1 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a1));
+                }
         }
         if (w < wend) {
             const uint64_t q0 = (uint64_t)w * d4 + t;
             const float4 g0 = __ldcs(grads + q0);
             float4 m0 = __ldcs(m + q0);
             float4 a0 = __ldcs(e + q0);
-            m0.x = fmaf(b1, m0.x, omb1 * g0.x); m0.y = fmaf(b1, m0.y, omb1 * g0.y);
-            m0.z = fmaf(b1, m0.z, omb1 * g0.z); m0.w = fmaf(b1, m0.w, omb1 * g0.w);
-            a0.x += m0.x; a0.y += m0.y; a0.z += m0.z; a0.w += m0.w;
+            SK_MOMENT(m0, a0, g0, mask)
+            gs.x += g0.x; gs.y += g0.y; gs.z += g0.z; gs.w += g0.w;
             __stcs(m + q0, m0);
             __stcs(e + q0, a0);
-            float* t0 = tables + (uint64_t)w * tstride;
+            float* t0 = A.tables + (uint64_t)w * tstride;
 #pragma unroll
-            for (uint32_t row = 0; row < r; ++row)
-                red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+            for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+                if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
         }
+        if (mask) ((float4*)A.gsum)[t] = gs;             // consumed by k_second_moment (or by the next launch)
     }
 }
 
 // Scalar form: any d, any alignment, any group size.  One thread per coordinate.
 __global__ void __launch_bounds__(kThreads)
-k_moment_sketch_scalar(const __grid_constant__ Params P, const float* __restrict__ grads, float* m, float* e,
-                       float* tables, uint32_t w0, uint32_t nw) {
+k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
     const float b1 = P.beta1, omb1 = 1.0f - P.beta1;
     const uint64_t tstride = (uint64_t)P.r * P.cs;
     for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads) {
+        const bool member = A.members && ((A.bitmap[j >> 5] >> (j & 31u)) & 1u);
+        float gs = (member && w0 > 0) ? A.gsum[j] : 0.0f;
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q = (uint64_t)w * P.d + j;
-            const float mm = fmaf(b1, m[q], omb1 * grads[q]);
-            const float a = mm + e[q];
-            m[q] = mm;
-            e[q] = a;
+            const float g = A.grads[q];
+            const float mm = fmaf(b1, A.m[q], omb1 * g);
+            const float a = mm + (member ? 0.0f : A.e[q]);
+            gs += g;
+            A.m[q] = mm;
+            A.e[q] = a;
             for (uint32_t row = 0; row < P.r; ++row) {
                 uint32_t b; float s;
                 coord_hash(P.row_key[row], P.log2g, P.G, j, b, s);
-                atomicAdd(tables + (uint64_t)w * tstride + (uint64_t)row * P.cs + b, s * a);
+                atomicAdd(A.tables + (uint64_t)w * tstride + (uint64_t)row * P.cs + b, s * a);
             }
         }
+        if (member) A.gsum[j] = gs;
     }
+}
+
+// For j in I_{t-1}: h = (sum_w g^(w)_j) / n ; v_j = beta2 v_j + (1-beta2) h^2 ; vhat_j = max(vhat_j, v_j).
+// The gradient sums were left in gsum by the moment kernel, which streams every gradient anyway.
+__global__ void __launch_bounds__(kThreads)
+k_second_moment(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A,
+                const uint32_t* __restrict__ I_prev, uint32_t k_prev) {
+    const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
+    if (q >= k_prev) return;
+    const uint32_t j = I_prev[q];
+    second_moment(P, A, j, A.gsum[j]);
 }
 
 // S = (S^(0) + S^(1) + ... + S^(n-1)) / n, workers added in index order (Algorithm 2, master side).
@@ -163,8 +200,8 @@ inline int grid_for(uint64_t items, int sm_count, int per_sm) {
 
 }  // namespace
 
-int launch_zero(float* p, uint64_t nfloats, cudaStream_t st) {
-    k_zero<<<grid_for(nfloats / 4, 148, 8), kThreads, 0, st>>>((float4*)p, nfloats / 4);
+int launch_zero(void* p, uint64_t bytes, cudaStream_t st) {   // bytes must be a multiple of 16
+    k_zero<<<grid_for(bytes / 16, 148, 8), kThreads, 0, st>>>((float4*)p, bytes / 16);
     return 1;
 }
 
@@ -173,11 +210,9 @@ int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st) {
     return 1;
 }
 
-int launch_second_moment(const Params& P, const float* grads, float* v, float* vhat, uint32_t* vstamp,
-                         const uint32_t* I_prev, uint32_t k_prev, uint32_t t, cudaStream_t st) {
-    if (k_prev == 0) return 0;
-    k_second_moment<<<(k_prev + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, grads, v, vhat, vstamp, I_prev,
-                                                                           k_prev, t);
+int launch_set_bits(const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st) {
+    if (count == 0) return 0;
+    k_set_bits<<<(count + kThreads - 1) / kThreads, kThreads, 0, st>>>(I, count, bitmap);
     return 1;
 }
 
@@ -187,22 +222,33 @@ int launch_v_materialize(const Params& P, const float* v, const uint32_t* vstamp
     return 1;
 }
 
-int launch_moment_sketch(const Params& P, const float* grads, float* m, float* e, float* tables, uint32_t w0,
-                         uint32_t nw, bool vec, int sm_count, cudaStream_t st) {
+int launch_masked_copy(const Params& P, const float* e, const uint32_t* bitmap, uint32_t workers, float* out,
+                       cudaStream_t st) {
+    const uint64_t total = (uint64_t)workers * P.d;
+    k_masked_copy<<<grid_for(total, 148, 16), kThreads, 0, st>>>(e, bitmap, P.d, total, out);
+    return 1;
+}
+
+int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,
+                         cudaStream_t st) {
     if (!vec) {
-        k_moment_sketch_scalar<<<grid_for(P.d, sm_count, 8), kThreads, 0, st>>>(P, grads, m, e, tables, w0, nw);
+        k_moment_sketch_scalar<<<grid_for(P.d, sm_count, 1), kThreads, 0, st>>>(P, A, w0, nw);
         return 1;
     }
-    const int grid = grid_for(P.d >> 2, sm_count, 8);
-    const float4* g4 = (const float4*)grads;
-    float4* m4 = (float4*)m;
-    float4* e4 = (float4*)e;
-#define SK_CASE(RR) case RR: k_moment_sketch_v4<RR><<<grid, kThreads, 0, st>>>(P, g4, m4, e4, tables, w0, nw); break;
+    const int grid = grid_for(P.d >> 2, sm_count, 1);    // the caller passes SMs x CTAs per SM
+#define SK_CASE(RR) case RR: k_moment_sketch_v4<RR><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
     switch (P.r) {
         SK_CASE(1) SK_CASE(2) SK_CASE(3) SK_CASE(4) SK_CASE(5) SK_CASE(6) SK_CASE(7) SK_CASE(8) SK_CASE(10)
-        default: k_moment_sketch_v4<0><<<grid, kThreads, 0, st>>>(P, g4, m4, e4, tables, w0, nw); break;
+        default: k_moment_sketch_v4<0><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
     }
 #undef SK_CASE
+    return 1;
+}
+
+int launch_second_moment(const Params& P, const MomentArgs& A, const uint32_t* I_prev, uint32_t k_prev,
+                         cudaStream_t st) {
+    if (k_prev == 0) return 0;
+    k_second_moment<<<(k_prev + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, A, I_prev, k_prev);
     return 1;
 }
 

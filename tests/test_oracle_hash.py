@@ -37,11 +37,11 @@ def _family(seed, log2g, c, row, i):
     G = c // g
     K = _mix((seed + (row + 1) * GOLDEN_GAMMA) & M64)
     q, o = divmod(i, g)
-    u1 = _mix((K + (2 * q + 1) * GOLDEN_GAMMA) & M64)
-    u2 = _mix((K + (2 * q + 2) * GOLDEN_GAMMA) & M64)
-    B = ((u1 >> 32) * G) >> 32
-    p = (u2 >> 32) % g
-    return g * B + (o ^ p), (-1 if (u1 >> o) & 1 else 1)
+    u = _mix((K + (q + 1) * GOLDEN_GAMMA) & M64)
+    hi, lo = divmod(u, 1 << 32)
+    B, rem = divmod(hi * G, 1 << 32)
+    p = (rem * g) >> 32                      # leading log2(g) bits of the 32-bit remainder
+    return g * B + (o ^ p), (-1 if (lo >> o) & 1 else 1)
 
 
 @pytest.mark.parametrize("log2g", [0, 1, 2, 3, 4, 5])
