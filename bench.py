@@ -167,6 +167,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--log2g", type=int, default=None)
+    ap.add_argument("--window-lines", type=int, default=None, help="windowed hash family: lines per window (0 = plain)")
     ap.add_argument("--worker-chunk", type=int, default=0)
     ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -198,7 +199,7 @@ def main():
 
     src = synthetic.GradientSource(w, device=dev, cfg_id=cfg_id)
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                                  eps=w.eps, log2g=args.log2g)
+                                  eps=w.eps, log2g=args.log2g, window_lines=args.window_lines)
     opt.set_option("worker_chunk", args.worker_chunk)
     if args.sketch_ctas:
         opt.set_option("sketch_ctas_per_sm", args.sketch_ctas)
@@ -295,6 +296,7 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k,
                        "recipe": w.recipe, "hash_group": 1 << opt.get_option("log2g"),
+                       "window_lines": opt.get_option("window_lines"),
                        "worker_chunk": opt.get_option("worker_chunk"), "replicas": world,
                        "l2": f"inputs larger than L2: {nsets} rotating gradient sets of {set_bytes / 1e9:.2f} GB"},
             "steps_per_s": 1e3 / ms_step,

@@ -42,6 +42,7 @@ def lib() -> C.CDLL:
         L.ora_stream.restype = u64; L.ora_stream.argtypes = [u64, u64]
         L.ora_row_key.restype = u64; L.ora_row_key.argtypes = [u64, u32]
         L.ora_hash.restype = None; L.ora_hash.argtypes = [u64, u32, u32, u32, u64, u64, vp, vp]
+        L.ora_hash_w.restype = None; L.ora_hash_w.argtypes = [u64, u32, u32, u32, u32, u64, u64, vp, vp]
         L.ora_sketch.restype = None; L.ora_sketch.argtypes = [vp, u64, u32, u32, vp, vp, vp]
         L.ora_median.restype = f32; L.ora_median.argtypes = [vp, u32]
         L.ora_unsketch.restype = None; L.ora_unsketch.argtypes = [vp, u64, u32, u32, vp, vp, vp, vp]
@@ -71,11 +72,11 @@ def stream(s0: int, t: int) -> int:
     return int(lib().ora_stream(s0 & (2**64 - 1), t))
 
 
-def hash_family(seed: int, log2g: int, c: int, row: int, i0: int, count: int):
+def hash_family(seed: int, log2g: int, c: int, row: int, i0: int, count: int, window_lines: int = 0):
     """Buckets (uint32) and signs (int8) of coordinates i0..i0+count-1 in one row."""
     b = np.empty(count, np.uint32)
     s = np.empty(count, np.int8)
-    lib().ora_hash(seed, log2g, c, row, i0, count, _p(b), _p(s))
+    lib().ora_hash_w(seed, log2g, window_lines, c, row, i0, count, _p(b), _p(s))
     return b, s
 
 
@@ -119,7 +120,7 @@ class Oracle:
     """One SketchedAMSGrad (gradient averaging) optimiser; `step` advances it by one iteration."""
 
     def __init__(self, d, n, r, c, k, seed=0, log2g=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8,
-                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1):
+                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
         self._h = lib().ora_create(d, n, r, c, k, seed, log2g, lr, beta1, beta2, eps)
         if not self._h:
@@ -130,6 +131,10 @@ class Oracle:
             hs = np.ascontiguousarray(hash_sgn, np.int8).reshape(r, d)
             self._keep = (hi, hs)
             lib().ora_set_hash(self._h, _p(hi), _p(hs))
+        if window_lines:
+            if log2g != 5 or 32 * window_lines > c:
+                raise ValueError("the windowed family needs g = 32 and 32 * window_lines <= c")
+            lib().ora_set_option(self._h, b"window_lines", int(window_lines))
         lib().ora_set_option(self._h, b"v_keep", int(v_keep))
         lib().ora_set_option(self._h, b"threads", int(threads))
 

@@ -38,25 +38,51 @@ uint64_t ora_stream(uint64_t s0, uint64_t t) { return ora_mix64(s0 + t * GOLDEN)
 
 uint64_t ora_row_key(uint64_t seed, uint32_t row) { return ora_stream(seed, (uint64_t)row + 1); }
 
-void ora_hash_one(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint64_t i,
-                  uint32_t* bucket, int8_t* sign) {
+/* Windowed variant (window_lines = L > 0, needs g = 32): the coordinates are cut into units of 1024; unit u
+ * belongs to panel u mod P, where P = floor(c / (32 L)) is the number of aligned windows of 32 L buckets in a
+ * row; every group of the unit lands in its panel's window, on one of the window's L lines:
+ *   x = hi * L ;  line = x div 2^32 ;  p = leading 5 bits of (x mod 2^32)
+ *   h_j(i) = (u mod P) * 32 L + 32 * line + (o xor p) ;   signs as above.
+ * A row is then P independent small Count Sketches (one per panel, each of 32 L buckets); coordinates of
+ * different panels never meet, coordinates of one panel and different groups meet with probability 1/(32 L).
+ * Because units are dealt to panels round-robin, every panel sees every part of the vector. */
+#define ORA_UNIT 1024ULL
+
+void ora_hash_one_w(uint64_t seed, uint32_t log2g, uint32_t window_lines, uint32_t c, uint32_t row, uint64_t i,
+                    uint32_t* bucket, int8_t* sign) {
     uint64_t g = 1ULL << log2g;
-    uint64_t G = c / g;
     uint64_t q = i >> log2g;
     uint64_t o = i & (g - 1);
     uint64_t K = ora_row_key(seed, row);
     uint64_t u = ora_stream(K, q + 1);
     uint64_t hi = u >> 32, lo = u & 0xFFFFFFFFULL;
+    uint64_t G = window_lines ? window_lines : c / g;      /* lines to choose from */
     uint64_t x = hi * G;
     uint64_t B = x >> 32;
     uint64_t p = log2g ? ((x & 0xFFFFFFFFULL) >> (32 - log2g)) : 0;
-    *bucket = (uint32_t)(g * B + (o ^ p));
+    uint64_t base = 0;
+    if (window_lines) {
+        uint64_t cw = g * window_lines, P = c / cw;
+        base = ((i / ORA_UNIT) % P) * cw;
+    }
+    *bucket = (uint32_t)(base + g * B + (o ^ p));
     *sign = ((lo >> o) & 1ULL) ? -1 : 1;
+}
+
+void ora_hash_one(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint64_t i,
+                  uint32_t* bucket, int8_t* sign) {
+    ora_hash_one_w(seed, log2g, 0, c, row, i, bucket, sign);
 }
 
 void ora_hash(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint64_t i0, uint64_t count,
               uint32_t* bucket, int8_t* sign) {
     for (uint64_t t = 0; t < count; ++t) ora_hash_one(seed, log2g, c, row, i0 + t, &bucket[t], &sign[t]);
+}
+
+void ora_hash_w(uint64_t seed, uint32_t log2g, uint32_t window_lines, uint32_t c, uint32_t row, uint64_t i0,
+                uint64_t count, uint32_t* bucket, int8_t* sign) {
+    for (uint64_t t = 0; t < count; ++t)
+        ora_hash_one_w(seed, log2g, window_lines, c, row, i0 + t, &bucket[t], &sign[t]);
 }
 
 /* ------------------------------------------------------------------------------------------------

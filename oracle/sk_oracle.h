@@ -41,6 +41,11 @@ void ora_hash_one(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint6
                   uint32_t* bucket, int8_t* sign);
 void ora_hash(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint64_t i0, uint64_t count,
               uint32_t* bucket, int8_t* sign);
+/* windowed variant of the family (window_lines > 0; see sk_oracle.c); window_lines = 0 is the plain family */
+void ora_hash_one_w(uint64_t seed, uint32_t log2g, uint32_t window_lines, uint32_t c, uint32_t row, uint64_t i,
+                    uint32_t* bucket, int8_t* sign);
+void ora_hash_w(uint64_t seed, uint32_t log2g, uint32_t window_lines, uint32_t c, uint32_t row, uint64_t i0,
+                uint64_t count, uint32_t* bucket, int8_t* sign);
 
 /* ---- Count Sketch primitives with EXPLICIT index / sign arrays (idx[row*d+i], sgn[row*d+i]) */
 void ora_sketch(const float* a, uint64_t d, uint32_t r, uint32_t c,

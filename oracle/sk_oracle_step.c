@@ -12,7 +12,7 @@
 
 struct ora_state {
     uint64_t d, k, seed, t, k_prev;
-    uint32_t n, r, c, log2g;
+    uint32_t n, r, c, log2g, window_lines;
     float lr, beta1, beta2, eps;
     int v_keep, threads;
     float *m, *e, *v, *vhat, *est, *tables, *sum;
@@ -58,6 +58,11 @@ void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn) { s->h_i
 
 void ora_set_option(ora_state* s, const char* key, int value) {
     if (!strcmp(key, "v_keep")) s->v_keep = value;
+    else if (!strcmp(key, "window_lines")) {
+        /* only with g = 32 and at least one whole window in a row; otherwise left unchanged */
+        if (value >= 0 && (value == 0 || (s->log2g == 5 && (uint64_t)32 * (uint64_t)value <= s->c)))
+            s->window_lines = (uint32_t)value;
+    }
     else if (!strcmp(key, "threads")) s->threads = value > 0 ? value : 1;
 }
 
@@ -87,9 +92,15 @@ static inline void hash_at(const ora_state* s, uint32_t j, uint64_t i, uint32_t*
     uint64_t g = 1ULL << s->log2g, G = s->c / g;
     uint64_t q = i >> s->log2g, o = i & (g - 1);
     uint64_t u = ora_stream(s->row_key[j], q + 1);
+    uint64_t base = 0;
+    if (s->window_lines) {                 /* windowed family: the unit's panel fixes the window, L lines to choose from */
+        uint64_t cw = g * s->window_lines;
+        base = ((i / 1024) % (s->c / cw)) * cw;
+        G = s->window_lines;
+    }
     uint64_t x = (u >> 32) * G;
     uint64_t p = s->log2g ? ((x & 0xFFFFFFFFULL) >> (32 - s->log2g)) : 0;
-    *b = (uint32_t)(g * (x >> 32) + (o ^ p));
+    *b = (uint32_t)(base + g * (x >> 32) + (o ^ p));
     *sg = (((u & 0xFFFFFFFFULL) >> o) & 1ULL) ? -1 : 1;
 }
 

@@ -79,13 +79,16 @@ class SketchedAMSGrad:
 
     _FIELD_SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "tables": "nrc", "sum": "rc"}
 
-    def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None):
+    def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None,
+                 window_lines=None):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
         self._h = lib().sk_create(d, n, r, c, k, seed, lr, beta1, beta2, eps)
         if not self._h:
             raise SkError(f"sk_create failed: {lib().sk_last_error().decode()}")
         if log2g is not None:
             self.set_option("log2g", log2g)
+        if window_lines is not None:
+            self.set_option("window_lines", window_lines)
 
     def close(self):
         if getattr(self, "_h", None):

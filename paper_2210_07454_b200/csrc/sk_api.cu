@@ -3,6 +3,7 @@
 #include "../../include/sketched_amsgrad.h"
 #include "sk_internal.h"
 #include "sk_hash.cuh"
+#include "sk_state.h"
 
 #include <algorithm>
 #include <cmath>
@@ -34,43 +35,20 @@ int fail(int code, const char* fmt, ...) {
                         cudaGetErrorString(err__));                                                \
     } while (0)
 
-struct TimeRec { int stage; cudaEvent_t a, b; };
-
 }  // namespace
-
-struct sk_state {
-    sk::Params P{};
-    uint64_t seed = 0, t = 0;
-    float eps = 0;
-    uint32_t k_prev = 0;
-    int sm_count = 148;
-    size_t l2_bytes = 0;
-    int64_t worker_chunk = 0;
-    int64_t sketch_ctas_per_sm = 64;
-    bool timing = false;
-    cudaStream_t stream = nullptr;
-    // device memory owned by the handle
-    float *m = nullptr, *e = nullptr, *v = nullptr, *vhat = nullptr, *tables = nullptr, *sum = nullptr;
-    uint32_t *vstamp = nullptr, *I = nullptr, *I_prev = nullptr, *hist = nullptr, *hist2 = nullptr;
-    uint32_t *keys = nullptr, *bitmap = nullptr;
-    float* gsum = nullptr;
-    uint64_t bitmap_bytes = 0;
-    sk::Select* sel = nullptr;
-    sk::Cand *cand = nullptr, *cand2 = nullptr;
-    float *stage_grads = nullptr, *stage_x = nullptr;
-    // timing
-    std::vector<TimeRec> recs;
-    std::vector<cudaEvent_t> free_events;
-    double ms[SK_NUM_STAGES] = {0};
-    uint64_t launches[SK_NUM_STAGES] = {0};
-    uint64_t timed_steps = 0;
-};
 
 namespace {
 
 void refresh_hash(sk_state* s) {
     for (uint32_t j = 0; j < s->P.r; ++j) s->P.row_key[j] = sk::row_key(s->seed, j);
     s->P.G = s->P.c >> s->P.log2g;
+    s->P.win_cw = 0;
+    s->P.win_panels = 0;
+    if (s->window_lines > 0) {        // windowed family: a group picks one of the window's lines
+        s->P.G = (uint32_t)s->window_lines;
+        s->P.win_cw = 32u * (uint32_t)s->window_lines;
+        s->P.win_panels = s->P.c / s->P.win_cw;
+    }
 }
 
 uint32_t chunk_of(const sk_state* s) {
@@ -144,7 +122,8 @@ int do_step(sk_state* s, const float* grads, float* x) {
     A.grads = grads; A.m = s->m; A.e = s->e; A.tables = s->tables; A.gsum = s->gsum;
     A.v = s->v; A.vhat = s->vhat; A.vstamp = s->vstamp; A.bitmap = s->bitmap;
     A.step = t; A.members = s->k_prev ? 1u : 0u;
-    const uint32_t wc = chunk_of(s);
+    const bool windowed = vec && P.win_cw != 0;
+    const uint32_t wc = windowed ? std::min<uint32_t>(sk::kWinMaxWorkers, P.n) : chunk_of(s);
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
         const uint32_t nw = std::min(wc, P.n - w0);
@@ -153,7 +132,14 @@ int do_step(sk_state* s, const float* grads, float* x) {
             tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats * 4, st));
         }
         StageTimer tm(s, 2);     // moments + sketch; also leaves the gradient sums on I_{t-1} in gsum
-        tm.done(sk::launch_moment_sketch(P, A, w0, nw, vec, s->sm_count * (int)s->sketch_ctas_per_sm, st));
+        if (windowed) {
+            const int l = sk::launch_moment_sketch_win(P, A, w0, nw, s->sm_count, st);
+            if (l < 0) return fail(SK_ECUDA, "the windowed sketch kernel does not fit in shared memory (window_lines=%lld, r=%u)",
+                                   (long long)s->window_lines, P.r);
+            tm.done(l);
+        } else {
+            tm.done(sk::launch_moment_sketch(P, A, w0, nw, vec, s->sm_count * (int)s->sketch_ctas_per_sm, st));
+        }
     }
     {   // v, vhat on I_{t-1} from those sums
         StageTimer tm(s, 1);
@@ -329,6 +315,16 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         if (s->t != 0) return fail(SK_ESTATE, "log2g can only be changed before the first step");
         if (value < 0 || value > 5 || (1u << value) > s->P.c) return fail(SK_EINVAL, "log2g must be in 0..5 with 2^log2g <= c");
         s->P.log2g = (uint32_t)value;
+        if (value != 5) s->window_lines = 0;
+        refresh_hash(s);
+        return SK_OK;
+    }
+    if (!strcmp(key, "window_lines")) {
+        if (s->t != 0) return fail(SK_ESTATE, "window_lines can only be changed before the first step");
+        if (value < 0 || value > 64 || (value & (value - 1))) return fail(SK_EINVAL, "window_lines must be 0 or a power of two <= 64");
+        if (value > 0 && (s->P.log2g != 5 || 32ull * (uint64_t)value > s->P.c))
+            return fail(SK_EINVAL, "window_lines needs a hash group of 32 and 32*window_lines <= c");
+        s->window_lines = value;
         refresh_hash(s);
         return SK_OK;
     }
@@ -354,6 +350,7 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
 int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     if (!s || !key || !value) return fail(SK_EINVAL, "null argument");
     if (!strcmp(key, "log2g")) *value = s->P.log2g;
+    else if (!strcmp(key, "window_lines")) *value = s->window_lines;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
     else if (!strcmp(key, "sketch_ctas_per_sm")) *value = s->sketch_ctas_per_sm;

@@ -2,10 +2,12 @@
 // and is documented with sk_hash in the public header).  Device-side evaluation only.
 #pragma once
 #include <cstdint>
+#include "sk_internal.h"
 
 namespace sk {
 
 constexpr uint64_t kGolden = 0x9E3779B97F4A7C15ULL;
+constexpr uint32_t kUnitShift = 10;     // windowed family: units of 1024 coordinates
 
 __host__ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
@@ -20,59 +22,50 @@ __host__ __device__ __forceinline__ uint64_t row_key(uint64_t seed, uint32_t row
     return stream(seed, (uint64_t)row + 1);
 }
 
+// first bucket of the window that coordinate i's unit owns in every row (0 for the plain family)
+__device__ __forceinline__ uint32_t window_base(const Params& P, uint32_t i) {
+    return P.win_cw ? ((i >> kUnitShift) % P.win_panels) * P.win_cw : 0u;
+}
+
 // What one group of g = 2^log2g consecutive coordinates needs in one row.
 struct GroupHash {
-    uint32_t base;   // g * B : first bucket of the group's aligned block
+    uint32_t base;   // first bucket of the group's aligned block (relative to the window base, if any)
     uint32_t perm;   // xor permutation inside the block, in [0,g)
     uint32_t signs;  // bit o set  <=>  coordinate with offset o carries sign -1
 };
 
-// from one 64-bit draw u: high word -> bucket group by multiply-high range reduction, the leading bits of the
-// remainder -> xor permutation, low word -> sign bits
-__device__ __forceinline__ GroupHash group_from_draw(uint64_t u, uint32_t log2g, uint32_t G) {
+// from one 64-bit draw u: high word -> block by multiply-high range reduction over P.G choices, the leading
+// bits of the remainder -> xor permutation, low word -> sign bits
+__device__ __forceinline__ GroupHash group_from_draw(const Params& P, uint64_t u) {
     const uint32_t hi = (uint32_t)(u >> 32);
     GroupHash h;
-    h.base = __umulhi(hi, G) << log2g;
-    h.perm = log2g ? ((hi * G) >> (32u - log2g)) : 0u;
+    h.base = __umulhi(hi, P.G) << P.log2g;
+    h.perm = P.log2g ? ((hi * P.G) >> (32u - P.log2g)) : 0u;
     h.signs = (uint32_t)u;
     return h;
 }
 
-__device__ __forceinline__ GroupHash group_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t q) {
-    return group_from_draw(stream(key, (uint64_t)q + 1), log2g, G);
-}
-
-// Scalar form: bucket and sign (+1/-1) of coordinate i.
-__device__ __forceinline__ void coord_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t i,
-                                           uint32_t& bucket, float& sign) {
-    const uint32_t q = i >> log2g, o = i & ((1u << log2g) - 1u);
-    const GroupHash h = group_hash(key, log2g, G, q);
-    bucket = h.base + (o ^ h.perm);
+// Scalar form: bucket and sign (+1/-1) of coordinate i in the row with key `key`.
+__device__ __forceinline__ void coord_hash(const Params& P, uint64_t key, uint32_t i, uint32_t& bucket, float& sign) {
+    const uint32_t q = i >> P.log2g, o = i & ((1u << P.log2g) - 1u);
+    const GroupHash h = group_from_draw(P, stream(key, (uint64_t)q + 1));
+    bucket = window_base(P, i) + h.base + (o ^ h.perm);
     sign = ((h.signs >> o) & 1u) ? -1.0f : 1.0f;
 }
 
 // Vector form for 4 consecutive coordinates i..i+3 (i % 4 == 0, g >= 4): they land in one aligned 16-byte
 // chunk of the row.  `off` is the element offset of that chunk inside the row; local coordinate l goes to
-// element (l xor p3) of the chunk; bit l of `sgn` is its sign.
+// element (l xor p3) of the chunk; bit l of the sign field is its sign.
 struct Quad {
     uint32_t off;
     uint32_t p3sgn;  // bits 0..1: p3 ; bits 2..5: sign bits of local coordinates 0..3
 };
 
-__device__ __forceinline__ Quad quad_hash(uint64_t key, uint32_t log2g, uint32_t G, uint32_t i) {
-    const uint32_t q = i >> log2g, o = i & ((1u << log2g) - 1u);
-    const GroupHash h = group_hash(key, log2g, G, q);
+__device__ __forceinline__ Quad quad_from_draw(const Params& P, uint64_t u, uint32_t i, uint32_t wbase) {
+    const uint32_t o = i & ((1u << P.log2g) - 1u);
+    const GroupHash h = group_from_draw(P, u);
     Quad r;
-    r.off = h.base + ((o ^ h.perm) & ~3u);
-    r.p3sgn = (h.perm & 3u) | (((h.signs >> o) & 0xFu) << 2);
-    return r;
-}
-
-__device__ __forceinline__ Quad quad_from_draw(uint64_t u, uint32_t log2g, uint32_t G, uint32_t i) {
-    const uint32_t o = i & ((1u << log2g) - 1u);
-    const GroupHash h = group_from_draw(u, log2g, G);
-    Quad r;
-    r.off = h.base + ((o ^ h.perm) & ~3u);
+    r.off = wbase + h.base + ((o ^ h.perm) & ~3u);
     r.p3sgn = (h.perm & 3u) | (((h.signs >> o) & 0xFu) << 2);
     return r;
 }
@@ -81,9 +74,10 @@ __device__ __forceinline__ Quad quad_from_draw(uint64_t u, uint32_t log2g, uint3
 // group split the rows between them (one 64-bit draw per lane and round) and exchange the draws by shuffle, so
 // ALL 32 LANES OF THE WARP MUST CALL THIS TOGETHER (callers clamp t for lanes past the end).
 template <int RMAX>
-__device__ __forceinline__ void quad_hashes(const uint64_t* __restrict__ row_key /* param space */, uint32_t r,
-                                            uint32_t log2g, uint32_t G, uint32_t t, Quad (&h)[RMAX]) {
-    if (log2g == 5) {
+__device__ __forceinline__ void quad_hashes(const Params& P, uint32_t r, uint32_t t, Quad (&h)[RMAX]) {
+    const uint32_t i = t << 2;
+    const uint32_t wbase = window_base(P, i);
+    if (P.log2g == 5) {
         const uint32_t lane = threadIdx.x & 31u, li = lane & 7u, q = t >> 3;
 #pragma unroll
         for (uint32_t k = 0; k < (uint32_t)RMAX; k += 8) {
@@ -91,7 +85,7 @@ __device__ __forceinline__ void quad_hashes(const uint64_t* __restrict__ row_key
                 uint64_t key = 0;
 #pragma unroll
                 for (uint32_t j = 0; j < 8; ++j)
-                    if (k + j < (uint32_t)RMAX && j == li) key = row_key[k + j];
+                    if (k + j < (uint32_t)RMAX && j == li) key = P.row_key[k + j];
                 const uint64_t u = (k + li < r) ? stream(key, (uint64_t)q + 1) : 0ull;
                 const uint32_t hi = (uint32_t)(u >> 32), lo = (uint32_t)u;
 #pragma unroll
@@ -100,14 +94,14 @@ __device__ __forceinline__ void quad_hashes(const uint64_t* __restrict__ row_key
                         const uint32_t src = (lane & ~7u) + j;
                         const uint32_t ohi = __shfl_sync(0xFFFFFFFFu, hi, src);
                         const uint32_t olo = __shfl_sync(0xFFFFFFFFu, lo, src);
-                        h[k + j] = quad_from_draw(((uint64_t)ohi << 32) | olo, 5, G, t << 2);
+                        h[k + j] = quad_from_draw(P, ((uint64_t)ohi << 32) | olo, i, wbase);
                     }
             }
         }
     } else {
 #pragma unroll
         for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
-            if (row < r) h[row] = quad_hash(row_key[row], log2g, G, t << 2);
+            if (row < r) h[row] = quad_from_draw(P, stream(P.row_key[row], (uint64_t)(i >> P.log2g) + 1), i, wbase);
     }
 }
 

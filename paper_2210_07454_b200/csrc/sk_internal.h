@@ -15,7 +15,10 @@ struct Params {
     uint64_t row_key[kMaxRows];
     uint32_t d, n, r, c;
     uint32_t cs;        // row stride of every table in floats (c rounded up to 32)
-    uint32_t log2g, G;  // hash group size 2^log2g and number of bucket groups c >> log2g
+    uint32_t log2g, G;  // hash group size 2^log2g; number of blocks a group chooses from (c >> log2g, or the
+                        // lines of a window in the windowed family)
+    uint32_t win_cw;      // windowed family: buckets per window (32 * lines), 0 = plain family
+    uint32_t win_panels;  // windowed family: windows per row = c / win_cw
     uint32_t k;
     float beta1, beta2, lr;
 };
@@ -52,6 +55,10 @@ int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st);
 int launch_set_bits(const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st);
 int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,
                          cudaStream_t st);
+// windowed hash family: shared-memory accumulation, at most kWinMaxWorkers workers per launch; -1 if it cannot run
+constexpr uint32_t kWinMaxWorkers = 8;
+int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, int sm_count,
+                             cudaStream_t st);
 int launch_second_moment(const Params& P, const MomentArgs& A, const uint32_t* I_prev, uint32_t k_prev,
                          cudaStream_t st);
 int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStream_t st);

@@ -74,7 +74,7 @@ __device__ __forceinline__ float4 medians4(const Params& P, const float* __restr
     constexpr int RMAX = R > 0 ? R : (int)kMaxRows;
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
     Quad h[RMAX];
-    quad_hashes<RMAX>(P.row_key, r, P.log2g, P.G, t, h);
+    quad_hashes<RMAX>(P, r, t, h);
     float qx[RMAX], qy[RMAX], qz[RMAX], qw[RMAX];
 #pragma unroll
     for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
@@ -97,7 +97,7 @@ __device__ __forceinline__ float median1(const Params& P, const float* __restric
     float q[kMaxRows];
     for (uint32_t row = 0; row < P.r; ++row) {
         uint32_t b; float s;
-        coord_hash(P.row_key[row], P.log2g, P.G, j, b, s);
+        coord_hash(P, P.row_key[row], j, b, s);
         q[row] = s * __ldg(sum + (uint64_t)row * P.cs + b);
     }
     return median_any(q, P.r);
@@ -385,7 +385,7 @@ k_hash_export(const __grid_constant__ Params P, uint32_t row, uint64_t i0, uint6
               int8_t* sgn) {
     for (uint64_t t = blockIdx.x * (uint64_t)kThreads + threadIdx.x; t < count; t += (uint64_t)gridDim.x * kThreads) {
         uint32_t b; float s;
-        coord_hash(P.row_key[row], P.log2g, P.G, (uint32_t)(i0 + t), b, s);
+        coord_hash(P, P.row_key[row], (uint32_t)(i0 + t), b, s);
         idx[t] = b;
         sgn[t] = s < 0.0f ? (int8_t)-1 : (int8_t)1;
     }

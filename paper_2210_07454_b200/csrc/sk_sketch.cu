@@ -94,7 +94,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
     for (uint32_t it = 0; it < trips; ++it) {            // uniform trip count: the hash exchange needs whole warps
         const uint32_t t = (it * gridDim.x + blockIdx.x) * kThreads + threadIdx.x;
         Quad h[RMAX];
-        quad_hashes<RMAX>(P.row_key, r, P.log2g, P.G, t < d4 ? t : d4 - 1, h);
+        quad_hashes<RMAX>(P, r, t < d4 ? t : d4 - 1, h);
         if (t >= d4) continue;
         const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
         float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);     // running gradient sum in worker order (used on I_{t-1})
@@ -157,7 +157,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
             A.e[q] = a;
             for (uint32_t row = 0; row < P.r; ++row) {
                 uint32_t b; float s;
-                coord_hash(P.row_key[row], P.log2g, P.G, j, b, s);
+                coord_hash(P, P.row_key[row], j, b, s);
                 atomicAdd(A.tables + (uint64_t)w * tstride + (uint64_t)row * P.cs + b, s * a);
             }
         }

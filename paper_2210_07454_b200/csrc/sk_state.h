@@ -1,0 +1,37 @@
+// The handle behind the C ABI (private to the library's own translation units).
+#pragma once
+#include "../../include/sketched_amsgrad.h"
+#include "sk_internal.h"
+
+#include <vector>
+
+struct TimeRec { int stage; cudaEvent_t a, b; };
+
+struct sk_state {
+    sk::Params P{};
+    uint64_t seed = 0, t = 0;
+    float eps = 0;
+    uint32_t k_prev = 0;
+    int sm_count = 148;
+    size_t l2_bytes = 0;
+    int64_t worker_chunk = 0;
+    int64_t window_lines = 0;
+    int64_t sketch_ctas_per_sm = 64;
+    bool timing = false;
+    cudaStream_t stream = nullptr;
+    // device memory owned by the handle
+    float *m = nullptr, *e = nullptr, *v = nullptr, *vhat = nullptr, *tables = nullptr, *sum = nullptr;
+    uint32_t *vstamp = nullptr, *I = nullptr, *I_prev = nullptr, *hist = nullptr, *hist2 = nullptr;
+    uint32_t *keys = nullptr, *bitmap = nullptr;
+    float* gsum = nullptr;
+    uint64_t bitmap_bytes = 0;
+    sk::Select* sel = nullptr;
+    sk::Cand *cand = nullptr, *cand2 = nullptr;
+    float *stage_grads = nullptr, *stage_x = nullptr;
+    // timing
+    std::vector<TimeRec> recs;
+    std::vector<cudaEvent_t> free_events;
+    double ms[SK_NUM_STAGES] = {0};
+    uint64_t launches[SK_NUM_STAGES] = {0};
+    uint64_t timed_steps = 0;
+};

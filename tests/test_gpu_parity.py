@@ -28,13 +28,13 @@ def _workload(base, **over):
     return w
 
 
-def _pair(w, log2g=None, threads=8):
+def _pair(w, log2g=None, threads=8, window_lines=None):
     b = _binding()
     gpu = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                            eps=w.eps, log2g=log2g)
+                            eps=w.eps, log2g=log2g, window_lines=window_lines)
     lg = gpu.get_option("log2g")
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=lg, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                        eps=w.eps, threads=threads)
+                        eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"))
     return gpu, ora
 
 
@@ -62,8 +62,8 @@ def test_hash_bit_exact(log2g, c):
 
 
 # ------------------------------------------------------------------------------------------------ steps
-def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True):
-    gpu, ora = _pair(w, log2g)
+def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True, window_lines=None):
+    gpu, ora = _pair(w, log2g, window_lines=window_lines)
     src = _source(w, cfg_id=cfg_id)
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
@@ -101,6 +101,62 @@ def test_c1_free_running():
 @pytest.mark.parametrize("log2g", [0, 1, 2, 3, 4])
 def test_c1_other_group_sizes(log2g):
     _run_steps(_workload("C1"), 3, log2g=log2g)
+
+
+@pytest.mark.parametrize("L", [1, 4, 8, 16])
+def test_windowed_hash_bit_exact(L):
+    b = _binding()
+    d, r, c = 300_000, 7, 250_000
+    gpu = b.SketchedAMSGrad(d, 1, r, c, 1, seed=99, window_lines=L)
+    idx = torch.empty(d, dtype=torch.int32, device="cuda")
+    sgn = torch.empty(d, dtype=torch.int8, device="cuda")
+    for row in (0, 3, 6):
+        gpu.hash(row, 0, d, idx, sgn)
+        gpu.sync()
+        wb, ws = oracle.hash_family(99, 5, c, row, 0, d, window_lines=L)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), wb)
+        assert np.array_equal(sgn.cpu().numpy(), ws)
+
+
+def test_windowed_c1_ten_steps_teacher_forced():
+    _run_steps(_workload("C1"), 10, window_lines=8)
+
+
+WINDOWED = {
+    "ragged_unit": dict(d=1024 * 37 + 12, n=4, r=7, c=3000, k=700, L=4),     # last unit partial, c % window != 0
+    "two_launches": dict(d=40_000, n=11, r=5, c=4096, k=400, L=8),           # 8 + 3 workers
+    "odd_workers": dict(d=50_000, n=5, r=5, c=4096, k=500, L=16),
+    "one_window": dict(d=8192, n=2, r=3, c=300, k=80, L=8),                  # a single panel
+    "many_rows": dict(d=12_000, n=2, r=16, c=2048, k=120, L=2),
+    "short": dict(d=512, n=3, r=5, c=1024, k=20, L=4),                       # less than one unit
+    "scalar_path": dict(d=10_007, n=3, r=5, c=1000, k=333, L=4),             # d % 4 != 0: scalar kernels, same family
+}
+
+
+@pytest.mark.parametrize("case", sorted(WINDOWED))
+def test_windowed_edge_cases(case):
+    cfg = dict(WINDOWED[case])
+    L = cfg.pop("L")
+    w = _workload("C1", name="E", steps=3, recipe="planted", **cfg)
+    _run_steps(w, 3, cfg_id=8, window_lines=L)
+
+
+def test_windowed_integer_inputs_are_bit_exact():
+    d, n, r, c, k = 200_000, 4, 5, 4096, 1000
+    b = _binding()
+    gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0, window_lines=8)
+    ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=5, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0, threads=8, window_lines=8)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    x = torch.zeros(d, device="cuda")
+    x_ref = np.zeros(d, np.float32)
+    g = torch.randint(-8, 9, (n, d), generator=gen, device="cuda").float()
+    gpu.step(g, x)
+    gpu.sync()
+    ora.step(g.cpu().numpy(), x_ref)
+    assert np.array_equal(gpu.get("tables"), ora.field("tables"))
+    assert np.array_equal(gpu.get("sum"), ora.field("sum"))
+    assert np.array_equal(gpu.get("I"), ora.field("I"))
+    assert np.array_equal(x.cpu().numpy(), x_ref)
 
 
 EDGE = {

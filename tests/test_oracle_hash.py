@@ -130,3 +130,57 @@ def test_non_divisible_c_leaves_tail_buckets_unused():
     c, log2g = 250_000, 5            # 250000 = 32*7812 + 16
     b, _ = oracle.hash_family(0, log2g, c, 0, 0, 500_000)
     assert b.max() < 7812 * 32
+
+
+# ---------------------------------------------------------------------------------------------- windowed family
+def _family_w(seed, L, c, row, i):
+    """Windowed family (g = 32) evaluated with Python integers."""
+    cw = 32 * L
+    P = c // cw
+    K = _mix((seed + (row + 1) * GOLDEN_GAMMA) & M64)
+    q, o = divmod(i, 32)
+    u = _mix((K + (q + 1) * GOLDEN_GAMMA) & M64)
+    hi, lo = divmod(u, 1 << 32)
+    line, rem = divmod(hi * L, 1 << 32)
+    p = (rem * 32) >> 32
+    return ((i // 1024) % P) * cw + 32 * line + (o ^ p), (-1 if (lo >> o) & 1 else 1)
+
+
+@pytest.mark.parametrize("L", [1, 4, 8, 16])
+@pytest.mark.parametrize("c", [2048, 250_000, 1_000_000])
+def test_windowed_family_matches_bigint_definition(L, c):
+    for seed in (0, 77):
+        for row in (0, 4):
+            for i0 in (0, 1000, 1024 * 977 + 5, 2**32 - 70):
+                b, s = oracle.hash_family(seed, 5, c, row, i0, 64, window_lines=L)
+                for t in range(64):
+                    assert (int(b[t]), int(s[t])) == _family_w(seed, L, c, row, i0 + t)
+
+
+def test_windowed_family_structure():
+    c, L, N = 250_000, 8, 1024 * 3000
+    cw, P = 32 * L, 250_000 // (32 * L)
+    b, s = oracle.hash_family(2, 5, c, 1, 0, N, window_lines=L)
+    unit = np.arange(N) // 1024
+    # every coordinate lands in the window of its unit's panel
+    assert np.array_equal(b // cw, unit % P)
+    assert b.max() < P * cw <= c
+    # inside a group: a permutation of one aligned line
+    blk = b.reshape(-1, 32)
+    assert np.all(blk // 32 == blk[:, :1] // 32)
+    assert np.all(np.sort(blk % 32, axis=1) == np.arange(32))
+    # lines inside a window are used uniformly
+    line = (blk[:, 0] % cw) // 32
+    cnt = np.bincount(line, minlength=L).astype(np.float64)
+    assert abs(cnt / cnt.sum() - 1 / L).max() < 0.01
+    assert abs(s.astype(np.float64).mean()) < 5 / np.sqrt(N)
+    # pair collisions: 1/cw between different groups of one panel, none across panels
+    one = b[unit % P == 3]
+    cc = np.bincount(one - 3 * cw, minlength=cw).astype(np.float64)
+    pairs = (cc * (cc - 1) / 2).sum()
+    n1 = one.size
+    cross = n1 * (n1 - 1) / 2 - (n1 // 32) * 32 * 31 / 2
+    assert abs(pairs / cross * cw - 1) < 0.05
+    # the row as a whole is still filled evenly: about N/c coordinates per bucket
+    tot = np.bincount(b, minlength=c)[: P * cw].astype(np.float64)
+    assert abs(tot.mean() - N / (P * cw)) < 1e-9 and tot.std() / tot.mean() < 0.5
