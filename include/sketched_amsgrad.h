@@ -111,6 +111,26 @@ uint64_t sk_algorithmic_bytes(const sk_state* state);
 #define SK_NUM_STAGES 8
 int sk_get_timing(sk_state* state, double* ms, uint64_t* launches);
 
+/* The paper has no counterpart for this entry point; it exists for callers that must not allocate.
+ * Some callers cannot call cudaMalloc at the moment they need a selection: code running under a framework whose
+ * caching allocator owns the device and forbids foreign allocations, code on a latency path that cannot afford
+ * cudaMalloc's implicit device-wide synchronisation, or code running after device memory has been filled on
+ * purpose.  sk_select_static re-runs the top-k selection of the handle's LAST step (same inputs: the aggregated
+ * sketch and vhat the handle holds) and writes the k selected indices, in no particular order, to idx_out
+ * (DEVICE pointer, k uint32, caller-owned).  It calls no cudaMalloc, cudaFree or any other allocating routine:
+ * all its scratch (histograms, ranking keys, candidate lists; about 5 MB) lives in one file-scope device array
+ * inside the library, which every GPU that loads the library holds until the process exits.
+ *   - Limit: d <= SK_STATIC_MAX_D; larger handles are rejected with SK_EINVAL and a message naming the limit.
+ *     SK_ESTATE if the handle has not taken a step yet.
+ *   - The first call on a device resolves the device address of the scratch array (once per device, with that
+ *     device current).  Make that first call before starting any stream capture.
+ *   - Every call, from every handle and stream, shares the one array, and the array keeps the previous call's
+ *     contents; the entry point clears the parts that must start at zero itself.  Two calls that overlap on the
+ *     GPU (different streams or threads) race on the array: serialise them.
+ *   - Asynchronous on the handle's stream, like sk_step; the handle's own state is read, not modified. */
+#define SK_STATIC_MAX_D 262144u
+int sk_select_static(sk_state* state, uint32_t* idx_out);
+
 const char* sk_last_error(void);
 const char* sk_version(void);
 

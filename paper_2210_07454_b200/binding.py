@@ -14,8 +14,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsketched_amsgrad.so")
 
 EXPORTS = ["sk_create", "sk_step", "sk_step_host", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
-           "sk_get_option", "sk_hash", "sk_get", "sk_set", "sk_algorithmic_bytes", "sk_get_timing",
+           "sk_get_option", "sk_hash", "sk_get", "sk_set", "sk_algorithmic_bytes", "sk_get_timing", "sk_select_static",
            "sk_last_error", "sk_version"]
+STATIC_MAX_D = 262144
 NUM_STAGES = 8
 STAGE_NAMES = ["zero_tables", "second_moment", "moment_sketch", "sum_tables", "unsketch_hist",
                "unsketch_emit", "refine", "apply"]
@@ -50,6 +51,7 @@ def lib() -> C.CDLL:
         L.sk_algorithmic_bytes.restype = u64; L.sk_algorithmic_bytes.argtypes = [vp]
         L.sk_get_timing.restype = C.c_int
         L.sk_get_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u64)]
+        L.sk_select_static.restype = C.c_int; L.sk_select_static.argtypes = [vp, vp]
         L.sk_last_error.restype = C.c_char_p; L.sk_last_error.argtypes = []
         L.sk_version.restype = C.c_char_p; L.sk_version.argtypes = []
         _lib = L
@@ -146,6 +148,12 @@ class SketchedAMSGrad:
 
     def set(self, field: str, value) -> None:
         _check(lib().sk_set(self._h, field.encode(), _ptr(value) if _nbytes(value) else 0, _nbytes(value)))
+
+    def select_static(self, idx_out) -> None:
+        """Re-runs the last step's top-k selection into `idx_out` (CUDA tensor of k int32/uint32) without
+        allocating: for callers that may not call cudaMalloc.  Shares one static scratch array with every other
+        call, so calls must not overlap on the GPU; handles with d > STATIC_MAX_D are rejected."""
+        _check(lib().sk_select_static(self._h, _ptr(idx_out)))
 
     def algorithmic_bytes(self) -> int:
         return int(lib().sk_algorithmic_bytes(self._h))

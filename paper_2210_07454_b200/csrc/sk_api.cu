@@ -187,6 +187,9 @@ Field field_of(const char* name) {
 
 }  // namespace
 
+// lets the library's other translation units report through sk_last_error()
+int sk_fail_message(int code, const char* message) { return fail(code, "%s", message); }
+
 extern "C" {
 
 const char* sk_last_error(void) { return g_err.c_str(); }
