@@ -56,7 +56,7 @@ int launch_set_bits(const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStr
 int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,
                          cudaStream_t st);
 // windowed hash family: shared-memory accumulation, at most kWinMaxWorkers workers per launch; -1 if it cannot run
-constexpr uint32_t kWinMaxWorkers = 8;
+constexpr uint32_t kWinMaxWorkers = 4;
 int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, int sm_count,
                              cudaStream_t st);
 int launch_second_moment(const Params& P, const MomentArgs& A, const uint32_t* I_prev, uint32_t k_prev,

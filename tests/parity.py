@@ -84,10 +84,18 @@ def compare_step(gpu, ora, x_gpu, x_ref, x_before, lr, check_tables=True, x_gpu_
     diff = index_sets_agree(I_gpu, ora.field("I"), est_ref, k, scale=sc)
     keep = np.ones(d, bool)
     keep[diff] = False
-    close(gpu.get("m"), ora.field("m"), "m", groups_axis=0)
+    m_gpu, m_ref = gpu.get("m"), ora.field("m")
+    for w in range(n):                                   # one worker at a time: its own RMS, bounded temporaries
+        close(m_gpu[w], m_ref[w], f"m[{w}]")
+    del m_gpu
     e_gpu, e_ref = gpu.get("e"), ora.field("e")
-    close(e_gpu[:, keep], e_ref[:, keep], "e", groups_axis=0)
+    for w in range(n):
+        if diff.size:
+            close(e_gpu[w][keep], e_ref[w][keep], f"e[{w}]")
+        else:
+            close(e_gpu[w], e_ref[w], f"e[{w}]")
     assert not e_gpu[:, I_gpu].any(), "e must be zero on I_t"
+    del e_gpu
     # x: compare the CHANGE against lr * RMS(Delta) scale
     dx_gpu = np.asarray(x_gpu, np.float64) - (x_before if x_gpu_before is None else np.asarray(x_gpu_before, np.float64))
     dx_ref = np.asarray(x_ref, np.float64) - x_before
