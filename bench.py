@@ -29,7 +29,10 @@ DEFAULT_WORKLOAD = "C3"      # d = 25.6M: the size the headline metric is quoted
 
 # DRAM traffic of the dominant kernel (moments + sketch) from an ncu capture, in bytes per worker-coordinate,
 # valid only for the kernel source it was taken on (sha256 of sk_sketch.cu); otherwise reported as null.
-NCU_TRAFFIC = {"sha256": None, "bytes_per_worker_coord": None}
+# Capture: C3 at half size (profiles/c3_half_moment_sketch_ncu_full.md): 1.2539 GB read + 0.7953 GB written for
+# 1.024e8 worker-coordinates; the traffic grows in proportion to n*d, so it is scaled to the timed launch.
+NCU_TRAFFIC = {"sha256": "344c47bb3055661d720ed9a8c3da46cc96e99f3df22309b02d6b5738241f0c38",
+               "bytes_per_worker_coord": 20.01}
 
 
 def _peaks():
