@@ -171,6 +171,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--log2g", type=int, default=None)
     ap.add_argument("--window-lines", type=int, default=None, help="windowed hash family: lines per window (0 = plain)")
+    ap.add_argument("--window-workers", type=int, default=0, help="workers per launch of the windowed sketch kernel")
     ap.add_argument("--worker-chunk", type=int, default=0)
     ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -204,6 +205,8 @@ def main():
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
                                   eps=w.eps, log2g=args.log2g, window_lines=args.window_lines)
     opt.set_option("worker_chunk", args.worker_chunk)
+    if args.window_workers:
+        opt.set_option("window_workers", args.window_workers)
     if args.sketch_ctas:
         opt.set_option("sketch_ctas_per_sm", args.sketch_ctas)
     # gradient buffers rotate so that no step finds its inputs in L2 (each set is far larger than L2 anyway)

@@ -123,7 +123,7 @@ int do_step(sk_state* s, const float* grads, float* x) {
     A.v = s->v; A.vhat = s->vhat; A.vstamp = s->vstamp; A.bitmap = s->bitmap;
     A.step = t; A.members = s->k_prev ? 1u : 0u;
     const bool windowed = vec && P.win_cw != 0;
-    const uint32_t wc = windowed ? std::min<uint32_t>(sk::kWinMaxWorkers, P.n) : chunk_of(s);
+    const uint32_t wc = windowed ? std::min<uint32_t>((uint32_t)s->window_workers, P.n) : chunk_of(s);
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
         const uint32_t nw = std::min(wc, P.n - w0);
@@ -331,6 +331,11 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         refresh_hash(s);
         return SK_OK;
     }
+    if (!strcmp(key, "window_workers")) {
+        if (value < 1 || value > (int64_t)sk::kWinMaxWorkers) return fail(SK_EINVAL, "window_workers must be in 1..4");
+        s->window_workers = value;
+        return SK_OK;
+    }
     if (!strcmp(key, "worker_chunk")) {
         if (value < 0) return fail(SK_EINVAL, "worker_chunk must be >= 0");
         s->worker_chunk = value;
@@ -354,6 +359,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     if (!s || !key || !value) return fail(SK_EINVAL, "null argument");
     if (!strcmp(key, "log2g")) *value = s->P.log2g;
     else if (!strcmp(key, "window_lines")) *value = s->window_lines;
+    else if (!strcmp(key, "window_workers")) *value = s->window_workers;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
     else if (!strcmp(key, "sketch_ctas_per_sm")) *value = s->sketch_ctas_per_sm;

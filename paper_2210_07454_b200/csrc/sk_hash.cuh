@@ -82,10 +82,7 @@ __device__ __forceinline__ void quad_hashes(const Params& P, uint32_t r, uint32_
 #pragma unroll
         for (uint32_t k = 0; k < (uint32_t)RMAX; k += 8) {
             if (k < r) {
-                uint64_t key = 0;
-#pragma unroll
-                for (uint32_t j = 0; j < 8; ++j)
-                    if (k + j < (uint32_t)RMAX && j == li) key = P.row_key[k + j];
+                const uint64_t key = P.row_key[(k + li) & (kMaxRows - 1u)];   // indexed read of the kernel parameter
                 const uint64_t u = (k + li < r) ? stream(key, (uint64_t)q + 1) : 0ull;
                 const uint32_t hi = (uint32_t)(u >> 32), lo = (uint32_t)u;
 #pragma unroll
@@ -111,11 +108,11 @@ __device__ __forceinline__ float flip(float a, uint32_t bit) {  // a * (bit ? -1
 
 // signed and permuted: out element e = s(l) * a_l with l = e xor p3
 __device__ __forceinline__ float4 quad_scatter(const Quad h, float4 a) {
-    const uint32_t s = h.p3sgn >> 2;
-    a.x = flip(a.x, s & 1u);
-    a.y = flip(a.y, (s >> 1) & 1u);
-    a.z = flip(a.z, (s >> 2) & 1u);
-    a.w = flip(a.w, (s >> 3) & 1u);
+    const uint32_t s = h.p3sgn;                       // sign bit of local coordinate l is bit 2 + l
+    a.x = __uint_as_float(__float_as_uint(a.x) ^ ((s << 29) & 0x80000000u));
+    a.y = __uint_as_float(__float_as_uint(a.y) ^ ((s << 28) & 0x80000000u));
+    a.z = __uint_as_float(__float_as_uint(a.z) ^ ((s << 27) & 0x80000000u));
+    a.w = __uint_as_float(__float_as_uint(a.w) ^ ((s << 26) & 0x80000000u));
     if (h.p3sgn & 1u) { float t = a.x; a.x = a.y; a.y = t; t = a.z; a.z = a.w; a.w = t; }
     if (h.p3sgn & 2u) { float t = a.x; a.x = a.z; a.z = t; t = a.y; a.y = a.w; a.w = t; }
     return a;
@@ -125,11 +122,11 @@ __device__ __forceinline__ float4 quad_scatter(const Quad h, float4 a) {
 __device__ __forceinline__ float4 quad_gather(const Quad h, float4 cch) {
     if (h.p3sgn & 1u) { float t = cch.x; cch.x = cch.y; cch.y = t; t = cch.z; cch.z = cch.w; cch.w = t; }
     if (h.p3sgn & 2u) { float t = cch.x; cch.x = cch.z; cch.z = t; t = cch.y; cch.y = cch.w; cch.w = t; }
-    const uint32_t s = h.p3sgn >> 2;
-    cch.x = flip(cch.x, s & 1u);
-    cch.y = flip(cch.y, (s >> 1) & 1u);
-    cch.z = flip(cch.z, (s >> 2) & 1u);
-    cch.w = flip(cch.w, (s >> 3) & 1u);
+    const uint32_t s = h.p3sgn;                       // sign bit of local coordinate l is bit 2 + l
+    cch.x = __uint_as_float(__float_as_uint(cch.x) ^ ((s << 29) & 0x80000000u));
+    cch.y = __uint_as_float(__float_as_uint(cch.y) ^ ((s << 28) & 0x80000000u));
+    cch.z = __uint_as_float(__float_as_uint(cch.z) ^ ((s << 27) & 0x80000000u));
+    cch.w = __uint_as_float(__float_as_uint(cch.w) ^ ((s << 26) & 0x80000000u));
     return cch;
 }
 

@@ -179,7 +179,7 @@ __device__ __forceinline__ void block_append(uint32_t n_a, uint32_t n_b, uint32_
     __shared__ uint32_t warp_tot[kThreads / 32];
     __shared__ uint32_t block_base[2];
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const uint32_t packed = n_a | (n_b << 16);              // each <= 4 per thread, <= 1024 per block
+    const uint32_t packed = n_a | (n_b << 16);              // each <= 16 per thread, <= 4096 per block
     uint32_t incl = packed;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -215,38 +215,52 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, Select* sel, uint32_t* I_o
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh2[b] = 0;
     __syncthreads();
     const uint32_t bin = sel->bin;
+    constexpr uint32_t U = 4;                                   // key loads in flight per thread and block-wide append
     const uint32_t items = VEC ? (d >> 2) : d;
-    const uint32_t trips = (items + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
+    const uint32_t tile = U * kThreads;
+    const uint32_t trips = (items + gridDim.x * tile - 1) / (gridDim.x * tile);
     for (uint32_t it = 0; it < trips; ++it) {
-        const uint32_t t = (it * gridDim.x + blockIdx.x) * kThreads + threadIdx.x;
-        uint32_t kq[4], idx0 = VEC ? (t << 2) : t, nk = 0;
-        if (t < items) {
-            if (VEC) {
-                const uint4 k4 = __ldcs((const uint4*)keys + t);
-                kq[0] = k4.x; kq[1] = k4.y; kq[2] = k4.z; kq[3] = k4.w;
-                nk = 4;
-            } else {
-                kq[0] = keys[t];
-                nk = 1;
+        const uint32_t t0 = (it * gridDim.x + blockIdx.x) * tile + threadIdx.x;
+        uint32_t kq[U][4], nk[U];
+#pragma unroll
+        for (uint32_t u = 0; u < U; ++u) {
+            const uint32_t t = t0 + u * kThreads;
+            nk[u] = 0;
+            if (t < items) {
+                if (VEC) {
+                    const uint4 k4 = __ldcs((const uint4*)keys + t);
+                    kq[u][0] = k4.x; kq[u][1] = k4.y; kq[u][2] = k4.z; kq[u][3] = k4.w;
+                    nk[u] = 4;
+                } else {
+                    kq[u][0] = keys[t];
+                    nk[u] = 1;
+                }
             }
         }
         uint32_t n_out = 0, n_cand = 0;
 #pragma unroll
-        for (uint32_t q = 0; q < 4; ++q)
-            if (q < nk) {
-                const uint32_t b = kq[q] >> kHistShift;
-                if (b == bin) { atomicAdd(&sh2[(kq[q] >> 7) & (kHistBins - 1u)], 1u); ++n_cand; }
-                n_out += b > bin;
-            }
-        uint32_t po, pc;
-        block_append(n_out, n_cand, &sel->cnt_out, &sel->cnt_cand, po, pc);
+        for (uint32_t u = 0; u < U; ++u)
 #pragma unroll
-        for (uint32_t q = 0; q < 4; ++q)
-            if (q < nk) {
-                const uint32_t b = kq[q] >> kHistShift;
-                if (b > bin) I_out[po++] = idx0 + q;
-                else if (b == bin) { cand[pc].key = kq[q]; cand[pc].idx = idx0 + q; ++pc; }
-            }
+            for (uint32_t q = 0; q < 4; ++q)
+                if (q < nk[u]) {
+                    const uint32_t b = kq[u][q] >> kHistShift;
+                    if (b == bin) { atomicAdd(&sh2[(kq[u][q] >> 7) & (kHistBins - 1u)], 1u); ++n_cand; }
+                    n_out += b > bin;
+                }
+        uint32_t po, pc;
+        block_append(n_out, n_cand, &sel->cnt_out, &sel->cnt_cand, po, pc);   // <= 16 per thread, <= 4096 per block
+#pragma unroll
+        for (uint32_t u = 0; u < U; ++u) {
+            const uint32_t t = t0 + u * kThreads;
+            const uint32_t idx0 = VEC ? (t << 2) : t;
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q)
+                if (q < nk[u]) {
+                    const uint32_t b = kq[u][q] >> kHistShift;
+                    if (b > bin) I_out[po++] = idx0 + q;
+                    else if (b == bin) { cand[pc].key = kq[u][q]; cand[pc].idx = idx0 + q; ++pc; }
+                }
+        }
     }
     __syncthreads();
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
@@ -431,7 +445,7 @@ int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cud
 
 int launch_emit(const Params& P, const uint32_t* keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2,
                 int sm_count, cudaStream_t st) {
-    if (P.d % 4 == 0) k_emit<true><<<grid_for(P.d >> 2, sm_count, 8), kThreads, 0, st>>>(P.d, keys, sel, I_out, cand, hist2);
+    if (P.d % 4 == 0) k_emit<true><<<grid_for((P.d >> 2) / 4 + 1, sm_count, 8), kThreads, 0, st>>>(P.d, keys, sel, I_out, cand, hist2);
     else k_emit<false><<<grid_for(P.d, sm_count, 8), kThreads, 0, st>>>(P.d, keys, sel, I_out, cand, hist2);
     return 1;
 }
