@@ -29,10 +29,10 @@ DEFAULT_WORKLOAD = "C3"      # d = 25.6M: the size the headline metric is quoted
 
 # DRAM traffic of the dominant kernel (moments + sketch) from an ncu capture, in bytes per worker-coordinate,
 # valid only for the kernel source it was taken on (sha256 of sk_sketch.cu); otherwise reported as null.
-# Capture: C3 at half size (profiles/c3_half_moment_sketch_ncu_full.md): 1.2539 GB read + 0.7953 GB written for
+# Capture: C3 at half size (profiles/c3_half_moment_sketch_ncu_full.md): 1.2539 GB read + 0.7941 GB written for
 # 1.024e8 worker-coordinates; the traffic grows in proportion to n*d, so it is scaled to the timed launch.
-NCU_TRAFFIC = {"sha256": "344c47bb3055661d720ed9a8c3da46cc96e99f3df22309b02d6b5738241f0c38",
-               "bytes_per_worker_coord": 20.01}
+NCU_TRAFFIC = {"sha256": "d7fcc51852afaab3c176519dbf7d85174eb2aa934de0f0ce02f90c93e0957250",
+               "bytes_per_worker_coord": 20.00}
 
 
 def _peaks():
@@ -172,6 +172,7 @@ def main():
     ap.add_argument("--log2g", type=int, default=None)
     ap.add_argument("--window-lines", type=int, default=None, help="windowed hash family: lines per window (0 = plain)")
     ap.add_argument("--window-workers", type=int, default=0, help="workers per launch of the windowed sketch kernel")
+    ap.add_argument("--window-red-rows", type=int, default=-1, help="rows the windowed kernel sketches by L2 reductions")
     ap.add_argument("--worker-chunk", type=int, default=0)
     ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -207,6 +208,8 @@ def main():
     opt.set_option("worker_chunk", args.worker_chunk)
     if args.window_workers:
         opt.set_option("window_workers", args.window_workers)
+    if args.window_red_rows >= 0:
+        opt.set_option("window_red_rows", args.window_red_rows)
     if args.sketch_ctas:
         opt.set_option("sketch_ctas_per_sm", args.sketch_ctas)
     # gradient buffers rotate so that no step finds its inputs in L2 (each set is far larger than L2 anyway)
@@ -217,15 +220,14 @@ def main():
     x = src.x0()
     torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()                              # started early: nvidia-smi takes a while to deliver samples
     for t in range(args.warmup):
         opt.step(gsets[t % nsets], x)
     opt.sync()
     opt.timing()                                     # clear launch counters
     opt.set_option("timing", 0 if args.no_stage_timing else 1)
-
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     if world > 1:
         import torch.distributed as dist
         dist.barrier()

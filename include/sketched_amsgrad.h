@@ -70,8 +70,14 @@ int sk_sync(sk_state* state);
 /* Options (integers):
  *   "log2g"        hash group size g = 2^log2g, 0..5 (Section II-C fixes no hash family; see sk_hash).
  *                  Only before the first step.  Default: the largest value <= 5 with 2^log2g <= c.
+ *   "window_lines" L > 0 selects the windowed variant of the hash family (needs g = 32, 32*L <= c): units of
+ *                  1024 coordinates map into one aligned window of 32*L buckets per row, which lets the sketch
+ *                  kernel accumulate in shared memory.  0 (default) = plain family.  Only before the first step.
+ *   "window_workers" (1..4) workers per launch and "window_red_rows" (0..4) rows sketched by L2 reductions
+ *                  instead of shared-memory windows, both for the windowed kernel only.
  *   "worker_chunk" workers whose tables are accumulated concurrently by the sketch kernel (0 = automatic,
  *                  sized so that the concurrently updated tables stay resident in L2).
+ *   "sketch_ctas_per_sm" grid size of the plain sketch kernel in blocks per SM (default 64: one tile per block).
  *   "timing"       1 = record CUDA events around each stage (see sk_get_timing); 0 = off (default). */
 int sk_set_option(sk_state* state, const char* key, int64_t value);
 /* Also readable: "I_count" (entries "I" currently holds: 0 before the first step, else k unless sk_set installed
@@ -104,8 +110,9 @@ int sk_set(sk_state* state, const char* field, const void* buf, uint64_t bytes);
  * written) + 12*n*k + 24*k (sparse gathers and updates on I_{t-1} and I_t). */
 uint64_t sk_algorithmic_bytes(const sk_state* state);
 
-/* Stage timing (option "timing" = 1).  Stages: 0 zero tables, 1 second moments on I_{t-1}, 2 moments+sketch,
- * 3 sum of sketches, 4 unsketch+histogram, 5 unsketch+emit, 6 threshold refinement, 7 apply on I_t.
+/* Stage timing (option "timing" = 1).  Stages: 0 zero tables, 1 unused (the second moments on I_{t-1} are updated
+ * inside stage 4), 2 moments+sketch, 3 sum of sketches, 4 ranking keys + histogram (+ v, vhat on I_{t-1}),
+ * 5 emit above the threshold bin, 6 threshold refinement, 7 apply on I_t.
  * Adds up the events of all steps since the last call into ms[0..7] (milliseconds) and launches[0..7]
  * (kernel launches), then clears them.  Synchronises the stream.  Returns the number of steps covered, or <0. */
 #define SK_NUM_STAGES 8

@@ -133,7 +133,7 @@ int do_step(sk_state* s, const float* grads, float* x) {
         }
         StageTimer tm(s, 2);     // moments + sketch; also leaves the gradient sums on I_{t-1} in gsum
         if (windowed) {
-            const int l = sk::launch_moment_sketch_win(P, A, w0, nw, s->sm_count, st);
+            const int l = sk::launch_moment_sketch_win(P, A, w0, nw, (uint32_t)s->window_red_rows, s->sm_count, st);
             if (l < 0) return fail(SK_ECUDA, "the windowed sketch kernel does not fit in shared memory (window_lines=%lld, r=%u)",
                                    (long long)s->window_lines, P.r);
             tm.done(l);
@@ -141,17 +141,14 @@ int do_step(sk_state* s, const float* grads, float* x) {
             tm.done(sk::launch_moment_sketch(P, A, w0, nw, vec, s->sm_count * (int)s->sketch_ctas_per_sm, st));
         }
     }
-    {   // v, vhat on I_{t-1} from those sums
-        StageTimer tm(s, 1);
-        tm.done(sk::launch_second_moment(P, A, s->I_prev, s->k_prev, st));
-    }
     {
         StageTimer tm(s, 3);
         tm.done(sk::launch_sum_tables(P, s->tables, s->sum, st));
     }
     {
         StageTimer tm(s, 4);
-        int l = sk::launch_unsketch_hist(P, s->sum, s->vhat, s->keys, s->hist, vec, s->sm_count, st);
+        // ranking keys; v and vhat on I_{t-1} are brought up to date on the way, from the sums in gsum
+        int l = sk::launch_unsketch_hist(P, A, s->sum, s->keys, s->hist, vec, s->sm_count, st);
         l += sk::launch_pick_bin(P, s->hist, s->sel, 0, st);
         tm.done(l);
     }
@@ -331,6 +328,11 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         refresh_hash(s);
         return SK_OK;
     }
+    if (!strcmp(key, "window_red_rows")) {
+        if (value < 0 || value > 4) return fail(SK_EINVAL, "window_red_rows must be in 0..4");
+        s->window_red_rows = value;
+        return SK_OK;
+    }
     if (!strcmp(key, "window_workers")) {
         if (value < 1 || value > (int64_t)sk::kWinMaxWorkers) return fail(SK_EINVAL, "window_workers must be in 1..4");
         s->window_workers = value;
@@ -360,6 +362,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     if (!strcmp(key, "log2g")) *value = s->P.log2g;
     else if (!strcmp(key, "window_lines")) *value = s->window_lines;
     else if (!strcmp(key, "window_workers")) *value = s->window_workers;
+    else if (!strcmp(key, "window_red_rows")) *value = s->window_red_rows;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
     else if (!strcmp(key, "sketch_ctas_per_sm")) *value = s->sketch_ctas_per_sm;

@@ -57,12 +57,11 @@ int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint
                          cudaStream_t st);
 // windowed hash family: shared-memory accumulation, at most kWinMaxWorkers workers per launch; -1 if it cannot run
 constexpr uint32_t kWinMaxWorkers = 4;
-int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, int sm_count,
-                             cudaStream_t st);
-int launch_second_moment(const Params& P, const MomentArgs& A, const uint32_t* I_prev, uint32_t k_prev,
-                         cudaStream_t st);
+int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, uint32_t r_red,
+                             int sm_count, cudaStream_t st);
 int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStream_t st);
-int launch_unsketch_hist(const Params& P, const float* sum, const float* vhat, uint32_t* keys, uint32_t* hist,
+// A.members != 0: also apply the second-moment update on I_{t-1} (bitmap, gsum, v, vstamp, vhat of A)
+int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum, uint32_t* keys, uint32_t* hist,
                          bool vec, int sm_count, cudaStream_t st);
 int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cudaStream_t st);
 int launch_emit(const Params& P, const uint32_t* keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2,

@@ -10,6 +10,7 @@
 // key = bit pattern of |estimate| (monotone for finite non-negative floats); ties go to the smaller index.
 #include "sk_internal.h"
 #include "sk_hash.cuh"
+#include "sk_moment.cuh"
 
 namespace sk {
 
@@ -104,9 +105,19 @@ __device__ __forceinline__ float median1(const Params& P, const float* __restric
 }
 
 // ---- pass A: ranking keys of all coordinates (stored) + histogram of key bits 30..19 -----------------------------
+// The pass streams vhat anyway, so it also carries the master's update of v and vhat on I_{t-1} (Algorithm 2):
+// where the membership bitmap is set, v and vhat are brought up to date from the gradient sums the moment kernel
+// left in gsum, before vhat is used.  A.members = 0 turns that off (a re-run of the selection must not repeat it).
+__device__ __forceinline__ void update_member(const Params& P, const MomentArgs& A, float gsum, float& v, uint32_t& stamp,
+                                              float& vh) {
+    v = second_moment_value(P, v, stamp, A.step, gsum);
+    stamp = A.step;
+    vh = fmaxf(vh, v);
+}
+
 template <int R, bool VEC>
 __global__ void __launch_bounds__(kThreads)
-k_unsketch_hist(const __grid_constant__ Params P, const float* __restrict__ sum, const float* __restrict__ vhat,
+k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, const float* __restrict__ sum,
                 uint32_t* keys, uint32_t* hist) {
     __shared__ uint32_t sh[kHistBins];
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh[b] = 0;
@@ -120,7 +131,20 @@ k_unsketch_hist(const __grid_constant__ Params P, const float* __restrict__ sum,
         if (VEC) {
             const float4 med = medians4<R>(P, sum, tc);
             if (live) {
-                const float4 vh = __ldcs((const float4*)vhat + t);
+                float4 vh = ((const float4*)A.vhat)[t];
+                const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
+                if (mask) {
+                    const float4 gs = ((const float4*)A.gsum)[t];
+                    float4 vv = ((const float4*)A.v)[t];
+                    uint4 vs = ((const uint4*)A.vstamp)[t];
+                    if (mask & 1u) update_member(P, A, gs.x, vv.x, vs.x, vh.x);
+                    if (mask & 2u) update_member(P, A, gs.y, vv.y, vs.y, vh.y);
+                    if (mask & 4u) update_member(P, A, gs.z, vv.z, vs.z, vh.z);
+                    if (mask & 8u) update_member(P, A, gs.w, vv.w, vs.w, vh.w);
+                    ((float4*)A.v)[t] = vv;
+                    ((uint4*)A.vstamp)[t] = vs;
+                    ((float4*)A.vhat)[t] = vh;
+                }
                 uint4 k4;
                 k4.x = key_rank(med.x, vh.x); k4.y = key_rank(med.y, vh.y);
                 k4.z = key_rank(med.z, vh.z); k4.w = key_rank(med.w, vh.w);
@@ -129,7 +153,14 @@ k_unsketch_hist(const __grid_constant__ Params P, const float* __restrict__ sum,
                 atomicAdd(&sh[k4.z >> kHistShift], 1u); atomicAdd(&sh[k4.w >> kHistShift], 1u);
             }
         } else if (live) {
-            const uint32_t key = key_rank(median1(P, sum, t), vhat[t]);
+            float vh = A.vhat[t];
+            if (A.members && ((A.bitmap[t >> 5] >> (t & 31u)) & 1u)) {
+                float vv = A.v[t];
+                uint32_t vs = A.vstamp[t];
+                update_member(P, A, A.gsum[t], vv, vs, vh);
+                A.v[t] = vv; A.vstamp[t] = vs; A.vhat[t] = vh;
+            }
+            const uint32_t key = key_rank(median1(P, sum, t), vh);
             keys[t] = key;
             atomicAdd(&sh[key >> kHistShift], 1u);
         }
@@ -427,14 +458,14 @@ inline int grid_for(uint64_t items, int sm_count, int per_sm) {
         default: KERNEL<0, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                           \
     }
 
-int launch_unsketch_hist(const Params& P, const float* sum, const float* vhat, uint32_t* keys, uint32_t* hist,
+int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum, uint32_t* keys, uint32_t* hist,
                          bool vec, int sm_count, cudaStream_t st) {
     if (!vec) {
-        k_unsketch_hist<0, false><<<grid_for(P.d, sm_count, 6), kThreads, 0, st>>>(P, sum, vhat, keys, hist);
+        k_unsketch_hist<0, false><<<grid_for(P.d, sm_count, 6), kThreads, 0, st>>>(P, A, sum, keys, hist);
         return 1;
     }
     const int grid = grid_for(P.d >> 2, sm_count, 6);
-    SK_ROWS_SWITCH(k_unsketch_hist, P, sum, vhat, keys, hist)
+    SK_ROWS_SWITCH(k_unsketch_hist, P, A, sum, keys, hist)
     return 1;
 }
 

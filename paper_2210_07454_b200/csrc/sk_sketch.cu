@@ -1,8 +1,9 @@
 // Dense half of the step: momentum + error-feedback accumulate + Count Sketch of every worker's vector
-// (Algorithm 2, worker side; Section II-C) fused with the master's second-moment update on I_{t-1}, and the
-// fixed-order sum of the n sketches.
+// (Algorithm 2, worker side; Section II-C), the gradient sums on I_{t-1} that the master's second-moment update
+// needs (the update itself rides on the key pass in sk_select.cu), and the fixed-order sum of the n sketches.
 #include "sk_internal.h"
 #include "sk_hash.cuh"
+#include "sk_moment.cuh"
 
 namespace sk {
 
@@ -30,26 +31,6 @@ __global__ void __launch_bounds__(kThreads) k_fill_u32(uint32_t* p, uint64_t n, 
 __global__ void __launch_bounds__(kThreads) k_set_bits(const uint32_t* __restrict__ I, uint32_t count, uint32_t* bitmap) {
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
     if (q < count) atomicOr(&bitmap[I[q] >> 5], 1u << (I[q] & 31u));
-}
-
-// v is kept lazily: vstamp[j] is the step at which v[j] was last brought up to date.  A coordinate outside
-// I_{t-1} only decays, v <- beta2 v (Algorithm 2's v update with h_t = 0 there), and vhat = max(vhat, v) cannot
-// change, so the decays are applied one fp32 multiply per owed step when the coordinate is next touched --
-// the same chain of roundings as applying them every step.
-__device__ __forceinline__ float decay_owed(float v, float beta2, uint32_t owed) {
-    for (uint32_t s = 0; s < owed && v != 0.0f; ++s) v = __fmul_rn(beta2, v);
-    return v;
-}
-
-// Master side of Algorithm 2 for one coordinate of I_{t-1}, given the sum of the workers' gradients there:
-// h = sum / n ; v = beta2 v + (1-beta2) h^2 ; vhat = max(vhat, v).
-__device__ __forceinline__ void second_moment(const Params& P, const MomentArgs& A, uint32_t j, float gsum) {
-    const float h = gsum / (float)P.n;
-    float vj = decay_owed(A.v[j], P.beta2, A.step - 1u - A.vstamp[j]);
-    vj = fmaf(P.beta2, vj, (1.0f - P.beta2) * h * h);
-    A.v[j] = vj;
-    A.vstamp[j] = A.step;
-    if (vj > A.vhat[j]) A.vhat[j] = vj;
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -135,7 +116,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
                 if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
         }
-        if (mask) ((float4*)A.gsum)[t] = gs;             // consumed by k_second_moment (or by the next launch)
+        if (mask) ((float4*)A.gsum)[t] = gs;             // consumed by the key pass (or by the next launch)
     }
 }
 
@@ -163,17 +144,6 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
         }
         if (member) A.gsum[j] = gs;
     }
-}
-
-// For j in I_{t-1}: h = (sum_w g^(w)_j) / n ; v_j = beta2 v_j + (1-beta2) h^2 ; vhat_j = max(vhat_j, v_j).
-// The gradient sums were left in gsum by the moment kernel, which streams every gradient anyway.
-__global__ void __launch_bounds__(kThreads)
-k_second_moment(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A,
-                const uint32_t* __restrict__ I_prev, uint32_t k_prev) {
-    const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
-    if (q >= k_prev) return;
-    const uint32_t j = I_prev[q];
-    second_moment(P, A, j, A.gsum[j]);
 }
 
 // S = (S^(0) + S^(1) + ... + S^(n-1)) / n, workers added in index order (Algorithm 2, master side).
@@ -242,13 +212,6 @@ int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint
         default: k_moment_sketch_v4<0><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
     }
 #undef SK_CASE
-    return 1;
-}
-
-int launch_second_moment(const Params& P, const MomentArgs& A, const uint32_t* I_prev, uint32_t k_prev,
-                         cudaStream_t st) {
-    if (k_prev == 0) return 0;
-    k_second_moment<<<(k_prev + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, A, I_prev, k_prev);
     return 1;
 }
 

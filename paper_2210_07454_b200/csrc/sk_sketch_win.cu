@@ -25,6 +25,7 @@ constexpr int kProducerThreads = 256;
 constexpr uint32_t kUnit = 1u << kUnitShift;      // 1024 coordinates
 constexpr uint32_t kGroupsPerUnit = kUnit / 32;   // 32
 constexpr int kMaxConsumerWarps = 16;
+constexpr uint32_t kMaxRedRows = 4;               // at most this many rows go through L2 reductions in this kernel
 
 __device__ __forceinline__ void red_add_v4(float* addr, float4 v) {
     asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
@@ -57,10 +58,14 @@ __device__ __forceinline__ void item_range(const Params& P, uint32_t item, uint3
 
 __global__ void __launch_bounds__(kProducerThreads + 32 * kMaxConsumerWarps)
 k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw,
-                    uint32_t slices, uint32_t units_total) {
+                    uint32_t slices, uint32_t units_total, uint32_t r_red) {
+    // rows [0, r_red) are sketched by the producers with reductions into the L2-resident tables; rows [r_red, r)
+    // by the consumers in shared-memory windows: the two mechanisms load different parts of the SM (the request
+    // port towards L2, and instruction issue + shared memory), so splitting the rows lets both stay below the
+    // time of the memory stream.
     extern __shared__ __align__(16) float smem[];
     const uint32_t r = P.r, cw = P.win_cw;
-    const uint32_t pairs = nw * r;
+    const uint32_t pairs = nw * (r - r_red);
     float* win = smem;                                         // [pairs][cw]
     float* stage = win + (size_t)pairs * cw;                   // [2][nw][1024]
     uint2* hsh = (uint2*)(stage + (size_t)2 * nw * kUnit);     // [2][r][32]: x = line*32 | perm, y = sign bits
@@ -75,6 +80,7 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
         float4* e = (float4*)A.e;
         const uint32_t d4 = P.d >> 2;
         const float b1 = P.beta1, omb1 = 1.0f - P.beta1;
+        const uint64_t tstride = (uint64_t)P.r * P.cs;
         uint32_t seq = 0;                                      // units produced by this block so far
         for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
             uint32_t panel, t_begin, t_end;
@@ -85,12 +91,14 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                 if (seq >= 2) bar_sync(3 + b, nthreads);       // wait until the consumers are done with buffer b
                 float* st = stage + (size_t)b * nw * kUnit;
                 uint2* hs = hsh + (size_t)b * r * kGroupsPerUnit;
-                for (uint32_t hq = tid; hq < r * kGroupsPerUnit; hq += kProducerThreads) {
+                for (uint32_t hq = r_red * kGroupsPerUnit + tid; hq < r * kGroupsPerUnit; hq += kProducerThreads) {
                     const uint32_t row = hq >> 5, s = hq & 31u;
                     const GroupHash gh = group_from_draw(P, stream(P.row_key[row], (uint64_t)unit * kGroupsPerUnit + s + 1));
                     hs[hq] = make_uint2(gh.base | gh.perm, gh.signs);
                 }
                 const uint32_t t = unit * (kUnit / 4) + tid;
+                Quad hr[kMaxRedRows];                          // this quad's hashes in the rows sketched by reductions
+                quad_hashes<kMaxRedRows>(P, r_red, t < d4 ? t : d4 - 1, hr);
                 if (t < d4) {
                     const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
                     float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -109,6 +117,13 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                         __stcs(e + q0, a0); __stcs(e + q1, a1);
                         ((float4*)(st + (size_t)w * kUnit))[tid] = a0;
                         ((float4*)(st + (size_t)(w + 1) * kUnit))[tid] = a1;
+                        float* t0 = A.tables + (uint64_t)(w0 + w) * tstride;
+#pragma unroll
+                        for (uint32_t row = 0; row < kMaxRedRows; ++row)
+                            if (row < r_red) {
+                                red_add_v4(t0 + (uint64_t)row * P.cs + hr[row].off, quad_scatter(hr[row], a0));
+                                red_add_v4(t0 + tstride + (uint64_t)row * P.cs + hr[row].off, quad_scatter(hr[row], a1));
+                            }
                     }
                     if (w < nw) {
                         const uint64_t q0 = (uint64_t)(w0 + w) * d4 + t;
@@ -120,6 +135,10 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                         __stcs(m + q0, m0);
                         __stcs(e + q0, a0);
                         ((float4*)(st + (size_t)w * kUnit))[tid] = a0;
+                        float* t0 = A.tables + (uint64_t)(w0 + w) * tstride;
+#pragma unroll
+                        for (uint32_t row = 0; row < kMaxRedRows; ++row)
+                            if (row < r_red) red_add_v4(t0 + (uint64_t)row * P.cs + hr[row].off, quad_scatter(hr[row], a0));
                     }
                     if (mask) ((float4*)A.gsum)[t] = gs;
                 } else {
@@ -161,7 +180,7 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                 const float* st = stage + (size_t)b * nw * kUnit;
                 const uint2* hs = hsh + (size_t)b * r * kGroupsPerUnit;
                 for (uint32_t pr = sub; pr < pairs; pr += nsub) {
-                    const uint32_t w = pr % nw, row = pr / nw;
+                    const uint32_t w = pr % nw, row = r_red + pr / nw;
                     float* wn = win + (size_t)pr * cw;
                     const float4* sw = (const float4*)(st + (size_t)w * kUnit) + l8;
                     const uint2* hr = hs + row * kGroupsPerUnit;
@@ -192,7 +211,7 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
             __syncwarp();
             // flush this sub-warp's windows: table[w][row][panel*cw + ...] += window
             for (uint32_t pr = sub; pr < pairs; pr += nsub) {
-                const uint32_t w = pr % nw, row = pr / nw;
+                const uint32_t w = pr % nw, row = r_red + pr / nw;
                 float* dstrow = A.tables + (uint64_t)(w0 + w) * tstride + (uint64_t)row * P.cs + (uint64_t)panel * cw;
                 for (uint32_t q = l8; q < cw / 4; q += 8) red_add_v4(dstrow + 4u * q, ((const float4*)(win + (size_t)pr * cw))[q]);
             }
@@ -208,16 +227,18 @@ inline uint32_t consumer_warps(uint32_t pairs) {
 
 }  // namespace
 
-size_t window_smem_bytes(const Params& P, uint32_t nw) {
-    return ((size_t)nw * P.r * P.win_cw + (size_t)2 * nw * kUnit) * 4 + (size_t)2 * P.r * kGroupsPerUnit * 8;
+size_t window_smem_bytes(const Params& P, uint32_t nw, uint32_t r_red) {
+    return ((size_t)nw * (P.r - r_red) * P.win_cw + (size_t)2 * nw * kUnit) * 4 + (size_t)2 * P.r * kGroupsPerUnit * 8;
 }
 
 // Enqueues the windowed kernel for workers w0..w0+nw-1 (nw <= kWinMaxWorkers).  Returns launches, or -1 if the
 // configuration does not fit in shared memory.
-int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, int sm_count,
-                             cudaStream_t st) {
-    const size_t smem = window_smem_bytes(P, nw);
-    const int threads = kProducerThreads + 32 * (int)consumer_warps(nw * P.r);
+int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, uint32_t r_red,
+                             int sm_count, cudaStream_t st) {
+    if (r_red > kMaxRedRows) r_red = kMaxRedRows;
+    if (r_red > P.r) r_red = P.r;
+    const size_t smem = window_smem_bytes(P, nw, r_red);
+    const int threads = kProducerThreads + 32 * (int)consumer_warps(nw * (P.r - r_red));
     static size_t configured = 0;
     if (smem > configured) {
         if (cudaFuncSetAttribute(k_moment_sketch_win, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -235,7 +256,7 @@ int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, 
     const uint64_t items = (uint64_t)P.win_panels * slices;
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const int grid = (int)(items < cap ? items : cap);
-    k_moment_sketch_win<<<grid, threads, smem, st>>>(P, A, w0, nw, slices, units_total);
+    k_moment_sketch_win<<<grid, threads, smem, st>>>(P, A, w0, nw, slices, units_total, r_red);
     return 1;
 }
 

@@ -17,6 +17,7 @@ struct sk_state {
     int64_t worker_chunk = 0;
     int64_t window_lines = 0;
     int64_t window_workers = 4;
+    int64_t window_red_rows = 0;
     int64_t sketch_ctas_per_sm = 64;
     bool timing = false;
     cudaStream_t stream = nullptr;

@@ -81,7 +81,9 @@ extern "C" int sk_select_static(sk_state* s, uint32_t* idx_out) {
 
     // the array is shared by all calls and keeps the last call's contents: clear what must start at zero
     sk::launch_zero(base + kOffHist, kOffKeys - kOffHist, st);
-    sk::launch_unsketch_hist(P, s->sum, s->vhat, keys, hist, vec, s->sm_count, st);
+    sk::MomentArgs A{};                 // members = 0: read vhat only, the step's own update is not repeated
+    A.vhat = s->vhat;
+    sk::launch_unsketch_hist(P, A, s->sum, keys, hist, vec, s->sm_count, st);
     sk::launch_pick_bin(P, hist, sel, 0, st);
     sk::launch_emit(P, keys, sel, idx_out, cand, hist2, s->sm_count, st);
     sk::launch_refine(P, sel, cand, cand2, hist2, idx_out, s->sm_count, st);

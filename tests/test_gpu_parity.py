@@ -141,6 +141,28 @@ def test_windowed_edge_cases(case):
     _run_steps(w, 3, cfg_id=8, window_lines=L)
 
 
+@pytest.mark.parametrize("red_rows", [0, 1, 3, 4])
+def test_windowed_rows_split_between_reductions_and_windows(red_rows):
+    # the windowed kernel sketches the first rows by L2 reductions and the rest in shared-memory windows;
+    # every split must give the same tables
+    w = _workload("C1", name="E", d=1024 * 21 + 64, n=5, r=5, c=4096, k=300, steps=2, recipe="planted")
+    gpu, ora = _pair(w, window_lines=8)
+    gpu.set_option("window_red_rows", red_rows)
+    src = _source(w, cfg_id=8)
+    x = src.x0()
+    x_ref = x.cpu().numpy().copy()
+    for t in (1, 2):
+        g = src.grads(t)
+        if t > 1:
+            force_state(gpu, ora)
+            x.copy_(torch.from_numpy(x_ref))
+        xb = x_ref.astype(np.float64).copy()
+        gpu.step(g, x)
+        gpu.sync()
+        ora.step(g.cpu().numpy(), x_ref)
+        compare_step(gpu, ora, x.cpu().numpy(), x_ref, xb, w.lr)
+
+
 def test_windowed_integer_inputs_are_bit_exact():
     d, n, r, c, k = 200_000, 4, 5, 4096, 1000
     b = _binding()
