@@ -120,7 +120,7 @@ class Oracle:
     """One SketchedAMSGrad (gradient averaging) optimiser; `step` advances it by one iteration."""
 
     def __init__(self, d, n, r, c, k, seed=0, log2g=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8,
-                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0):
+                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0, variant="ga"):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
         self._h = lib().ora_create(d, n, r, c, k, seed, log2g, lr, beta1, beta2, eps)
         if not self._h:
@@ -135,6 +135,9 @@ class Oracle:
             if log2g != 5 or 32 * window_lines > c:
                 raise ValueError("the windowed family needs g = 32 and 32 * window_lines <= c")
             lib().ora_set_option(self._h, b"window_lines", int(window_lines))
+        if variant not in ("ga", "pa"):
+            raise ValueError("variant must be 'ga' (Algorithm 2) or 'pa' (Algorithm 1)")
+        lib().ora_set_option(self._h, b"variant_pa", int(variant == "pa"))
         lib().ora_set_option(self._h, b"v_keep", int(v_keep))
         lib().ora_set_option(self._h, b"threads", int(threads))
 
@@ -154,7 +157,8 @@ class Oracle:
         if rc != 0:
             raise RuntimeError(f"ora_step failed: {rc}")
 
-    _SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "tables": "nrc", "sum": "rc"}
+    _SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "tables": "nrc", "sum": "rc",
+               "vw": "nd", "vhatw": "nd"}
 
     def field(self, name: str) -> np.ndarray:
         """A numpy VIEW of the oracle's own buffer (writable: teacher forcing writes through it)."""

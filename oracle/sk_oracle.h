@@ -21,6 +21,9 @@
  *     values"); e_t^(i) is a_t^(i) with the coordinates of I_t set to zero (Lemma 3's proof).
  *   - Even r: lower median.  Ties in top-k: the smaller index wins.
  *
+ * ora_step also implements Algorithm 1 (parameter averaging) when the option "variant_pa" is set: per-worker
+ * v and vhat from the worker's own gradient, the sketched vector is m/sqrt(vhat) + e, and the unsketch takes no vhat.
+ *
  * Parity pins: see tests/test_oracle_*.py.  Nothing here is "parity unpinned" except the five large
  * benchmark workloads themselves, for which the paper prints no expected values.
  */
@@ -64,7 +67,9 @@ ora_state* ora_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k
 void ora_destroy(ora_state* s);
 /* inject explicit hash arrays (r*d each) instead of the seeded family; pointers must outlive the state */
 void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn);
-void ora_set_option(ora_state* s, const char* key, int value);   /* "v_keep", "threads" */
+/* "v_keep", "threads", "window_lines" (windowed hash family), "variant_pa" (1 = Algorithm 1, parameter averaging;
+   per-worker v and vhat are then the fields "vw" and "vhatw", n*d each) */
+void ora_set_option(ora_state* s, const char* key, int value);
 int  ora_step(ora_state* s, const float* grads /* n*d worker-major */, float* x /* d, in place */);
 
 /* field access: "m","e" (n*d) "v","vhat","est" (d) "tables" (n*r*c) "sum" (r*c) -> float*;

@@ -14,7 +14,8 @@ struct ora_state {
     uint64_t d, k, seed, t, k_prev;
     uint32_t n, r, c, log2g, window_lines;
     float lr, beta1, beta2, eps;
-    int v_keep, threads;
+    int v_keep, threads, variant_pa;
+    float *vw, *vhatw;       /* parameter-averaging variant: per-worker v and vhat (n*d each) */
     float *m, *e, *v, *vhat, *est, *tables, *sum;
     uint32_t *I, *I_prev;
     uint8_t* mask;
@@ -51,7 +52,7 @@ ora_state* ora_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k
 void ora_destroy(ora_state* s) {
     if (!s) return;
     free(s->m); free(s->e); free(s->v); free(s->vhat); free(s->est); free(s->tables); free(s->sum);
-    free(s->I); free(s->I_prev); free(s->mask); free(s->row_key); free(s);
+    free(s->I); free(s->I_prev); free(s->mask); free(s->row_key); free(s->vw); free(s->vhatw); free(s);
 }
 
 void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn) { s->h_idx = idx; s->h_sgn = sgn; }
@@ -64,6 +65,16 @@ void ora_set_option(ora_state* s, const char* key, int value) {
             s->window_lines = (uint32_t)value;
     }
     else if (!strcmp(key, "threads")) s->threads = value > 0 ? value : 1;
+    else if (!strcmp(key, "variant_pa")) {
+        /* Algorithm 1 (parameter averaging); only before the first step.  v_0^(i) = vhat_0^(i) = eps. */
+        if (value && !s->vw && s->t == 0) {
+            size_t nd = (size_t)s->n * s->d;
+            s->vw = (float*)malloc(nd * sizeof(float));
+            s->vhatw = (float*)malloc(nd * sizeof(float));
+            for (size_t q = 0; q < nd; ++q) s->vw[q] = s->vhatw[q] = s->eps;
+        }
+        if (s->t == 0) s->variant_pa = value ? 1 : 0;
+    }
 }
 
 void* ora_field(ora_state* s, const char* name) {
@@ -76,6 +87,8 @@ void* ora_field(ora_state* s, const char* name) {
     if (!strcmp(name, "sum")) return s->sum;
     if (!strcmp(name, "I")) return s->I;
     if (!strcmp(name, "I_prev")) return s->I_prev;
+    if (!strcmp(name, "vw")) return s->vw;
+    if (!strcmp(name, "vhatw")) return s->vhatw;
     return NULL;
 }
 
@@ -104,7 +117,10 @@ static inline void hash_at(const ora_state* s, uint32_t j, uint64_t i, uint32_t*
     *sg = (((u & 0xFFFFFFFFULL) >> o) & 1ULL) ? -1 : 1;
 }
 
+static int ora_step_pa(ora_state* s, const float* grads, float* x);
+
 int ora_step(ora_state* s, const float* grads, float* x) {
+    if (s->variant_pa) return ora_step_pa(s, grads, x);
     const uint64_t d = s->d, k = s->k;
     const uint32_t n = s->n, r = s->r, c = s->c;
     const double b1 = (double)s->beta1, b2 = (double)s->beta2, lr = (double)s->lr;
@@ -193,6 +209,80 @@ int ora_step(ora_state* s, const float* grads, float* x) {
         for (uint32_t w = 0; w < n; ++w) s->e[(uint64_t)w * d + j] = 0.0f;
     }
 
+    memcpy(s->I_prev, s->I, (size_t)k * sizeof(uint32_t));
+    s->k_prev = k;
+    s->t += 1;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * SketchedAMSGrad with PARAMETER averaging (Algorithm 1).  Every worker runs its own AMSGrad moments:
+ *   m = beta1 m + (1-beta1) g ;  v = beta2 v + (1-beta2) g^2 ;  vhat = max(vhat, v)        (per worker)
+ *   a = m / sqrt(vhat) + rho e            the vector the worker sketches (kept in the e buffer)
+ *   S = (1/n) sum_w S(a^(w)) ;  Delta = Top-k(U(S)) with the plain unsketch (no vhat argument)
+ *   Delta takes the exact worker means of a on I_t (Section III-A) ;  x -= alpha Delta
+ *   e = a with the coordinates of I_t removed
+ * est, sum, tables, I are stored in the same fields as for Algorithm 2.
+ * ------------------------------------------------------------------------------------------------ */
+static int ora_step_pa(ora_state* s, const float* grads, float* x) {
+    const uint64_t d = s->d, k = s->k;
+    const uint32_t n = s->n, r = s->r, c = s->c;
+    const double b1 = (double)s->beta1, b2 = (double)s->beta2, lr = (double)s->lr;
+    const double rho = 1.0;
+#ifdef _OPENMP
+    omp_set_num_threads(s->threads);
+#endif
+#pragma omp parallel for schedule(static)
+    for (uint64_t q = 0; q < (uint64_t)n * d; ++q) {
+        const double g = (double)grads[q];
+        s->m[q] = (float)(b1 * (double)s->m[q] + (1.0 - b1) * g);
+        s->vw[q] = (float)(b2 * (double)s->vw[q] + (1.0 - b2) * g * g);
+        if (s->vw[q] > s->vhatw[q]) s->vhatw[q] = s->vw[q];
+        s->e[q] = (float)((double)s->m[q] / sqrt((double)s->vhatw[q]) + rho * (double)s->e[q]);
+    }
+#pragma omp parallel
+    {
+        double* acc = (double*)malloc((size_t)c * sizeof(double));
+#pragma omp for schedule(dynamic, 1)
+        for (uint64_t wj = 0; wj < (uint64_t)n * r; ++wj) {
+            uint32_t w = (uint32_t)(wj / r), j = (uint32_t)(wj % r);
+            const float* a = s->e + (uint64_t)w * d;
+            memset(acc, 0, (size_t)c * sizeof(double));
+            for (uint64_t i = 0; i < d; ++i) {
+                uint32_t b; int8_t sg;
+                hash_at(s, j, i, &b, &sg);
+                acc[b] += (double)sg * (double)a[i];
+            }
+            float* row = s->tables + ((uint64_t)w * r + j) * c;
+            for (uint32_t b = 0; b < c; ++b) row[b] = (float)acc[b];
+        }
+        free(acc);
+    }
+#pragma omp parallel for schedule(static)
+    for (uint64_t q = 0; q < (uint64_t)r * c; ++q) {
+        double acc = 0.0;
+        for (uint32_t w = 0; w < n; ++w) acc += (double)s->tables[(uint64_t)w * r * c + q];
+        s->sum[q] = (float)(acc / (double)n);
+    }
+#pragma omp parallel for schedule(static)
+    for (uint64_t i = 0; i < d; ++i) {
+        float q[64];
+        for (uint32_t j = 0; j < r; ++j) {
+            uint32_t b; int8_t sg;
+            hash_at(s, j, i, &b, &sg);
+            q[j] = (float)sg * s->sum[(uint64_t)j * c + b];
+        }
+        s->est[i] = ora_median(q, r);
+    }
+    ora_topk(s->est, d, k, s->I);
+    for (uint64_t t = 0; t < k; ++t) {
+        uint64_t j = s->I[t];
+        double abar = 0.0;
+        for (uint32_t w = 0; w < n; ++w) abar += (double)s->e[(uint64_t)w * d + j];
+        abar /= (double)n;
+        x[j] = (float)((double)x[j] - lr * abar);
+        for (uint32_t w = 0; w < n; ++w) s->e[(uint64_t)w * d + j] = 0.0f;
+    }
     memcpy(s->I_prev, s->I, (size_t)k * sizeof(uint32_t));
     s->k_prev = k;
     s->t += 1;
