@@ -170,6 +170,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--log2g", type=int, default=None)
+    ap.add_argument("--variant", default="ga", choices=["ga", "pa"],
+                    help="ga = gradient averaging (Algorithm 2, the headline path); pa = parameter averaging (Algorithm 1)")
     ap.add_argument("--window-lines", type=int, default=None, help="windowed hash family: lines per window (0 = plain)")
     ap.add_argument("--window-workers", type=int, default=0, help="workers per launch of the windowed sketch kernel")
     ap.add_argument("--window-red-rows", type=int, default=-1, help="rows the windowed kernel sketches by L2 reductions")
@@ -204,7 +206,7 @@ def main():
 
     src = synthetic.GradientSource(w, device=dev, cfg_id=cfg_id)
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                                  eps=w.eps, log2g=args.log2g, window_lines=args.window_lines)
+                                  eps=w.eps, log2g=args.log2g, window_lines=args.window_lines, variant=args.variant)
     opt.set_option("worker_chunk", args.worker_chunk)
     if args.window_workers:
         opt.set_option("window_workers", args.window_workers)
@@ -255,7 +257,7 @@ def main():
     # dominant kernel: moments + sketch.  Algorithmic bytes per launch: 20 B per worker-coordinate streamed
     # (read g, m, e; write m, e) plus the worker tables it fills (4 B per bucket).
     k1_launches = max(1, stage_launches[2])
-    k1_bytes_step = 20 * w.n * w.d + 4 * w.n * w.r * w.c
+    k1_bytes_step = (20 if args.variant == "ga" else 36) * w.n * w.d + 4 * w.n * w.r * w.c
     roofline = None
     if not args.no_stage_timing and stage_ms[2] > 0:
         k1_ms = stage_ms[2] / k1_launches
@@ -263,9 +265,9 @@ def main():
         achieved = k1_bytes / (k1_ms * 1e-3) / 1e9
         sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2210_07454_b200", "csrc", "sk_sketch.cu"), "rb").read()).hexdigest()
         traffic = None
-        if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"]:
+        if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"] and args.variant == "ga":
             traffic = NCU_TRAFFIC["bytes_per_worker_coord"] * w.n * w.d * args.steps / k1_launches
-        roofline = {"bound": "hbm", "kernel": "k_moment_sketch_v4", "achieved": achieved, "peak": peak,
+        roofline = {"bound": "hbm", "kernel": "k_moment_sketch_v4" if args.variant == "ga" else "k_moment_sketch_pa_v4", "achieved": achieved, "peak": peak,
                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                     "ms_per_launch": k1_ms, "launches_per_step": k1_launches / args.steps,
                     "algorithmic_bytes_per_launch": k1_bytes}
@@ -303,7 +305,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k,
-                       "recipe": w.recipe, "hash_group": 1 << opt.get_option("log2g"),
+                       "recipe": w.recipe, "variant": args.variant, "hash_group": 1 << opt.get_option("log2g"),
                        "window_lines": opt.get_option("window_lines"),
                        "worker_chunk": opt.get_option("worker_chunk"), "replicas": world,
                        "l2": f"inputs larger than L2: {nsets} rotating gradient sets of {set_bytes / 1e9:.2f} GB"},

@@ -70,6 +70,10 @@ int sk_sync(sk_state* state);
 /* Options (integers):
  *   "log2g"        hash group size g = 2^log2g, 0..5 (Section II-C fixes no hash family; see sk_hash).
  *                  Only before the first step.  Default: the largest value <= 5 with 2^log2g <= c.
+ *   "variant"      0 (default) = gradient averaging, Algorithm 2; 1 = parameter averaging, Algorithm 1: every worker
+ *                  keeps its own v and vhat (fields "vw", "vhatw", n*d each, initial value eps) from its own
+ *                  gradient, sketches m/sqrt(vhat) + e, the unsketch takes no vhat and x moves by the plain mean
+ *                  of the exact values on I_t.  Only before the first step; allocates 8*n*d bytes.
  *   "window_lines" L > 0 selects the windowed variant of the hash family (needs g = 32, 32*L <= c): units of
  *                  1024 coordinates map into one aligned window of 32*L buckets per row, which lets the sketch
  *                  kernel accumulate in shared memory.  0 (default) = plain family.  Only before the first step.
@@ -100,6 +104,7 @@ int sk_hash(const sk_state* state, uint32_t row, uint64_t i0, uint64_t count,
  *   "tables"  n*r*c  the worker sketches S_t^(w) of the last step;  "sum"  r*c  the aggregate S_t
  *   "est"     d    the estimates of the last step (recomputed on request from "sum" and "vhat"; get only)
  *   "I"       k uint32  I_t of the last step, ascending (get);  set: installs I_{t-1} for the next step
+ *   "vw","vhatw" n*d  per-worker second moments (parameter-averaging variant only; "v","vhat" are then unavailable)
  *   "t"       1 uint64  number of steps taken
  * Both calls synchronise the stream. */
 int sk_get(sk_state* state, const char* field, void* buf, uint64_t bytes);

@@ -79,10 +79,11 @@ def _nbytes(t) -> int:
 class SketchedAMSGrad:
     """Handle over ``sk_create`` / ``sk_step`` / ``sk_destroy`` and the auxiliary calls."""
 
-    _FIELD_SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "tables": "nrc", "sum": "rc"}
+    _FIELD_SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "tables": "nrc", "sum": "rc",
+                     "vw": "nd", "vhatw": "nd"}
 
     def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None,
-                 window_lines=None):
+                 window_lines=None, variant="ga"):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
         self._h = lib().sk_create(d, n, r, c, k, seed, lr, beta1, beta2, eps)
         if not self._h:
@@ -91,6 +92,10 @@ class SketchedAMSGrad:
             self.set_option("log2g", log2g)
         if window_lines is not None:
             self.set_option("window_lines", window_lines)
+        if variant not in ("ga", "pa"):
+            raise SkError("variant must be 'ga' (Algorithm 2, gradient averaging) or 'pa' (Algorithm 1)")
+        if variant == "pa":
+            self.set_option("variant", 1)
 
     def close(self):
         if getattr(self, "_h", None):

@@ -122,7 +122,8 @@ int do_step(sk_state* s, const float* grads, float* x) {
     A.grads = grads; A.m = s->m; A.e = s->e; A.tables = s->tables; A.gsum = s->gsum;
     A.v = s->v; A.vhat = s->vhat; A.vstamp = s->vstamp; A.bitmap = s->bitmap;
     A.step = t; A.members = s->k_prev ? 1u : 0u;
-    const bool windowed = vec && P.win_cw != 0;
+    A.vw = s->vw; A.vhatw = s->vhatw; A.variant = (uint32_t)s->variant;
+    const bool windowed = vec && P.win_cw != 0 && s->variant == 0;   // the windowed kernel implements Algorithm 2 only
     const uint32_t wc = windowed ? std::min<uint32_t>((uint32_t)s->window_workers, P.n) : chunk_of(s);
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
@@ -163,7 +164,7 @@ int do_step(sk_state* s, const float* grads, float* x) {
     {
         StageTimer tm(s, 7);     // the bitmap of I_{t-1} has served its purpose: clear it, then apply marks I_t
         int l = sk::launch_zero(s->bitmap, s->bitmap_bytes, st);
-        l += sk::launch_apply(P, s->I, s->vhat, s->e, x, s->bitmap, st);
+        l += sk::launch_apply(P, s->I, s->variant == 1 ? nullptr : s->vhat, s->e, x, s->bitmap, st);
         tm.done(l);
     }
     SK_CUDA(cudaGetLastError());
@@ -174,11 +175,11 @@ int do_step(sk_state* s, const float* grads, float* x) {
     return SK_OK;
 }
 
-enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_BAD };
+enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_VW, F_VHATW, F_BAD };
 
 Field field_of(const char* name) {
-    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t"};
-    for (int q = 0; q < 9; ++q) if (!strcmp(name, names[q])) return (Field)q;
+    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t", "vw", "vhatw"};
+    for (int q = 0; q < 11; ++q) if (!strcmp(name, names[q])) return (Field)q;
     return F_BAD;
 }
 
@@ -265,7 +266,7 @@ void sk_destroy(sk_state* s) {
     if (s->stream) cudaStreamSynchronize(s->stream); else cudaDeviceSynchronize();
     for (void* p : {(void*)s->m, (void*)s->e, (void*)s->v, (void*)s->vhat, (void*)s->vstamp, (void*)s->tables,
                     (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->hist2, (void*)s->sel, (void*)s->cand, (void*)s->cand2,
-                    (void*)s->keys, (void*)s->gsum, (void*)s->bitmap,
+                    (void*)s->keys, (void*)s->gsum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw,
                     (void*)s->stage_grads, (void*)s->stage_x})
         if (p) cudaFree(p);
     for (const TimeRec& r : s->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -328,6 +329,23 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         refresh_hash(s);
         return SK_OK;
     }
+    if (!strcmp(key, "variant")) {
+        if (s->t != 0) return fail(SK_ESTATE, "variant can only be changed before the first step");
+        if (value != 0 && value != 1) return fail(SK_EINVAL, "variant must be 0 (gradient averaging) or 1 (parameter averaging)");
+        if (value == 1 && !s->vw) {                   // v_0^(w) = vhat_0^(w) = eps on every worker (Algorithm 1)
+            const uint64_t nd = (uint64_t)s->P.n * s->P.d;
+            if (cudaMalloc((void**)&s->vw, nd * 4) != cudaSuccess || cudaMalloc((void**)&s->vhatw, nd * 4) != cudaSuccess)
+                return fail(SK_ENOMEM, "cudaMalloc of the per-worker second moments failed: %s",
+                            cudaGetErrorString(cudaGetLastError()));
+            uint32_t eps_bits;
+            memcpy(&eps_bits, &s->eps, 4);
+            sk::launch_fill_u32((uint32_t*)s->vw, nd, eps_bits, s->stream);
+            sk::launch_fill_u32((uint32_t*)s->vhatw, nd, eps_bits, s->stream);
+            SK_CUDA(cudaStreamSynchronize(s->stream));
+        }
+        s->variant = value;
+        return SK_OK;
+    }
     if (!strcmp(key, "window_red_rows")) {
         if (value < 0 || value > 4) return fail(SK_EINVAL, "window_red_rows must be in 0..4");
         s->window_red_rows = value;
@@ -362,6 +380,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     if (!strcmp(key, "log2g")) *value = s->P.log2g;
     else if (!strcmp(key, "window_lines")) *value = s->window_lines;
     else if (!strcmp(key, "window_workers")) *value = s->window_workers;
+    else if (!strcmp(key, "variant")) *value = s->variant;
     else if (!strcmp(key, "window_red_rows")) *value = s->window_red_rows;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
@@ -384,6 +403,8 @@ int sk_hash(const sk_state* s, uint32_t row, uint64_t i0, uint64_t count, uint32
 uint64_t sk_algorithmic_bytes(const sk_state* s) {
     if (!s) return 0;
     const uint64_t n = s->P.n, d = s->P.d, r = s->P.r, c = s->P.c, k = s->P.k;
+    if (s->variant == 1)     // Algorithm 1: read g,m,v,vhat,e and write m,v,vhat,e; no master-side second moments
+        return 36 * n * d + 8 * n * r * c + 4 * r * c + 8 * n * k + 8 * k;
     return 20 * n * d + 4 * d + 8 * n * r * c + 4 * r * c + 12 * n * k + 24 * k;
 }
 

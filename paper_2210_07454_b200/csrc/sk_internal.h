@@ -47,6 +47,9 @@ struct MomentArgs {
     const uint32_t* bitmap;  // membership of I_{t-1}: bit j of word j/32
     uint32_t step;           // t (1-based)
     uint32_t members;        // 0 when I_{t-1} is empty
+    // parameter-averaging variant (Algorithm 1): per-worker second moments, n*d each; variant = 1
+    float *vw, *vhatw;
+    uint32_t variant;        // 0 = gradient averaging (Algorithm 2), 1 = parameter averaging (Algorithm 1)
 };
 
 // Launchers.  Each enqueues on `st` and returns the number of kernels it launched.
@@ -68,6 +71,7 @@ int launch_emit(const Params& P, const uint32_t* keys, Select* sel, uint32_t* I_
                 int sm_count, cudaStream_t st);
 int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
                   int sm_count, cudaStream_t st);
+// vhat == nullptr: parameter averaging, the update is the plain mean (Algorithm 1)
 int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, float* x, uint32_t* bitmap,
                  cudaStream_t st);
 // helpers for state export / import

@@ -130,7 +130,13 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
         const uint32_t tc = live ? t : items - 1;
         if (VEC) {
             const float4 med = medians4<R>(P, sum, tc);
-            if (live) {
+            if (live && A.variant == 1) {                     // parameter averaging: U(S) takes no vhat (Algorithm 1)
+                uint4 k4;
+                k4.x = key_of(med.x); k4.y = key_of(med.y); k4.z = key_of(med.z); k4.w = key_of(med.w);
+                ((uint4*)keys)[t] = k4;
+                atomicAdd(&sh[k4.x >> kHistShift], 1u); atomicAdd(&sh[k4.y >> kHistShift], 1u);
+                atomicAdd(&sh[k4.z >> kHistShift], 1u); atomicAdd(&sh[k4.w >> kHistShift], 1u);
+            } else if (live) {
                 float4 vh = ((const float4*)A.vhat)[t];
                 const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
                 if (mask) {
@@ -152,6 +158,10 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
                 atomicAdd(&sh[k4.x >> kHistShift], 1u); atomicAdd(&sh[k4.y >> kHistShift], 1u);
                 atomicAdd(&sh[k4.z >> kHistShift], 1u); atomicAdd(&sh[k4.w >> kHistShift], 1u);
             }
+        } else if (live && A.variant == 1) {
+            const uint32_t key = key_of(median1(P, sum, t));
+            keys[t] = key;
+            atomicAdd(&sh[key >> kHistShift], 1u);
         } else if (live) {
             float vh = A.vhat[t];
             if (A.members && ((A.bitmap[t >> 5] >> (t & 31u)) & 1u)) {
@@ -413,7 +423,7 @@ k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const 
     }
     for (; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
     abar = abar / (float)P.n;
-    const float delta = scale_est(abar, vhat[j]);
+    const float delta = vhat ? scale_est(abar, vhat[j]) : abar;
     x[j] = x[j] - P.lr * delta;
     atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
 }
@@ -422,7 +432,7 @@ __global__ void __launch_bounds__(kThreads)
 k_estimates(const __grid_constant__ Params P, const float* __restrict__ sum, const float* __restrict__ vhat,
             float* est) {
     for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads)
-        est[j] = scale_est(median1(P, sum, j), vhat[j]);
+        est[j] = vhat ? scale_est(median1(P, sum, j), vhat[j]) : median1(P, sum, j);
 }
 
 __global__ void __launch_bounds__(kThreads)

@@ -120,6 +120,54 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
     }
 }
 
+// Parameter averaging (Algorithm 1): every worker keeps its own v and vhat from its own gradient,
+//   m = beta1 m + (1-beta1) g ; v = beta2 v + (1-beta2) g^2 ; vhat = max(vhat, v) ; a = m / sqrt(vhat) + e,
+// and a is what is sketched.  Reads g, m, v, vhat, e and writes m, v, vhat, a: 36 bytes per worker-coordinate.
+__device__ __forceinline__ void pa_moment(float b1, float omb1, float b2, float omb2, float g, float& m, float& v,
+                                          float& vh, float& a, bool masked) {
+    m = fmaf(b1, m, omb1 * g);
+    v = fmaf(b2, v, omb2 * g * g);
+    vh = fmaxf(vh, v);
+    a = __fdiv_rn(m, __fsqrt_rn(vh)) + (masked ? 0.0f : a);
+}
+
+template <int R>
+__global__ void __launch_bounds__(kThreads, 3)
+k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
+    const float4* __restrict__ grads = (const float4*)A.grads;
+    float4* m = (float4*)A.m;
+    float4* e = (float4*)A.e;
+    float4* vw = (float4*)A.vw;
+    float4* vhw = (float4*)A.vhatw;
+    const uint32_t r = R > 0 ? (uint32_t)R : P.r;
+    const uint32_t d4 = P.d >> 2;
+    const float b1 = P.beta1, omb1 = 1.0f - P.beta1, b2 = P.beta2, omb2 = 1.0f - P.beta2;
+    const uint64_t tstride = (uint64_t)P.r * P.cs;
+    constexpr int RMAX = R > 0 ? R : (int)kMaxRows;
+    const uint32_t trips = (d4 + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
+    for (uint32_t it = 0; it < trips; ++it) {
+        const uint32_t t = (it * gridDim.x + blockIdx.x) * kThreads + threadIdx.x;
+        Quad h[RMAX];
+        quad_hashes<RMAX>(P, r, t < d4 ? t : d4 - 1, h);
+        if (t >= d4) continue;
+        const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
+        for (uint32_t w = w0; w < w0 + nw; ++w) {
+            const uint64_t q0 = (uint64_t)w * d4 + t;
+            const float4 g0 = __ldcs(grads + q0);
+            float4 m0 = __ldcs(m + q0), v0 = __ldcs(vw + q0), h0 = __ldcs(vhw + q0), a0 = __ldcs(e + q0);
+            pa_moment(b1, omb1, b2, omb2, g0.x, m0.x, v0.x, h0.x, a0.x, mask & 1u);
+            pa_moment(b1, omb1, b2, omb2, g0.y, m0.y, v0.y, h0.y, a0.y, mask & 2u);
+            pa_moment(b1, omb1, b2, omb2, g0.z, m0.z, v0.z, h0.z, a0.z, mask & 4u);
+            pa_moment(b1, omb1, b2, omb2, g0.w, m0.w, v0.w, h0.w, a0.w, mask & 8u);
+            __stcs(m + q0, m0); __stcs(vw + q0, v0); __stcs(vhw + q0, h0); __stcs(e + q0, a0);
+            float* t0 = A.tables + (uint64_t)w * tstride;
+#pragma unroll
+            for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+                if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+        }
+    }
+}
+
 // Scalar form: any d, any alignment, any group size.  One thread per coordinate.
 __global__ void __launch_bounds__(kThreads)
 k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
@@ -131,8 +179,16 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q = (uint64_t)w * P.d + j;
             const float g = A.grads[q];
-            const float mm = fmaf(b1, A.m[q], omb1 * g);
-            const float a = mm + (member ? 0.0f : A.e[q]);
+            float mm, a;
+            if (A.variant == 1) {
+                float vv = A.vw[q], vh = A.vhatw[q];
+                mm = A.m[q]; a = A.e[q];
+                pa_moment(b1, omb1, P.beta2, 1.0f - P.beta2, g, mm, vv, vh, a, member);
+                A.vw[q] = vv; A.vhatw[q] = vh;
+            } else {
+                mm = fmaf(b1, A.m[q], omb1 * g);
+                a = mm + (member ? 0.0f : A.e[q]);
+            }
             gs += g;
             A.m[q] = mm;
             A.e[q] = a;
@@ -142,7 +198,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
                 atomicAdd(A.tables + (uint64_t)w * tstride + (uint64_t)row * P.cs + b, s * a);
             }
         }
-        if (member) A.gsum[j] = gs;
+        if (member && A.variant == 0) A.gsum[j] = gs;
     }
 }
 
@@ -206,6 +262,15 @@ int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint
         return 1;
     }
     const int grid = grid_for(P.d >> 2, sm_count, 1);    // the caller passes SMs x CTAs per SM
+    if (A.variant == 1) {
+#define SK_CASE(RR) case RR: k_moment_sketch_pa_v4<RR><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
+        switch (P.r) {
+            SK_CASE(1) SK_CASE(2) SK_CASE(3) SK_CASE(4) SK_CASE(5) SK_CASE(6) SK_CASE(7) SK_CASE(8) SK_CASE(10)
+            default: k_moment_sketch_pa_v4<0><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
+        }
+#undef SK_CASE
+        return 1;
+    }
 #define SK_CASE(RR) case RR: k_moment_sketch_v4<RR><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
     switch (P.r) {
         SK_CASE(1) SK_CASE(2) SK_CASE(3) SK_CASE(4) SK_CASE(5) SK_CASE(6) SK_CASE(7) SK_CASE(8) SK_CASE(10)

@@ -16,6 +16,8 @@ struct sk_state {
     size_t l2_bytes = 0;
     int64_t worker_chunk = 0;
     int64_t window_lines = 0;
+    int64_t variant = 0;          // 0 = gradient averaging (Algorithm 2), 1 = parameter averaging (Algorithm 1)
+    float *vw = nullptr, *vhatw = nullptr;   // per-worker v, vhat of the parameter-averaging variant (n*d each)
     int64_t window_workers = 4;
     int64_t window_red_rows = 0;
     int64_t sketch_ctas_per_sm = 64;

@@ -83,6 +83,7 @@ extern "C" int sk_select_static(sk_state* s, uint32_t* idx_out) {
     sk::launch_zero(base + kOffHist, kOffKeys - kOffHist, st);
     sk::MomentArgs A{};                 // members = 0: read vhat only, the step's own update is not repeated
     A.vhat = s->vhat;
+    A.variant = (uint32_t)s->variant;
     sk::launch_unsketch_hist(P, A, s->sum, keys, hist, vec, s->sm_count, st);
     sk::launch_pick_bin(P, hist, sel, 0, st);
     sk::launch_emit(P, keys, sel, idx_out, cand, hist2, s->sm_count, st);

@@ -59,25 +59,30 @@ def index_sets_agree(I_gpu, I_ref, est_ref, k, what="I", rel=REL, scale=None):
     return diff
 
 
-def force_state(gpu, ora):
-    """Teacher forcing: install the oracle's state (m, e, v, vhat, I_{t-1}, t) in the GPU handle."""
+def force_state(gpu, ora, variant="ga"):
+    """Teacher forcing: install the oracle's state (m, e, v, vhat or vw, vhatw, I_{t-1}, t) in the GPU handle."""
     t = np.array([ora.t], np.uint64)
     gpu.set("t", t)
-    for f in ("m", "e", "v", "vhat"):
+    for f in (("m", "e", "v", "vhat") if variant == "ga" else ("m", "e", "vw", "vhatw")):
         gpu.set(f, np.ascontiguousarray(ora.field(f)))
     gpu.set("I", np.ascontiguousarray(ora.field("I_prev")))
 
 
-def compare_step(gpu, ora, x_gpu, x_ref, x_before, lr, check_tables=True, x_gpu_before=None):
+def compare_step(gpu, ora, x_gpu, x_ref, x_before, lr, check_tables=True, x_gpu_before=None, variant="ga"):
     """Compares every stage output of the step both sides just took from the same state and gradients."""
     d, n, k = ora.d, ora.n, ora.k
     if check_tables:
         close(gpu.get("tables"), ora.field("tables"), "worker sketches", groups_axis=1)
     close(gpu.get("sum"), ora.field("sum"), "aggregated sketch", groups_axis=0)
-    close(gpu.get("vhat"), ora.field("vhat"), "vhat")
-    close(gpu.get("v"), ora.field("v"), "v")
+    if variant == "ga":
+        close(gpu.get("vhat"), ora.field("vhat"), "vhat")
+        close(gpu.get("v"), ora.field("v"), "v")
+        sc = est_scale(ora.field("sum"), ora.field("vhat"))
+    else:                       # Algorithm 1: per-worker second moments (sums of non-negative terms: element-relative),
+        np.testing.assert_allclose(gpu.get("vw"), ora.field("vw"), rtol=REL, atol=0)       # and a plain unsketch
+        np.testing.assert_allclose(gpu.get("vhatw"), ora.field("vhatw"), rtol=REL, atol=0)
+        sc = est_scale(ora.field("sum"), np.ones(d, np.float32))
     est_ref = ora.field("est")
-    sc = est_scale(ora.field("sum"), ora.field("vhat"))
     close(gpu.get("est"), est_ref, "estimates", scale=sc)
     I_gpu = gpu.get("I")
     assert np.all(np.diff(I_gpu.astype(np.int64)) > 0)

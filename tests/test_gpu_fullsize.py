@@ -14,19 +14,19 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 
-def _setup(name, window_lines=None):
+def _setup(name, window_lines=None, variant="ga"):
     from paper_2210_07454_b200 import binding, synthetic
     w = synthetic.WORKLOADS[name]
     src = synthetic.GradientSource(w, device="cuda")
     gpu = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                                  eps=w.eps, window_lines=window_lines)
+                                  eps=w.eps, window_lines=window_lines, variant=variant)
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=gpu.get_option("log2g"), lr=w.lr,
                         beta1=w.beta1, beta2=w.beta2, eps=w.eps, threads=32,
-                        window_lines=gpu.get_option("window_lines"))
+                        window_lines=gpu.get_option("window_lines"), variant=variant)
     return w, src, gpu, ora
 
 
-def _one_step(w, src, gpu, ora, t, x_gpu, x_ref):
+def _one_step(w, src, gpu, ora, t, x_gpu, x_ref, variant="ga"):
     g = src.grads(t)
     g_host = g.cpu().numpy()
     x_before = x_ref.astype(np.float64).copy()
@@ -34,7 +34,7 @@ def _one_step(w, src, gpu, ora, t, x_gpu, x_ref):
     gpu.sync()
     del g
     ora.step(g_host, x_ref)
-    return compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr)
+    return compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, variant=variant)
 
 
 @pytest.mark.parametrize("name", ["C2", "C3"])
@@ -53,6 +53,16 @@ def test_c3_windowed_family_first_step():
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
     _one_step(w, src, gpu, ora, 1, x_gpu, x_ref)
+
+
+def test_c3_parameter_averaging_two_teacher_forced_steps():
+    w, src, gpu, ora = _setup("C3", variant="pa")
+    x_gpu = src.x0()
+    x_ref = x_gpu.cpu().numpy().copy()
+    _one_step(w, src, gpu, ora, 1, x_gpu, x_ref, variant="pa")
+    force_state(gpu, ora, "pa")
+    x_gpu.copy_(torch.from_numpy(x_ref))
+    _one_step(w, src, gpu, ora, 2, x_gpu, x_ref, variant="pa")
 
 
 @pytest.mark.parametrize("name", ["C4", "C5"])

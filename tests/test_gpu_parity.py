@@ -28,13 +28,13 @@ def _workload(base, **over):
     return w
 
 
-def _pair(w, log2g=None, threads=8, window_lines=None):
+def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga"):
     b = _binding()
     gpu = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                            eps=w.eps, log2g=log2g, window_lines=window_lines)
+                            eps=w.eps, log2g=log2g, window_lines=window_lines, variant=variant)
     lg = gpu.get_option("log2g")
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=lg, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                        eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"))
+                        eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"), variant=variant)
     return gpu, ora
 
 
@@ -62,8 +62,8 @@ def test_hash_bit_exact(log2g, c):
 
 
 # ------------------------------------------------------------------------------------------------ steps
-def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True, window_lines=None):
-    gpu, ora = _pair(w, log2g, window_lines=window_lines)
+def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True, window_lines=None, variant="ga"):
+    gpu, ora = _pair(w, log2g, window_lines=window_lines, variant=variant)
     src = _source(w, cfg_id=cfg_id)
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
@@ -72,7 +72,7 @@ def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=Tru
         g = src.grads(t)
         g_host = g.cpu().numpy()
         if teacher and t > 1:
-            force_state(gpu, ora)
+            force_state(gpu, ora, variant)
             x_gpu.copy_(torch.from_numpy(x_ref))
         x_before = x_ref.astype(np.float64).copy()
         x_gpu_before = x_gpu.cpu().numpy().copy()
@@ -80,7 +80,7 @@ def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=Tru
         gpu.sync()
         ora.step(g_host, x_ref)
         diff = compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, check_tables=check_tables,
-                            x_gpu_before=x_gpu_before)
+                            x_gpu_before=x_gpu_before, variant=variant)
         if diff.size and diverged_at is None:
             diverged_at = t
             if not teacher:
@@ -200,6 +200,44 @@ EDGE = {
 def test_edge_cases(case):
     w = _workload("C1", name="E", steps=3, recipe="planted", **EDGE[case])
     _run_steps(w, 3, cfg_id=7)
+
+
+# ---------------------------------------------------------------------------- parameter averaging (Algorithm 1)
+def test_pa_c1_ten_steps_teacher_forced():
+    _run_steps(_workload("C1"), 10, variant="pa")
+
+
+PA_CASES = {
+    "scalar_path": dict(d=10_007, n=3, r=5, c=1000, k=333),
+    "rows16_odd_workers": dict(d=12_000, n=5, r=16, c=1024, k=120),
+    "even_rows": dict(d=30_000, n=2, r=10, c=2048, k=300),
+    "k_eq_d": dict(d=2048, n=2, r=3, c=4096, k=2048),
+    "windowed_family": dict(d=40_000, n=6, r=5, c=4096, k=400, L=8),   # Algorithm 1 on the windowed hash family
+}
+
+
+@pytest.mark.parametrize("case", sorted(PA_CASES))
+def test_pa_edge_cases(case):
+    cfg = dict(PA_CASES[case])
+    L = cfg.pop("L", None)
+    w = _workload("C1", name="E", steps=3, recipe="planted", **cfg)
+    _run_steps(w, 3, cfg_id=7, variant="pa", window_lines=L)
+
+
+def test_pa_state_fields_and_errors():
+    b = _binding()
+    ga = b.SketchedAMSGrad(1000, 2, 3, 256, 10)
+    with pytest.raises(b.SkError):
+        ga.get("vw")                                  # per-worker second moments exist only for Algorithm 1
+    pa = b.SketchedAMSGrad(1000, 2, 3, 256, 10, variant="pa", eps=1e-3)
+    assert np.all(pa.get("vw") == np.float32(1e-3)) and np.all(pa.get("vhatw") == np.float32(1e-3))
+    with pytest.raises(b.SkError):
+        pa.get("vhat")
+    x = torch.zeros(1000, device="cuda")
+    pa.step(torch.ones((2, 1000), device="cuda"), x)
+    with pytest.raises(b.SkError):
+        pa.set_option("variant", 0)                   # fixed after the first step
+    assert pa.algorithmic_bytes() == 36 * 2 * 1000 + 8 * 2 * 3 * 256 + 4 * 3 * 256 + 8 * 2 * 10 + 8 * 10
 
 
 def test_worker_chunking_matches_single_pass():
