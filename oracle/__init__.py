@@ -120,7 +120,7 @@ class Oracle:
     """One SketchedAMSGrad (gradient averaging) optimiser; `step` advances it by one iteration."""
 
     def __init__(self, d, n, r, c, k, seed=0, log2g=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8,
-                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0, variant="ga"):
+                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0, variant="ga", P=1):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
         self._h = lib().ora_create(d, n, r, c, k, seed, log2g, lr, beta1, beta2, eps)
         if not self._h:
@@ -138,6 +138,10 @@ class Oracle:
         if variant not in ("ga", "pa"):
             raise ValueError("variant must be 'ga' (Algorithm 2) or 'pa' (Algorithm 1)")
         lib().ora_set_option(self._h, b"variant_pa", int(variant == "pa"))
+        if P != 1:
+            if P < 1 or P * k > d:
+                raise ValueError("P must be >= 1 with P*k <= d")
+            lib().ora_set_option(self._h, b"P", int(P))
         lib().ora_set_option(self._h, b"v_keep", int(v_keep))
         lib().ora_set_option(self._h, b"threads", int(threads))
 
@@ -165,7 +169,7 @@ class Oracle:
         ptr = lib().ora_field(self._h, name.encode())
         if not ptr:
             raise KeyError(name)
-        if name in ("I", "I_prev"):
+        if name in ("I", "I_prev", "cand"):
             cnt = int(lib().ora_count(self._h, name.encode()))
             buf = (C.c_uint32 * max(cnt, 1)).from_address(ptr)
             return np.frombuffer(buf, np.uint32, cnt)

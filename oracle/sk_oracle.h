@@ -67,7 +67,8 @@ ora_state* ora_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k
 void ora_destroy(ora_state* s);
 /* inject explicit hash arrays (r*d each) instead of the seeded family; pointers must outlive the state */
 void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn);
-/* "v_keep", "threads", "window_lines" (windowed hash family), "variant_pa" (1 = Algorithm 1, parameter averaging;
+/* "P" (candidate multiplier of the second round, Section III-A: top P*k by estimate, then top-k by exact value;
+   the candidates of the last step are the uint32 field "cand"), "v_keep", "threads", "window_lines" (windowed hash family), "variant_pa" (1 = Algorithm 1, parameter averaging;
    per-worker v and vhat are then the fields "vw" and "vhatw", n*d each) */
 void ora_set_option(ora_state* s, const char* key, int value);
 int  ora_step(ora_state* s, const float* grads /* n*d worker-major */, float* x /* d, in place */);

@@ -15,6 +15,8 @@ struct ora_state {
     uint32_t n, r, c, log2g, window_lines;
     float lr, beta1, beta2, eps;
     int v_keep, threads, variant_pa;
+    uint32_t P;              /* candidate multiplier of the second round (Section III-A); 1 = no second round */
+    uint32_t* cand;          /* the P*k candidates of the last step, ascending */
     float *vw, *vhatw;       /* parameter-averaging variant: per-worker v and vhat (n*d each) */
     float *m, *e, *v, *vhat, *est, *tables, *sum;
     uint32_t *I, *I_prev;
@@ -32,6 +34,7 @@ ora_state* ora_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k
     s->d = d; s->n = n; s->r = r; s->c = c; s->k = k; s->seed = seed; s->log2g = log2g;
     s->lr = lr; s->beta1 = beta1; s->beta2 = beta2; s->eps = eps;
     s->threads = 1;
+    s->P = 1;
     s->m = (float*)calloc((size_t)n * d, sizeof(float));        /* m_0 = 0 */
     s->e = (float*)calloc((size_t)n * d, sizeof(float));        /* e_0 = 0 */
     s->v = (float*)malloc((size_t)d * sizeof(float));
@@ -52,7 +55,7 @@ ora_state* ora_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k
 void ora_destroy(ora_state* s) {
     if (!s) return;
     free(s->m); free(s->e); free(s->v); free(s->vhat); free(s->est); free(s->tables); free(s->sum);
-    free(s->I); free(s->I_prev); free(s->mask); free(s->row_key); free(s->vw); free(s->vhatw); free(s);
+    free(s->I); free(s->I_prev); free(s->mask); free(s->row_key); free(s->vw); free(s->vhatw); free(s->cand); free(s);
 }
 
 void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn) { s->h_idx = idx; s->h_sgn = sgn; }
@@ -65,6 +68,13 @@ void ora_set_option(ora_state* s, const char* key, int value) {
             s->window_lines = (uint32_t)value;
     }
     else if (!strcmp(key, "threads")) s->threads = value > 0 ? value : 1;
+    else if (!strcmp(key, "P")) {
+        if (value >= 1 && (uint64_t)value * s->k <= s->d && s->t == 0) {
+            s->P = (uint32_t)value;
+            free(s->cand);
+            s->cand = (uint32_t*)calloc((size_t)s->P * s->k, sizeof(uint32_t));
+        }
+    }
     else if (!strcmp(key, "variant_pa")) {
         /* Algorithm 1 (parameter averaging); only before the first step.  v_0^(i) = vhat_0^(i) = eps. */
         if (value && !s->vw && s->t == 0) {
@@ -87,6 +97,7 @@ void* ora_field(ora_state* s, const char* name) {
     if (!strcmp(name, "sum")) return s->sum;
     if (!strcmp(name, "I")) return s->I;
     if (!strcmp(name, "I_prev")) return s->I_prev;
+    if (!strcmp(name, "cand")) return s->cand;
     if (!strcmp(name, "vw")) return s->vw;
     if (!strcmp(name, "vhatw")) return s->vhatw;
     return NULL;
@@ -96,6 +107,7 @@ uint64_t ora_count(ora_state* s, const char* name) {
     if (!strcmp(name, "I_prev")) return s->k_prev;
     if (!strcmp(name, "I")) return s->t ? s->k : 0;
     if (!strcmp(name, "t")) return s->t;
+    if (!strcmp(name, "cand")) return (s->t && s->P > 1) ? (uint64_t)s->P * s->k : 0;
     return 0;
 }
 
@@ -118,6 +130,33 @@ static inline void hash_at(const ora_state* s, uint32_t j, uint64_t i, uint32_t*
 }
 
 static int ora_step_pa(ora_state* s, const float* grads, float* x);
+
+/* Second round of Section III-A ("In practice ..."): of the estimates take the P*k largest as candidates, fetch the
+ * EXACT values of the compressed vector there -- `exact[j]` is computed by the caller for the candidates only --
+ * and keep the k candidates of largest exact magnitude (ties: smaller index).  With P = 1 this is plain Top-k of
+ * the estimates.  `scale` is vhat for Algorithm 2 (exact value = mean_w a / sqrt(vhat)) or NULL for Algorithm 1. */
+static void select_with_second_round(ora_state* s, const float* scale) {
+    const uint64_t d = s->d, k = s->k;
+    if (s->P <= 1) { ora_topk(s->est, d, k, s->I); return; }
+    const uint64_t pk = (uint64_t)s->P * k;
+    ora_topk(s->est, d, pk, s->cand);
+    float* exact = (float*)calloc((size_t)d, sizeof(float));       /* zero off the candidate set */
+    for (uint64_t t = 0; t < pk; ++t) {
+        uint64_t j = s->cand[t];
+        double abar = 0.0;
+        for (uint32_t w = 0; w < s->n; ++w) abar += (double)s->e[(uint64_t)w * d + j];
+        abar /= (double)s->n;
+        exact[j] = (float)(scale ? abar / sqrt((double)scale[j]) : abar);
+    }
+    /* top-k of the exact magnitudes among the candidates: every non-candidate holds 0 and, to keep a zero-valued
+       candidate ahead of non-candidates, the selection runs over the candidate list itself */
+    float* cval = (float*)malloc((size_t)pk * sizeof(float));
+    uint32_t* pos = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+    for (uint64_t t = 0; t < pk; ++t) cval[t] = exact[s->cand[t]];
+    ora_topk(cval, pk, k, pos);            /* cand is ascending, so "smaller position" = "smaller index" */
+    for (uint64_t t = 0; t < k; ++t) s->I[t] = s->cand[pos[t]];
+    free(pos); free(cval); free(exact);
+}
 
 int ora_step(ora_state* s, const float* grads, float* x) {
     if (s->variant_pa) return ora_step_pa(s, grads, x);
@@ -194,8 +233,8 @@ int ora_step(ora_state* s, const float* grads, float* x) {
         s->est[i] = (float)((double)ora_median(q, r) / sqrt((double)s->vhat[i]));
     }
 
-    /* I_t = index set of Top-k of the estimates */
-    ora_topk(s->est, d, k, s->I);
+    /* I_t = index set of Top-k of the estimates (after the second round on P*k candidates when P > 1) */
+    select_with_second_round(s, s->vhat);
 
     /* Delta_t = (1/n) sum_w Delta_t^(w): exact coordinates of vhat^{-1/2} a_t^(w) on I_t;
        x_{t+1} = x_t - alpha_t Delta_t ;  e_t^(w) = a_t^(w) with the coordinates of I_t removed */
@@ -274,7 +313,7 @@ static int ora_step_pa(ora_state* s, const float* grads, float* x) {
         }
         s->est[i] = ora_median(q, r);
     }
-    ora_topk(s->est, d, k, s->I);
+    select_with_second_round(s, NULL);
     for (uint64_t t = 0; t < k; ++t) {
         uint64_t j = s->I[t];
         double abar = 0.0;

@@ -188,3 +188,72 @@ def test_threads_do_not_change_results():
         outs.append((x.copy(), o.field("e").copy(), o.field("sum").copy(), o.field("I").copy()))
     for a, b in zip(*outs):
         assert np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------------- second round with P*k candidates
+def test_second_round_selects_by_exact_values_among_candidates():
+    # Section III-A: take the P*k largest estimates as candidates, fetch the exact values there, keep the k largest
+    # exact magnitudes.  Checked against a brute-force restatement with numpy on a lossy sketch.
+    d, n, r, c, k, P = 4000, 3, 5, 1024, 40, 4
+    rng = np.random.default_rng(11)
+    o = oracle.Oracle(d, n, r, c, k, seed=2, log2g=2, lr=1e-2, eps=1e-6, P=P)
+    o1 = oracle.Oracle(d, n, r, c, k, seed=2, log2g=2, lr=1e-2, eps=1e-6)
+    x = np.zeros(d, np.float32); x1 = x.copy()
+    hits = []
+    for t in range(4):
+        g = (rng.standard_normal((n, d)) * rng.uniform(0.01, 1.0, d)).astype(np.float32)
+        e_prev = o.field("e").copy()
+        o.step(g, x)
+        est, vh, I, cand = o.field("est"), o.field("vhat"), o.field("I"), o.field("cand")
+        assert len(cand) == P * k and np.array_equal(cand, oracle.topk(est, P * k))
+        a = (o.field("m").astype(np.float64) + e_prev.astype(np.float64)).astype(np.float32)
+        exact = (a.astype(np.float64).mean(0) / np.sqrt(vh.astype(np.float64))).astype(np.float32)
+        order = np.lexsort((cand, -np.abs(exact[cand])))                 # exact magnitude desc, index asc
+        assert np.array_equal(I, np.sort(cand[order[:k]]))
+        assert np.isin(I, cand).all()
+        true_top = np.argsort(-np.abs(exact), kind="stable")[:k]
+        hits.append(np.isin(true_top, I).mean())
+        # error feedback still masks exactly I_t
+        assert not o.field("e")[:, I].any()
+    # the same run without the second round recovers fewer of the true top-k on this lossy sketch
+    base = []
+    rng = np.random.default_rng(11)
+    for t in range(4):
+        g = (rng.standard_normal((n, d)) * rng.uniform(0.01, 1.0, d)).astype(np.float32)
+        e_prev = o1.field("e").copy()
+        o1.step(g, x1)
+        a = (o1.field("m").astype(np.float64) + e_prev.astype(np.float64)).astype(np.float32)
+        exact = (a.astype(np.float64).mean(0) / np.sqrt(o1.field("vhat").astype(np.float64))).astype(np.float32)
+        base.append(np.isin(np.argsort(-np.abs(exact), kind="stable")[:k], o1.field("I")).mean())
+    assert hits[0] > base[0] + 0.1 and hits[0] > 0.6, (hits, base)    # first step: both start from the same state
+
+
+def test_second_round_is_neutral_for_a_lossless_sketch_and_for_p1():
+    d, n, k = 300, 2, 20
+    hi, hs = _identity(d)
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal((3, n, d)).astype(np.float32)
+    res = []
+    for P in (1, 3):
+        o = oracle.Oracle(d, n, 1, d, k, hash_idx=hi, hash_sgn=hs, lr=1e-2, eps=1e-6, P=P)
+        x = np.zeros(d, np.float32)
+        for t in range(3):
+            o.step(g[t], x)
+        res.append((x.copy(), o.field("I").copy(), o.field("e").copy()))
+    for a, b in zip(*res):
+        assert np.array_equal(a, b)
+
+
+def test_second_round_parameter_averaging():
+    d, n, r, c, k, P = 3000, 2, 3, 128, 30, 4
+    rng = np.random.default_rng(12)
+    o = oracle.Oracle(d, n, r, c, k, seed=3, log2g=0, lr=1e-2, eps=1e-6, P=P, variant="pa")
+    x = np.zeros(d, np.float32)
+    for t in range(2):
+        e_prev = o.field("e").copy()
+        o.step(rng.standard_normal((n, d)).astype(np.float32), x)
+    cand, I = o.field("cand"), o.field("I")
+    a = (o.field("m").astype(np.float64) / np.sqrt(o.field("vhatw").astype(np.float64)) + e_prev).astype(np.float32)
+    exact = a.astype(np.float64).mean(0).astype(np.float32)
+    order = np.lexsort((cand, -np.abs(exact[cand])))
+    assert np.array_equal(I, np.sort(cand[order[:k]]))
