@@ -117,7 +117,7 @@ def reduce_sum(value: float, world: int, device) -> float:
     return float(t.item())
 
 
-def cpu_oracle_rate(w, scale: int, steps: int, threads: int):
+def cpu_oracle_rate(w, scale: int, steps: int, threads: int, variant: str = "ga", P: int = 1):
     """Times the CPU oracle, as it stands, on `steps` steps of the workload scaled down by `scale`."""
     import oracle
     from paper_2210_07454_b200 import synthetic
@@ -127,7 +127,7 @@ def cpu_oracle_rate(w, scale: int, steps: int, threads: int):
     while (1 << lg) > ws.c:
         lg -= 1
     o = oracle.Oracle(ws.d, ws.n, ws.r, ws.c, ws.k, seed=ws.seed, log2g=lg, lr=ws.lr, beta1=ws.beta1, beta2=ws.beta2,
-                      eps=ws.eps, threads=threads)
+                      eps=ws.eps, threads=threads, variant=variant, P=P)
     x = src.x0().numpy()
     grads = [src.grads(t).numpy() for t in range(1, min(steps, 2) + 1)]
     times = []
@@ -147,7 +147,7 @@ def run_reference(args, w):
     threads = os.cpu_count() or 1
     scale = args.ref_scale
     total = args.steps + args.warmup
-    ws, times, sample = cpu_oracle_rate(w, scale, total, threads)
+    ws, times, sample = cpu_oracle_rate(w, scale, total, threads, args.variant, args.P)
     timed = times[args.warmup:]
     ms = 1e3 * sum(timed) / len(timed)
     value = ws.n * ws.d / (ms * 1e-3) / 1e9
@@ -170,6 +170,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--log2g", type=int, default=None)
+    ap.add_argument("--P", type=int, default=1,
+                    help="candidate multiplier of the second selection round (Section III-A); 1 = no second round")
     ap.add_argument("--variant", default="ga", choices=["ga", "pa"],
                     help="ga = gradient averaging (Algorithm 2, the headline path); pa = parameter averaging (Algorithm 1)")
     ap.add_argument("--window-lines", type=int, default=None, help="windowed hash family: lines per window (0 = plain)")
@@ -206,7 +208,8 @@ def main():
 
     src = synthetic.GradientSource(w, device=dev, cfg_id=cfg_id)
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                                  eps=w.eps, log2g=args.log2g, window_lines=args.window_lines, variant=args.variant)
+                                  eps=w.eps, log2g=args.log2g, window_lines=args.window_lines, variant=args.variant,
+                                  P=args.P)
     opt.set_option("worker_chunk", args.worker_chunk)
     if args.window_workers:
         opt.set_option("window_workers", args.window_workers)
@@ -297,7 +300,7 @@ def main():
     if world == 1 and not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
         scale = 4
-        ws, times, sample = cpu_oracle_rate(w, scale, 3, threads)
+        ws, times, sample = cpu_oracle_rate(w, scale, 3, threads, args.variant, args.P)
         cpu = {"value": ws.n * ws.d / (sum(times[1:]) / len(times[1:])) / 1e9, "unit": UNIT, "cores": threads,
                "kind": "oracle", "sample": sample}
 
@@ -305,7 +308,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k,
-                       "recipe": w.recipe, "variant": args.variant, "hash_group": 1 << opt.get_option("log2g"),
+                       "recipe": w.recipe, "variant": args.variant, "P": args.P, "hash_group": 1 << opt.get_option("log2g"),
                        "window_lines": opt.get_option("window_lines"),
                        "worker_chunk": opt.get_option("worker_chunk"), "replicas": world,
                        "l2": f"inputs larger than L2: {nsets} rotating gradient sets of {set_bytes / 1e9:.2f} GB"},

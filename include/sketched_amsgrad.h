@@ -70,6 +70,10 @@ int sk_sync(sk_state* state);
 /* Options (integers):
  *   "log2g"        hash group size g = 2^log2g, 0..5 (Section II-C fixes no hash family; see sk_hash).
  *                  Only before the first step.  Default: the largest value <= 5 with 2^log2g <= c.
+ *   "P"            candidate multiplier of the second round (Section III-A, "In practice ..."): the P*k largest
+ *                  estimates become candidates, their exact values are fetched from the workers' vectors, and the
+ *                  k candidates of largest exact magnitude form I_t (ties: smaller index).  1 (default) = no second
+ *                  round.  P*k <= d.  Only before the first step.  The candidates of the last step are field "cand".
  *   "variant"      0 (default) = gradient averaging, Algorithm 2; 1 = parameter averaging, Algorithm 1: every worker
  *                  keeps its own v and vhat (fields "vw", "vhatw", n*d each, initial value eps) from its own
  *                  gradient, sketches m/sqrt(vhat) + e, the unsketch takes no vhat and x moves by the plain mean
@@ -105,6 +109,7 @@ int sk_hash(const sk_state* state, uint32_t row, uint64_t i0, uint64_t count,
  *   "est"     d    the estimates of the last step (recomputed on request from "sum" and "vhat"; get only)
  *   "I"       k uint32  I_t of the last step, ascending (get);  set: installs I_{t-1} for the next step
  *   "vw","vhatw" n*d  per-worker second moments (parameter-averaging variant only; "v","vhat" are then unavailable)
+ *   "cand"    P*k uint32  candidates of the last step's second round, ascending (get only; empty when P = 1)
  *   "t"       1 uint64  number of steps taken
  * Both calls synchronise the stream. */
 int sk_get(sk_state* state, const char* field, void* buf, uint64_t bytes);

@@ -121,7 +121,7 @@ class Oracle:
 
     def __init__(self, d, n, r, c, k, seed=0, log2g=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8,
                  hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0, variant="ga", P=1):
-        self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
+        self.d, self.n, self.r, self.c, self.k, self.P = d, n, r, c, k, P
         self._h = lib().ora_create(d, n, r, c, k, seed, log2g, lr, beta1, beta2, eps)
         if not self._h:
             raise ValueError("ora_create rejected the arguments")

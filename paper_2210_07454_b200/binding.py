@@ -83,7 +83,7 @@ class SketchedAMSGrad:
                      "vw": "nd", "vhatw": "nd"}
 
     def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None,
-                 window_lines=None, variant="ga"):
+                 window_lines=None, variant="ga", P=1):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
         self._h = lib().sk_create(d, n, r, c, k, seed, lr, beta1, beta2, eps)
         if not self._h:
@@ -96,6 +96,9 @@ class SketchedAMSGrad:
             raise SkError("variant must be 'ga' (Algorithm 2, gradient averaging) or 'pa' (Algorithm 1)")
         if variant == "pa":
             self.set_option("variant", 1)
+        self.P = P
+        if P != 1:
+            self.set_option("P", P)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -138,6 +141,8 @@ class SketchedAMSGrad:
         if out is None:
             if field == "I":
                 out = np.empty(self._count_I(), np.uint32)
+            elif field == "cand":
+                out = np.empty(self.P * self.k if (self.P > 1 and self._count_I()) else 0, np.uint32)
             elif field == "t":
                 out = np.empty(1, np.uint64)
             else:

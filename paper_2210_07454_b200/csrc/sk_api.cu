@@ -150,16 +150,37 @@ int do_step(sk_state* s, const float* grads, float* x) {
         StageTimer tm(s, 4);
         // ranking keys; v and vhat on I_{t-1} are brought up to date on the way, from the sums in gsum
         int l = sk::launch_unsketch_hist(P, A, s->sum, s->keys, s->hist, vec, s->sm_count, st);
-        l += sk::launch_pick_bin(P, s->hist, s->sel, 0, st);
+        sk::Params Q = P;
+        Q.k = (uint32_t)s->cand_mult * P.k;         // with a second round the first selection takes P*k candidates
+        l += sk::launch_pick_bin(Q, s->hist, s->sel, 0, st);
         tm.done(l);
     }
-    {
-        StageTimer tm(s, 5);
-        tm.done(sk::launch_emit(P, s->keys, s->sel, s->I, s->cand, s->hist2, s->sm_count, st));
-    }
-    {
+    if (s->cand_mult <= 1) {
+        {
+            StageTimer tm(s, 5);
+            tm.done(sk::launch_emit(P, s->keys, nullptr, s->sel, s->I, s->cand, s->hist2, s->sm_count, st));
+        }
         StageTimer tm(s, 6);
         tm.done(sk::launch_refine(P, s->sel, s->cand, s->cand2, s->hist2, s->I, s->sm_count, st));
+    } else {
+        // Second round (Section III-A): the P*k largest estimates become candidates, their exact values are
+        // fetched, and the k candidates of largest exact magnitude are kept (ties: smaller index).
+        sk::Params Q = P;                       // first selection: P*k of d (the threshold bin was picked for P*k)
+        Q.k = (uint32_t)s->cand_mult * P.k;
+        {
+            StageTimer tm(s, 5);
+            tm.done(sk::launch_emit(Q, s->keys, nullptr, s->sel, s->Ic, s->cand, s->hist2, s->sm_count, st));
+        }
+        StageTimer tm(s, 6);
+        int l = sk::launch_refine(Q, s->sel, s->cand, s->cand2, s->hist2, s->Ic, s->sm_count, st);
+        l += sk::launch_exact_keys(P, s->Ic, Q.k, s->variant == 1 ? nullptr : s->vhat, s->e, s->keys2, s->hist,
+                                   s->sm_count, st);
+        sk::Params Q2 = P;                      // second selection: k of the P*k candidates, keyed by exact value
+        Q2.d = Q.k;
+        l += sk::launch_pick_bin(Q2, s->hist, s->sel, 0, st);
+        l += sk::launch_emit(Q2, s->keys2, s->Ic, s->sel, s->I, s->cand, s->hist2, s->sm_count, st);
+        l += sk::launch_refine(Q2, s->sel, s->cand, s->cand2, s->hist2, s->I, s->sm_count, st);
+        tm.done(l);
     }
     {
         StageTimer tm(s, 7);     // the bitmap of I_{t-1} has served its purpose: clear it, then apply marks I_t
@@ -175,11 +196,11 @@ int do_step(sk_state* s, const float* grads, float* x) {
     return SK_OK;
 }
 
-enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_VW, F_VHATW, F_BAD };
+enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_VW, F_VHATW, F_CAND, F_BAD };
 
 Field field_of(const char* name) {
-    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t", "vw", "vhatw"};
-    for (int q = 0; q < 11; ++q) if (!strcmp(name, names[q])) return (Field)q;
+    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t", "vw", "vhatw", "cand"};
+    for (int q = 0; q < 12; ++q) if (!strcmp(name, names[q])) return (Field)q;
     return F_BAD;
 }
 
@@ -266,7 +287,7 @@ void sk_destroy(sk_state* s) {
     if (s->stream) cudaStreamSynchronize(s->stream); else cudaDeviceSynchronize();
     for (void* p : {(void*)s->m, (void*)s->e, (void*)s->v, (void*)s->vhat, (void*)s->vstamp, (void*)s->tables,
                     (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->hist2, (void*)s->sel, (void*)s->cand, (void*)s->cand2,
-                    (void*)s->keys, (void*)s->gsum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw,
+                    (void*)s->keys, (void*)s->gsum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw, (void*)s->Ic, (void*)s->keys2,
                     (void*)s->stage_grads, (void*)s->stage_x})
         if (p) cudaFree(p);
     for (const TimeRec& r : s->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -329,6 +350,18 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         refresh_hash(s);
         return SK_OK;
     }
+    if (!strcmp(key, "P")) {
+        if (s->t != 0) return fail(SK_ESTATE, "P can only be changed before the first step");
+        if (value < 1 || (uint64_t)value * s->P.k > s->P.d) return fail(SK_EINVAL, "P must be >= 1 with P*k <= d");
+        if (value > 1) {
+            if (s->Ic) { cudaFree(s->Ic); cudaFree(s->keys2); s->Ic = s->keys2 = nullptr; }
+            const uint64_t pk = (uint64_t)value * s->P.k;
+            if (cudaMalloc((void**)&s->Ic, pk * 4) != cudaSuccess || cudaMalloc((void**)&s->keys2, pk * 4) != cudaSuccess)
+                return fail(SK_ENOMEM, "cudaMalloc of the candidate buffers failed: %s", cudaGetErrorString(cudaGetLastError()));
+        }
+        s->cand_mult = value;
+        return SK_OK;
+    }
     if (!strcmp(key, "variant")) {
         if (s->t != 0) return fail(SK_ESTATE, "variant can only be changed before the first step");
         if (value != 0 && value != 1) return fail(SK_EINVAL, "variant must be 0 (gradient averaging) or 1 (parameter averaging)");
@@ -381,6 +414,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     else if (!strcmp(key, "window_lines")) *value = s->window_lines;
     else if (!strcmp(key, "window_workers")) *value = s->window_workers;
     else if (!strcmp(key, "variant")) *value = s->variant;
+    else if (!strcmp(key, "P")) *value = s->cand_mult;
     else if (!strcmp(key, "window_red_rows")) *value = s->window_red_rows;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
@@ -403,9 +437,11 @@ int sk_hash(const sk_state* s, uint32_t row, uint64_t i0, uint64_t count, uint32
 uint64_t sk_algorithmic_bytes(const sk_state* s) {
     if (!s) return 0;
     const uint64_t n = s->P.n, d = s->P.d, r = s->P.r, c = s->P.c, k = s->P.k;
+    // second round: per candidate, its index, the n workers' values (and vhat) in, its exact value out
+    const uint64_t second = s->cand_mult > 1 ? (uint64_t)s->cand_mult * k * (4 * n + (s->variant == 1 ? 8 : 12)) : 0;
     if (s->variant == 1)     // Algorithm 1: read g,m,v,vhat,e and write m,v,vhat,e; no master-side second moments
-        return 36 * n * d + 8 * n * r * c + 4 * r * c + 8 * n * k + 8 * k;
-    return 20 * n * d + 4 * d + 8 * n * r * c + 4 * r * c + 12 * n * k + 24 * k;
+        return 36 * n * d + 8 * n * r * c + 4 * r * c + 8 * n * k + 8 * k + second;
+    return 20 * n * d + 4 * d + 8 * n * r * c + 4 * r * c + 12 * n * k + 24 * k + second;
 }
 
 int sk_get_timing(sk_state* s, double* ms, uint64_t* launches) {

@@ -67,8 +67,12 @@ int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStre
 int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum, uint32_t* keys, uint32_t* hist,
                          bool vec, int sm_count, cudaStream_t st);
 int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cudaStream_t st);
-int launch_emit(const Params& P, const uint32_t* keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2,
-                int sm_count, cudaStream_t st);
+// selection runs over P.d keys for the P.k largest; idx_map != nullptr: key t belongs to coordinate idx_map[t]
+int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, Select* sel, uint32_t* I_out, Cand* cand,
+                uint32_t* hist2, int sm_count, cudaStream_t st);
+// second round: exact values of `count` candidate coordinates as ranking keys, with their first-level histogram
+int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const float* vhat, const float* e,
+                      uint32_t* keys2, uint32_t* hist, int sm_count, cudaStream_t st);
 int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
                   int sm_count, cudaStream_t st);
 // vhat == nullptr: parameter averaging, the update is the plain mean (Algorithm 1)

@@ -251,7 +251,9 @@ __device__ __forceinline__ void block_append(uint32_t n_a, uint32_t n_b, uint32_
 // 12 key bits ---------------------------------------------------------------------------------------------------
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
-k_emit(uint32_t d, const uint32_t* __restrict__ keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2) {
+k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx_map, Select* sel, uint32_t* I_out,
+       Cand* cand, uint32_t* hist2) {
+    // idx_map (scalar form only): keys[t] belongs to coordinate idx_map[t] instead of t (second round on a candidate list)
     __shared__ uint32_t sh2[kHistBins];
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh2[b] = 0;
     __syncthreads();
@@ -293,7 +295,7 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, Select* sel, uint32_t* I_o
 #pragma unroll
         for (uint32_t u = 0; u < U; ++u) {
             const uint32_t t = t0 + u * kThreads;
-            const uint32_t idx0 = VEC ? (t << 2) : t;
+            const uint32_t idx0 = VEC ? (t << 2) : ((idx_map && nk[u]) ? idx_map[t] : t);
 #pragma unroll
             for (uint32_t q = 0; q < 4; ++q)
                 if (q < nk[u]) {
@@ -404,6 +406,29 @@ __global__ void __launch_bounds__(1024) k_resolve(uint32_t k, Select* sel, const
     }
 }
 
+// ---- second round (Section III-A): exact value of every candidate, as a ranking key, + first-level histogram ----
+// candidates C (P*k coordinates by estimate): key2[q] = bits(| mean_w a^(w)_j / sqrt(vhat_j) |), j = C[q]
+// (vhat == nullptr: parameter averaging, the exact value is the plain mean).
+__global__ void __launch_bounds__(kThreads)
+k_exact_keys(const __grid_constant__ Params P, const uint32_t* __restrict__ C, uint32_t count,
+             const float* __restrict__ vhat, const float* __restrict__ e, uint32_t* keys2, uint32_t* hist) {
+    __shared__ uint32_t sh[kHistBins];
+    for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh[b] = 0;
+    __syncthreads();
+    for (uint32_t q = blockIdx.x * kThreads + threadIdx.x; q < count; q += gridDim.x * kThreads) {
+        const uint32_t j = C[q];
+        float abar = 0.0f;
+        for (uint32_t w = 0; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
+        abar = abar / (float)P.n;
+        const uint32_t key = key_of(vhat ? scale_est(abar, vhat[j]) : abar);
+        keys2[q] = key;
+        atomicAdd(&sh[key >> kHistShift], 1u);
+    }
+    __syncthreads();
+    for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
+        if (sh[b]) atomicAdd(&hist[b], sh[b]);
+}
+
 // ---- apply on I_t: x_j -= lr * mean_w a^(w)_j / sqrt(vhat_j).  The error-feedback reset e^(w)_j = 0 is recorded
 // as a bit in the membership bitmap of I_t, which the next step's moment kernel honours. -----------------------
 __global__ void __launch_bounds__(kThreads)
@@ -484,10 +509,18 @@ int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cud
     return 1;
 }
 
-int launch_emit(const Params& P, const uint32_t* keys, Select* sel, uint32_t* I_out, Cand* cand, uint32_t* hist2,
-                int sm_count, cudaStream_t st) {
-    if (P.d % 4 == 0) k_emit<true><<<grid_for((P.d >> 2) / 4 + 1, sm_count, 8), kThreads, 0, st>>>(P.d, keys, sel, I_out, cand, hist2);
-    else k_emit<false><<<grid_for(P.d, sm_count, 8), kThreads, 0, st>>>(P.d, keys, sel, I_out, cand, hist2);
+int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, Select* sel, uint32_t* I_out, Cand* cand,
+                uint32_t* hist2, int sm_count, cudaStream_t st) {
+    if (P.d % 4 == 0 && !idx_map)
+        k_emit<true><<<grid_for((P.d >> 2) / 4 + 1, sm_count, 8), kThreads, 0, st>>>(P.d, keys, nullptr, sel, I_out, cand, hist2);
+    else
+        k_emit<false><<<grid_for(P.d, sm_count, 8), kThreads, 0, st>>>(P.d, keys, idx_map, sel, I_out, cand, hist2);
+    return 1;
+}
+
+int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const float* vhat, const float* e,
+                      uint32_t* keys2, uint32_t* hist, int sm_count, cudaStream_t st) {
+    k_exact_keys<<<grid_for(count, sm_count, 8), kThreads, 0, st>>>(P, C, count, vhat, e, keys2, hist);
     return 1;
 }
 

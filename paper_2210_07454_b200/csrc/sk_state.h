@@ -16,6 +16,8 @@ struct sk_state {
     size_t l2_bytes = 0;
     int64_t worker_chunk = 0;
     int64_t window_lines = 0;
+    int64_t cand_mult = 1;        // P of Section III-A: candidates of the second round = P * k (1 = no second round)
+    uint32_t *Ic = nullptr, *keys2 = nullptr;   // the P*k candidates and their exact-value keys
     int64_t variant = 0;          // 0 = gradient averaging (Algorithm 2), 1 = parameter averaging (Algorithm 1)
     float *vw = nullptr, *vhatw = nullptr;   // per-worker v, vhat of the parameter-averaging variant (n*d each)
     int64_t window_workers = 4;

@@ -65,6 +65,7 @@ extern "C" int sk_select_static(sk_state* s, uint32_t* idx_out) {
         return sk_fail_message(SK_EINVAL, msg);
     }
     if (s->t == 0) return sk_fail_message(SK_ESTATE, "sk_select_static: no step has been taken yet");
+    if (s->cand_mult > 1) return sk_fail_message(SK_ESTATE, "sk_select_static: not available with a second round (P > 1)");
     char msg[200];
     unsigned char* base = nullptr;
     int rc = scratch_for_device(&base, msg, sizeof msg);
@@ -86,7 +87,7 @@ extern "C" int sk_select_static(sk_state* s, uint32_t* idx_out) {
     A.variant = (uint32_t)s->variant;
     sk::launch_unsketch_hist(P, A, s->sum, keys, hist, vec, s->sm_count, st);
     sk::launch_pick_bin(P, hist, sel, 0, st);
-    sk::launch_emit(P, keys, sel, idx_out, cand, hist2, s->sm_count, st);
+    sk::launch_emit(P, keys, nullptr, sel, idx_out, cand, hist2, s->sm_count, st);
     sk::launch_refine(P, sel, cand, cand2, hist2, idx_out, s->sm_count, st);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) {

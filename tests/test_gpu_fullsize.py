@@ -14,15 +14,15 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 
-def _setup(name, window_lines=None, variant="ga"):
+def _setup(name, window_lines=None, variant="ga", P=1):
     from paper_2210_07454_b200 import binding, synthetic
     w = synthetic.WORKLOADS[name]
     src = synthetic.GradientSource(w, device="cuda")
     gpu = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                                  eps=w.eps, window_lines=window_lines, variant=variant)
+                                  eps=w.eps, window_lines=window_lines, variant=variant, P=P)
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=gpu.get_option("log2g"), lr=w.lr,
                         beta1=w.beta1, beta2=w.beta2, eps=w.eps, threads=32,
-                        window_lines=gpu.get_option("window_lines"), variant=variant)
+                        window_lines=gpu.get_option("window_lines"), variant=variant, P=P)
     return w, src, gpu, ora
 
 
@@ -33,8 +33,13 @@ def _one_step(w, src, gpu, ora, t, x_gpu, x_ref, variant="ga"):
     gpu.step(g, x_gpu)
     gpu.sync()
     del g
+    exact = None
+    if ora.P > 1:          # gradient averaging only: what the second round ranks by, mean_w(m_t + e_{t-1}) / sqrt(vhat_t)
+        e_sum = ora.field("e").astype(np.float64).sum(axis=0)
     ora.step(g_host, x_ref)
-    return compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, variant=variant)
+    if ora.P > 1:
+        exact = (ora.field("m").astype(np.float64).sum(axis=0) + e_sum) / w.n / np.sqrt(ora.field("vhat").astype(np.float64))
+    return compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, variant=variant, exact_ref=exact)
 
 
 @pytest.mark.parametrize("name", ["C2", "C3"])
@@ -63,6 +68,16 @@ def test_c3_parameter_averaging_two_teacher_forced_steps():
     force_state(gpu, ora, "pa")
     x_gpu.copy_(torch.from_numpy(x_ref))
     _one_step(w, src, gpu, ora, 2, x_gpu, x_ref, variant="pa")
+
+
+def test_c3_second_round_two_teacher_forced_steps():
+    w, src, gpu, ora = _setup("C3", P=4)           # the candidate multiplier the paper's experiments use
+    x_gpu = src.x0()
+    x_ref = x_gpu.cpu().numpy().copy()
+    _one_step(w, src, gpu, ora, 1, x_gpu, x_ref)
+    force_state(gpu, ora)
+    x_gpu.copy_(torch.from_numpy(x_ref))
+    _one_step(w, src, gpu, ora, 2, x_gpu, x_ref)
 
 
 @pytest.mark.parametrize("name", ["C4", "C5"])

@@ -28,13 +28,13 @@ def _workload(base, **over):
     return w
 
 
-def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga"):
+def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga", P=1):
     b = _binding()
     gpu = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                            eps=w.eps, log2g=log2g, window_lines=window_lines, variant=variant)
+                            eps=w.eps, log2g=log2g, window_lines=window_lines, variant=variant, P=P)
     lg = gpu.get_option("log2g")
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=lg, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                        eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"), variant=variant)
+                        eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"), variant=variant, P=P)
     return gpu, ora
 
 
@@ -62,8 +62,19 @@ def test_hash_bit_exact(log2g, c):
 
 
 # ------------------------------------------------------------------------------------------------ steps
-def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True, window_lines=None, variant="ga"):
-    gpu, ora = _pair(w, log2g, window_lines=window_lines, variant=variant)
+def _exact_values(ora, e_before, variant):
+    """What the second round ranks by: the preconditioned mean over the workers of a_t = (this step's m, scaled for
+    Algorithm 1) + e_{t-1}, recomputed here from the oracle's state around the step."""
+    if variant == "pa":
+        a = ora.field("m").astype(np.float64) / np.sqrt(ora.field("vhatw").astype(np.float64)) + e_before
+        return a.mean(axis=0)
+    a = ora.field("m").astype(np.float64) + e_before
+    return a.mean(axis=0) / np.sqrt(ora.field("vhat").astype(np.float64))
+
+
+def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True, window_lines=None, variant="ga",
+               P=1):
+    gpu, ora = _pair(w, log2g, window_lines=window_lines, variant=variant, P=P)
     src = _source(w, cfg_id=cfg_id)
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
@@ -78,9 +89,11 @@ def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=Tru
         x_gpu_before = x_gpu.cpu().numpy().copy()
         gpu.step(g, x_gpu)
         gpu.sync()
+        e_before = ora.field("e").astype(np.float64) if P > 1 else None
         ora.step(g_host, x_ref)
         diff = compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, check_tables=check_tables,
-                            x_gpu_before=x_gpu_before, variant=variant)
+                            x_gpu_before=x_gpu_before, variant=variant,
+                            exact_ref=_exact_values(ora, e_before, variant) if P > 1 else None)
         if diff.size and diverged_at is None:
             diverged_at = t
             if not teacher:
@@ -238,6 +251,68 @@ def test_pa_state_fields_and_errors():
     with pytest.raises(b.SkError):
         pa.set_option("variant", 0)                   # fixed after the first step
     assert pa.algorithmic_bytes() == 36 * 2 * 1000 + 8 * 2 * 3 * 256 + 4 * 3 * 256 + 8 * 2 * 10 + 8 * 10
+
+
+# ------------------------------------------------------------- second round of the selection (Section III-A, P > 1)
+@pytest.mark.parametrize("P", [2, 4])
+def test_second_round_c1_ten_steps_teacher_forced(P):
+    _run_steps(_workload("C1"), 10, P=P)
+
+
+SECOND_ROUND = {
+    "scalar_path": dict(d=10_007, n=3, r=5, c=1000, k=333, P=3),
+    "candidates_are_everything": dict(d=4096, n=2, r=3, c=512, k=1024, P=4),       # P*k = d
+    "k_1": dict(d=20_000, n=4, r=5, c=1024, k=1, P=8),
+    "tiny_sketch_many_candidates": dict(d=50_000, n=4, r=3, c=256, k=500, P=16),   # estimates nearly useless
+    "pa": dict(d=30_000, n=3, r=5, c=2048, k=300, P=2, variant="pa"),
+    "windowed_family": dict(d=40_000, n=6, r=5, c=4096, k=400, P=2, L=8),
+}
+
+
+@pytest.mark.parametrize("case", sorted(SECOND_ROUND))
+def test_second_round_edge_cases(case):
+    cfg = dict(SECOND_ROUND[case])
+    P, L, variant = cfg.pop("P"), cfg.pop("L", None), cfg.pop("variant", "ga")
+    w = _workload("C1", name="E", steps=3, recipe="planted", **cfg)
+    _run_steps(w, 3, cfg_id=7, variant=variant, window_lines=L, P=P)
+
+
+def test_second_round_integer_inputs_are_bit_exact():
+    # integer gradients, beta1 = 0 and eps = 1: estimates and exact values are exact small rationals with ties
+    # everywhere, so the candidates and the final set must match the oracle index for index
+    d, n, r, c, k, P = 100_000, 4, 5, 2048, 500, 4
+    b = _binding()
+    gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0, P=P)
+    ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=gpu.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
+                        threads=8, P=P)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    x = torch.zeros(d, device="cuda")
+    x_ref = np.zeros(d, np.float32)
+    g = torch.randint(-8, 9, (n, d), generator=gen, device="cuda").float()
+    gpu.step(g, x)
+    gpu.sync()
+    ora.step(g.cpu().numpy(), x_ref)
+    assert np.array_equal(gpu.get("cand"), ora.field("cand"))
+    assert np.array_equal(gpu.get("I"), ora.field("I"))
+    assert np.array_equal(gpu.get("e"), ora.field("e"))
+    assert np.array_equal(x.cpu().numpy(), x_ref)
+
+
+def test_second_round_option_errors():
+    b = _binding()
+    with pytest.raises(b.SkError):
+        b.SketchedAMSGrad(1000, 2, 3, 256, 400, P=3)          # P*k > d
+    with pytest.raises(b.SkError):
+        b.SketchedAMSGrad(1000, 2, 3, 256, 10, P=0)
+    gpu = b.SketchedAMSGrad(1000, 2, 3, 256, 10, P=2)
+    assert gpu.get_option("P") == 2 and gpu.get("cand").size == 0
+    x = torch.zeros(1000, device="cuda")
+    gpu.step(torch.ones((2, 1000), device="cuda"), x)
+    assert gpu.get("cand").size == 20
+    with pytest.raises(b.SkError):
+        gpu.set_option("P", 1)                                # fixed after the first step
+    with pytest.raises(b.SkError):
+        gpu.select_static(torch.empty(10, dtype=torch.int32, device="cuda"))
 
 
 def test_worker_chunking_matches_single_pass():
