@@ -125,6 +125,10 @@ int do_step(sk_state* s, const float* grads, float* x) {
     A.vw = s->vw; A.vhatw = s->vhatw; A.variant = (uint32_t)s->variant;
     const bool windowed = vec && P.win_cw != 0 && s->variant == 0;   // the windowed kernel implements Algorithm 2 only
     const uint32_t wc = windowed ? std::min<uint32_t>((uint32_t)s->window_workers, P.n) : chunk_of(s);
+    // With a second round the sketch kernel also leaves sum_w a^(w) per coordinate, so that each of the P*k exact
+    // values costs one gather instead of n (the windowed kernel does not: there every worker's value is gathered).
+    A.asum = (s->cand_mult > 1 && !windowed) ? s->asum : nullptr;
+    const float* asum = A.asum;
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
         const uint32_t nw = std::min(wc, P.n - w0);
@@ -173,7 +177,7 @@ int do_step(sk_state* s, const float* grads, float* x) {
         }
         StageTimer tm(s, 6);
         int l = sk::launch_refine(Q, s->sel, s->cand, s->cand2, s->hist2, s->Ic, s->sm_count, st);
-        l += sk::launch_exact_keys(P, s->Ic, Q.k, s->variant == 1 ? nullptr : s->vhat, s->e, s->keys2, s->hist,
+        l += sk::launch_exact_keys(P, s->Ic, Q.k, s->variant == 1 ? nullptr : s->vhat, s->e, asum, s->keys2, s->hist,
                                    s->sm_count, st);
         sk::Params Q2 = P;                      // second selection: k of the P*k candidates, keyed by exact value
         Q2.d = Q.k;
@@ -185,7 +189,7 @@ int do_step(sk_state* s, const float* grads, float* x) {
     {
         StageTimer tm(s, 7);     // the bitmap of I_{t-1} has served its purpose: clear it, then apply marks I_t
         int l = sk::launch_zero(s->bitmap, s->bitmap_bytes, st);
-        l += sk::launch_apply(P, s->I, s->variant == 1 ? nullptr : s->vhat, s->e, x, s->bitmap, st);
+        l += sk::launch_apply(P, s->I, s->variant == 1 ? nullptr : s->vhat, s->e, asum, x, s->bitmap, st);
         tm.done(l);
     }
     SK_CUDA(cudaGetLastError());
@@ -287,7 +291,7 @@ void sk_destroy(sk_state* s) {
     if (s->stream) cudaStreamSynchronize(s->stream); else cudaDeviceSynchronize();
     for (void* p : {(void*)s->m, (void*)s->e, (void*)s->v, (void*)s->vhat, (void*)s->vstamp, (void*)s->tables,
                     (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->hist2, (void*)s->sel, (void*)s->cand, (void*)s->cand2,
-                    (void*)s->keys, (void*)s->gsum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw, (void*)s->Ic, (void*)s->keys2,
+                    (void*)s->keys, (void*)s->gsum, (void*)s->asum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw, (void*)s->Ic, (void*)s->keys2,
                     (void*)s->stage_grads, (void*)s->stage_x})
         if (p) cudaFree(p);
     for (const TimeRec& r : s->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -354,9 +358,10 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         if (s->t != 0) return fail(SK_ESTATE, "P can only be changed before the first step");
         if (value < 1 || (uint64_t)value * s->P.k > s->P.d) return fail(SK_EINVAL, "P must be >= 1 with P*k <= d");
         if (value > 1) {
-            if (s->Ic) { cudaFree(s->Ic); cudaFree(s->keys2); s->Ic = s->keys2 = nullptr; }
+            if (s->Ic) { cudaFree(s->Ic); cudaFree(s->keys2); cudaFree(s->asum); s->Ic = s->keys2 = nullptr; s->asum = nullptr; }
             const uint64_t pk = (uint64_t)value * s->P.k;
-            if (cudaMalloc((void**)&s->Ic, pk * 4) != cudaSuccess || cudaMalloc((void**)&s->keys2, pk * 4) != cudaSuccess)
+            if (cudaMalloc((void**)&s->Ic, pk * 4) != cudaSuccess || cudaMalloc((void**)&s->keys2, pk * 4) != cudaSuccess ||
+                cudaMalloc((void**)&s->asum, ((uint64_t)s->P.d + 3) / 4 * 16) != cudaSuccess)
                 return fail(SK_ENOMEM, "cudaMalloc of the candidate buffers failed: %s", cudaGetErrorString(cudaGetLastError()));
         }
         s->cand_mult = value;

@@ -41,6 +41,7 @@ struct Cand { uint32_t key, idx; };
 struct MomentArgs {
     const float* grads;
     float *m, *e, *tables;
+    float* asum;             // d or nullptr: running sum over the workers of a_t, in worker order (second round of Section III-A)
     float* gsum;             // running gradient sums on I_{t-1} when the workers are processed in several launches
     float *v, *vhat;
     uint32_t* vstamp;        // step at which v[j] was last brought up to date
@@ -71,12 +72,15 @@ int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cud
 int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, Select* sel, uint32_t* I_out, Cand* cand,
                 uint32_t* hist2, int sm_count, cudaStream_t st);
 // second round: exact values of `count` candidate coordinates as ranking keys, with their first-level histogram
+// asum != nullptr: sum_w a^(w) per coordinate is read from there instead of gathering e for every worker
 int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const float* vhat, const float* e,
+                      const float* asum,
                       uint32_t* keys2, uint32_t* hist, int sm_count, cudaStream_t st);
 int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
                   int sm_count, cudaStream_t st);
 // vhat == nullptr: parameter averaging, the update is the plain mean (Algorithm 1)
-int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, float* x, uint32_t* bitmap,
+int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, const float* asum, float* x,
+                 uint32_t* bitmap,
                  cudaStream_t st);
 // helpers for state export / import
 int launch_estimates(const Params& P, const float* sum, const float* vhat, float* est, cudaStream_t st);

@@ -411,14 +411,16 @@ __global__ void __launch_bounds__(1024) k_resolve(uint32_t k, Select* sel, const
 // (vhat == nullptr: parameter averaging, the exact value is the plain mean).
 __global__ void __launch_bounds__(kThreads)
 k_exact_keys(const __grid_constant__ Params P, const uint32_t* __restrict__ C, uint32_t count,
-             const float* __restrict__ vhat, const float* __restrict__ e, uint32_t* keys2, uint32_t* hist) {
+             const float* __restrict__ vhat, const float* __restrict__ e, const float* __restrict__ asum,
+             uint32_t* keys2, uint32_t* hist) {
     __shared__ uint32_t sh[kHistBins];
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh[b] = 0;
     __syncthreads();
     for (uint32_t q = blockIdx.x * kThreads + threadIdx.x; q < count; q += gridDim.x * kThreads) {
         const uint32_t j = C[q];
         float abar = 0.0f;
-        for (uint32_t w = 0; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
+        if (asum) abar = asum[j];
+        else for (uint32_t w = 0; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
         abar = abar / (float)P.n;
         const uint32_t key = key_of(vhat ? scale_est(abar, vhat[j]) : abar);
         keys2[q] = key;
@@ -433,12 +435,14 @@ k_exact_keys(const __grid_constant__ Params P, const uint32_t* __restrict__ C, u
 // as a bit in the membership bitmap of I_t, which the next step's moment kernel honours. -----------------------
 __global__ void __launch_bounds__(kThreads)
 k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const float* __restrict__ vhat,
-        const float* __restrict__ e, float* x, uint32_t* bitmap) {
+        const float* __restrict__ e, const float* __restrict__ asum, float* x, uint32_t* bitmap) {
+    // asum != nullptr: the sketch kernel left sum_w a^(w) (added in worker order) there, one gather instead of n
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
     if (q >= P.k) return;
     const uint32_t j = I[q];
     float abar = 0.0f;
-    uint32_t w = 0;
+    uint32_t w = asum ? P.n : 0;
+    if (asum) abar = asum[j];
     for (; w + 8 <= P.n; w += 8) {                           // eight independent gathers in flight, added in order
         float a[8];
 #pragma unroll
@@ -519,8 +523,8 @@ int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, 
 }
 
 int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const float* vhat, const float* e,
-                      uint32_t* keys2, uint32_t* hist, int sm_count, cudaStream_t st) {
-    k_exact_keys<<<grid_for(count, sm_count, 8), kThreads, 0, st>>>(P, C, count, vhat, e, keys2, hist);
+                      const float* asum, uint32_t* keys2, uint32_t* hist, int sm_count, cudaStream_t st) {
+    k_exact_keys<<<grid_for(count, sm_count, 8), kThreads, 0, st>>>(P, C, count, vhat, e, asum, keys2, hist);
     return 1;
 }
 
@@ -532,9 +536,9 @@ int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, u
     return 3;
 }
 
-int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, float* x, uint32_t* bitmap,
-                 cudaStream_t st) {
-    k_apply<<<(P.k + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, I, vhat, e, x, bitmap);
+int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, const float* asum, float* x,
+                 uint32_t* bitmap, cudaStream_t st) {
+    k_apply<<<(P.k + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, I, vhat, e, asum, x, bitmap);
     return 1;
 }
 

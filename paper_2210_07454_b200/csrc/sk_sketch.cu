@@ -80,6 +80,8 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
         const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
         float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);     // running gradient sum in worker order (used on I_{t-1})
         if (mask && w0 > 0) gs = ((const float4*)A.gsum)[t];
+        float4 as = make_float4(0.f, 0.f, 0.f, 0.f);     // running sum of a in worker order: the exact values of
+        if (A.asum && w0 > 0) as = ((const float4*)A.asum)[t];   // Section III-A's second round reads them from it
         uint32_t w = w0;
         const uint32_t wend = w0 + nw;
         for (; w + 2 <= wend; w += 2) {                  // two workers per trip: six 16-byte loads in flight
@@ -91,6 +93,8 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             SK_MOMENT(m1, a1, g1, mask)
             gs.x = (gs.x + g0.x) + g1.x; gs.y = (gs.y + g0.y) + g1.y;
             gs.z = (gs.z + g0.z) + g1.z; gs.w = (gs.w + g0.w) + g1.w;
+            as.x = (as.x + a0.x) + a1.x; as.y = (as.y + a0.y) + a1.y;
+            as.z = (as.z + a0.z) + a1.z; as.w = (as.w + a0.w) + a1.w;
             __stcs(m + q0, m0); __stcs(m + q1, m1);
             __stcs(e + q0, a0); __stcs(e + q1, a1);
             float* t0 = A.tables + (uint64_t)w * tstride;
@@ -109,6 +113,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             float4 a0 = __ldcs(e + q0);
             SK_MOMENT(m0, a0, g0, mask)
             gs.x += g0.x; gs.y += g0.y; gs.z += g0.z; gs.w += g0.w;
+            as.x += a0.x; as.y += a0.y; as.z += a0.z; as.w += a0.w;
             __stcs(m + q0, m0);
             __stcs(e + q0, a0);
             float* t0 = A.tables + (uint64_t)w * tstride;
@@ -117,6 +122,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
                 if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
         }
         if (mask) ((float4*)A.gsum)[t] = gs;             // consumed by the key pass (or by the next launch)
+        if (A.asum) ((float4*)A.asum)[t] = as;
     }
 }
 
@@ -151,6 +157,8 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
         quad_hashes<RMAX>(P, r, t < d4 ? t : d4 - 1, h);
         if (t >= d4) continue;
         const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
+        float4 as = make_float4(0.f, 0.f, 0.f, 0.f);     // running sum of a in worker order
+        if (A.asum && w0 > 0) as = ((const float4*)A.asum)[t];
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q0 = (uint64_t)w * d4 + t;
             const float4 g0 = __ldcs(grads + q0);
@@ -164,7 +172,9 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
 #pragma unroll
             for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
                 if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+            as.x += a0.x; as.y += a0.y; as.z += a0.z; as.w += a0.w;
         }
+        if (A.asum) ((float4*)A.asum)[t] = as;
     }
 }
 
@@ -176,6 +186,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
     for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads) {
         const bool member = A.members && ((A.bitmap[j >> 5] >> (j & 31u)) & 1u);
         float gs = (member && w0 > 0) ? A.gsum[j] : 0.0f;
+        float as = (A.asum && w0 > 0) ? A.asum[j] : 0.0f;
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q = (uint64_t)w * P.d + j;
             const float g = A.grads[q];
@@ -190,6 +201,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
                 a = mm + (member ? 0.0f : A.e[q]);
             }
             gs += g;
+            as += a;
             A.m[q] = mm;
             A.e[q] = a;
             for (uint32_t row = 0; row < P.r; ++row) {
@@ -199,6 +211,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
             }
         }
         if (member && A.variant == 0) A.gsum[j] = gs;
+        if (A.asum) A.asum[j] = as;
     }
 }
 

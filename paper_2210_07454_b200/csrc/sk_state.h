@@ -30,6 +30,7 @@ struct sk_state {
     uint32_t *vstamp = nullptr, *I = nullptr, *I_prev = nullptr, *hist = nullptr, *hist2 = nullptr;
     uint32_t *keys = nullptr, *bitmap = nullptr;
     float* gsum = nullptr;
+    float* asum = nullptr;        // d, only with a second round: sum over the workers of a_t (worker order), written by the sketch kernel
     uint64_t bitmap_bytes = 0;
     sk::Select* sel = nullptr;
     sk::Cand *cand = nullptr, *cand2 = nullptr;

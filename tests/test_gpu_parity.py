@@ -277,7 +277,8 @@ def test_second_round_edge_cases(case):
     _run_steps(w, 3, cfg_id=7, variant=variant, window_lines=L, P=P)
 
 
-def test_second_round_integer_inputs_are_bit_exact():
+@pytest.mark.parametrize("chunk", [0, 1, 3])
+def test_second_round_integer_inputs_are_bit_exact(chunk):
     # integer gradients, beta1 = 0 and eps = 1: estimates and exact values are exact small rationals with ties
     # everywhere, so the candidates and the final set must match the oracle index for index
     d, n, r, c, k, P = 100_000, 4, 5, 2048, 500, 4
@@ -285,6 +286,7 @@ def test_second_round_integer_inputs_are_bit_exact():
     gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0, P=P)
     ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=gpu.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
                         threads=8, P=P)
+    gpu.set_option("worker_chunk", chunk)            # workers in several launches: the running sums carry over
     gen = torch.Generator(device="cuda").manual_seed(5)
     x = torch.zeros(d, device="cuda")
     x_ref = np.zeros(d, np.float32)
