@@ -183,6 +183,9 @@ def main():
     ap.add_argument("--ref-scale", type=int, default=16)
     ap.add_argument("--scale", type=int, default=1, help="run the workload at 1/SCALE size (profiling captures)")
     ap.add_argument("--grad-sets", type=int, default=0, help="rotating gradient sets (0 = as many as fit, 2..4)")
+    ap.add_argument("--partition-workers", action="store_true",
+                    help="split the workload's n workers over the processes (one step = three phases with two "
+                         "all-reduces between them) instead of running one full replica per process")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-timing", action="store_true")
     args = ap.parse_args()
@@ -206,10 +209,18 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    src = synthetic.GradientSource(w, device=dev, cfg_id=cfg_id)
+    n_all = w.n
+    if args.partition_workers:                       # this process holds n / world of the workers; x is replicated
+        assert w.n % world == 0, f"--partition-workers needs the workers ({w.n}) to divide by the processes ({world})"
+        w = synthetic.Workload(**{**w.__dict__, "n": w.n // world})
+    src = synthetic.GradientSource(w, device=dev, cfg_id=cfg_id + (100 * rank if args.partition_workers else 0))
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
                                   eps=w.eps, log2g=args.log2g, window_lines=args.window_lines, variant=args.variant,
-                                  P=args.P)
+                                  P=args.P, workers_total=n_all if args.partition_workers else None)
+    step = opt.step
+    if args.partition_workers:
+        from paper_2210_07454_b200.partitioned import PartitionedStep
+        step = PartitionedStep(opt, dev).step
     opt.set_option("worker_chunk", args.worker_chunk)
     if args.window_workers:
         opt.set_option("window_workers", args.window_workers)
@@ -229,7 +240,7 @@ def main():
     if rank == 0:
         sampler.start()                              # started early: nvidia-smi takes a while to deliver samples
     for t in range(args.warmup):
-        opt.step(gsets[t % nsets], x)
+        step(gsets[t % nsets], x)
     opt.sync()
     opt.timing()                                     # clear launch counters
     opt.set_option("timing", 0 if args.no_stage_timing else 1)
@@ -240,7 +251,7 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for t in range(args.steps):
-        opt.step(gsets[(args.warmup + t) % nsets], x)
+        step(gsets[(args.warmup + t) % nsets], x)
     ev1.record()
     torch.cuda.synchronize()
     if world > 1:
@@ -253,7 +264,8 @@ def main():
     launches = reduce_sum(float(sum(stage_launches)), world, dev)
 
     ms_step = ms_total / args.steps
-    value = world * w.n * w.d / (ms_step * 1e-3) / 1e9
+    units = n_all * w.d if args.partition_workers else world * w.n * w.d     # worker-coordinates per step, whole job
+    value = units / (ms_step * 1e-3) / 1e9
     peak, peak_kind = _peaks()
     b_alg = opt.algorithmic_bytes()
 
@@ -282,15 +294,25 @@ def main():
         hg.copy_(gsets[0])
         hx = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
         hx.copy_(x)
-        opt.step_host(hg, hx)                         # warm-up (allocates the staging buffers)
+        if args.partition_workers:                    # the phases take device buffers: stage through torch copies
+            gdev = gsets[0]
+
+            def step_host(hgrads, hxx):
+                gdev.copy_(hgrads, non_blocking=True)
+                x.copy_(hxx, non_blocking=True)
+                step(gdev, x)
+                hxx.copy_(x)
+        else:
+            step_host = opt.step_host
+        step_host(hg, hx)                             # warm-up (allocates the staging buffers)
         if world > 1:
             dist.barrier()
         t0 = time.perf_counter()
         for _ in range(args.e2e_steps):
-            opt.step_host(hg, hx)
+            step_host(hg, hx)
         torch.cuda.synchronize()
         dt = reduce_max(time.perf_counter() - t0, world, dev)
-        e2e = {"value": world * w.n * w.d * args.e2e_steps / dt / 1e9, "unit": UNIT,
+        e2e = {"value": units * args.e2e_steps / dt / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": 4 * w.n * w.d + 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
                "ms_per_step": 1e3 * dt / args.e2e_steps, "steps": args.e2e_steps}
 
@@ -305,12 +327,15 @@ def main():
                "kind": "oracle", "sample": sample}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong" if args.partition_workers else "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k,
+            "config": {"workload": w.name, "d": w.d, "n": n_all, "r": w.r, "c": w.c, "k": w.k,
                        "recipe": w.recipe, "variant": args.variant, "P": args.P, "hash_group": 1 << opt.get_option("log2g"),
                        "window_lines": opt.get_option("window_lines"),
-                       "worker_chunk": opt.get_option("worker_chunk"), "replicas": world,
+                       "worker_chunk": opt.get_option("worker_chunk"),
+                       "replicas": 1 if args.partition_workers else world,
+                       "workers_per_process": w.n, "partitioned": bool(args.partition_workers),
                        "l2": f"inputs larger than L2: {nsets} rotating gradient sets of {set_bytes / 1e9:.2f} GB"},
             "steps_per_s": 1e3 / ms_step,
             "step_roofline": {"algorithmic_bytes": b_alg, "achieved_gbs": b_alg / (ms_step * 1e-3) / 1e9,

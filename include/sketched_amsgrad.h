@@ -59,6 +59,34 @@ int sk_step(const float* grads, float* x, sk_state* state);
  * but is not required.  The staging buffers are allocated on first use and freed by sk_destroy. */
 int sk_step_host(const float* grads_host, float* x_host, sk_state* state);
 
+/* ---- One iteration with the WORKERS PARTITIONED over several processes (one GPU each) -----------------------------
+ * Every process creates a handle for its own n workers (same d, r, c, k, seed, hyper-parameters and options on all
+ * of them), sets the option "workers_total" to the number of workers over all processes, and keeps a replica of x.
+ * Algorithms 1 and 2 couple the workers only through sums, and those sums are what the processes exchange: per
+ * iteration the sketch, the gradient entries on I_{t-1} and the exact values of the candidates, i.e. the
+ * |S| + k + P*k floats of Section III-B (the update is applied by every replica, so it is not sent back).  An
+ * iteration is three calls with one sum over the processes (an all-reduce, done by the caller) between them:
+ *
+ *   sk_step_local (grads, exchange1, state)      moments, a_t and sketches of this process's workers
+ *   -- caller: exchange1 <- sum over processes of exchange1 --
+ *   sk_step_select(exchange1, exchange2, state)  second moments on I_{t-1}, unsketch, selection of the candidates
+ *   -- caller: exchange2 <- sum over processes of exchange2 --
+ *   sk_step_finish(exchange2, x, state)          second round (P > 1), update of x, new I_t
+ *
+ * exchange1: device, sk_exchange_floats(state, 1) floats, 16-byte aligned: this process's share of the mean sketch
+ *   (r rows of c floats, each row padded to a multiple of 32), then, for Algorithm 2, its gradient sums on I_{t-1}
+ *   in ascending index order, zero-padded to k.  exchange2: device, sk_exchange_floats(state, 2) = P*k floats: its
+ *   sums of a_t at the candidates in ascending index order.  Both are caller-owned; the library writes them in the
+ *   first call of each pair and reads the summed values in the second.  The sum must give every process the same
+ *   bits (NCCL's all-reduce does), since every process then takes the same selection from them.
+ * grads: this process's n*d gradients, as for sk_step.  All work is enqueued on the handle's stream; nothing
+ * synchronises.  Calls out of order return SK_ESTATE.  With one process the result equals sk_step's up to the
+ * rounding of the sums. */
+uint64_t sk_exchange_floats(const sk_state* state, int which /* 1 or 2 */);
+int sk_step_local(const float* grads, float* exchange1, sk_state* state);
+int sk_step_select(const float* exchange1, float* exchange2, sk_state* state);
+int sk_step_finish(const float* exchange2, float* x, sk_state* state);
+
 /* Releases everything sk_create and later calls allocated.  NULL is accepted. */
 void sk_destroy(sk_state* state);
 
@@ -70,10 +98,12 @@ int sk_sync(sk_state* state);
 /* Options (integers):
  *   "log2g"        hash group size g = 2^log2g, 0..5 (Section II-C fixes no hash family; see sk_hash).
  *                  Only before the first step.  Default: the largest value <= 5 with 2^log2g <= c.
- *   "P"            candidate multiplier of the second round (Section III-A, "In practice ..."): the P*k largest
+ *   "P"            candidate multiplier of the second round (Section III-A): the P*k largest
  *                  estimates become candidates, their exact values are fetched from the workers' vectors, and the
  *                  k candidates of largest exact magnitude form I_t (ties: smaller index).  1 (default) = no second
  *                  round.  P*k <= d.  Only before the first step.  The candidates of the last step are field "cand".
+ *   "workers_total" number of workers the means are taken over, >= n; default n.  Set it on every handle of a
+ *                  partitioned step (see sk_step_local) to the sum of their n.  Only before the first step.
  *   "variant"      0 (default) = gradient averaging, Algorithm 2; 1 = parameter averaging, Algorithm 1: every worker
  *                  keeps its own v and vhat (fields "vw", "vhatw", n*d each, initial value eps) from its own
  *                  gradient, sketches m/sqrt(vhat) + e, the unsketch takes no vhat and x moves by the plain mean

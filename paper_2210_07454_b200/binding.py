@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libsketched_amsgrad.so")
 
 EXPORTS = ["sk_create", "sk_step", "sk_step_host", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
            "sk_get_option", "sk_hash", "sk_get", "sk_set", "sk_algorithmic_bytes", "sk_get_timing", "sk_select_static",
-           "sk_last_error", "sk_version"]
+           "sk_exchange_floats", "sk_step_local", "sk_step_select", "sk_step_finish", "sk_last_error", "sk_version"]
 STATIC_MAX_D = 262144
 NUM_STAGES = 8
 STAGE_NAMES = ["zero_tables", "second_moment", "moment_sketch", "sum_tables", "unsketch_hist",
@@ -52,6 +52,10 @@ def lib() -> C.CDLL:
         L.sk_get_timing.restype = C.c_int
         L.sk_get_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u64)]
         L.sk_select_static.restype = C.c_int; L.sk_select_static.argtypes = [vp, vp]
+        L.sk_exchange_floats.restype = u64; L.sk_exchange_floats.argtypes = [vp, C.c_int]
+        L.sk_step_local.restype = C.c_int; L.sk_step_local.argtypes = [vp, vp, vp]
+        L.sk_step_select.restype = C.c_int; L.sk_step_select.argtypes = [vp, vp, vp]
+        L.sk_step_finish.restype = C.c_int; L.sk_step_finish.argtypes = [vp, vp, vp]
         L.sk_last_error.restype = C.c_char_p; L.sk_last_error.argtypes = []
         L.sk_version.restype = C.c_char_p; L.sk_version.argtypes = []
         _lib = L
@@ -83,7 +87,7 @@ class SketchedAMSGrad:
                      "vw": "nd", "vhatw": "nd"}
 
     def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None,
-                 window_lines=None, variant="ga", P=1):
+                 window_lines=None, variant="ga", P=1, workers_total=None):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
         self._h = lib().sk_create(d, n, r, c, k, seed, lr, beta1, beta2, eps)
         if not self._h:
@@ -99,6 +103,8 @@ class SketchedAMSGrad:
         self.P = P
         if P != 1:
             self.set_option("P", P)
+        if workers_total is not None:     # this handle holds n of the workers of a partitioned step
+            self.set_option("workers_total", workers_total)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -116,6 +122,19 @@ class SketchedAMSGrad:
     def step_host(self, grads, x) -> None:
         """Same step with host buffers (numpy arrays or CPU tensors, ideally pinned); x is updated in place."""
         _check(lib().sk_step_host(_ptr(grads), _ptr(x), self._h))
+
+    # -- one iteration in three phases, the workers partitioned over processes (see partitioned.py) ----
+    def exchange_floats(self, which: int) -> int:
+        return int(lib().sk_exchange_floats(self._h, which))
+
+    def step_local(self, grads, exchange1) -> None:
+        _check(lib().sk_step_local(_ptr(grads), _ptr(exchange1), self._h))
+
+    def step_select(self, exchange1, exchange2) -> None:
+        _check(lib().sk_step_select(_ptr(exchange1), _ptr(exchange2), self._h))
+
+    def step_finish(self, exchange2, x) -> None:
+        _check(lib().sk_step_finish(_ptr(exchange2), _ptr(x), self._h))
 
     # -- auxiliaries ------------------------------------------------------------------------------------
     def sync(self) -> None:

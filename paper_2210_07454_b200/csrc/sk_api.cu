@@ -111,25 +111,41 @@ int check_status(sk_state* s) {
     return SK_OK;
 }
 
-int do_step(sk_state* s, const float* grads, float* x) {
-    const sk::Params& P = s->P;
-    const bool vec = (P.d % 4 == 0) && P.log2g >= 2 && ((uintptr_t)grads % 16 == 0) && ((uintptr_t)x % 16 == 0);
-    cudaStream_t st = s->stream;
-    const uint32_t t = (uint32_t)(s->t + 1);
-    if (s->timing && s->recs.size() > 4096) { int rc = flush_timing(s); if (rc) return rc; }
-
+sk::MomentArgs moment_args(const sk_state* s, const float* grads) {
     sk::MomentArgs A{};
     A.grads = grads; A.m = s->m; A.e = s->e; A.tables = s->tables; A.gsum = s->gsum;
     A.v = s->v; A.vhat = s->vhat; A.vstamp = s->vstamp; A.bitmap = s->bitmap;
-    A.step = t; A.members = s->k_prev ? 1u : 0u;
+    A.step = (uint32_t)(s->t + 1); A.members = s->k_prev ? 1u : 0u;
     A.vw = s->vw; A.vhatw = s->vhatw; A.variant = (uint32_t)s->variant;
+    return A;
+}
+
+// One iteration is three phases.  sk_step runs them back to back.  With the workers partitioned over processes
+// (sk_step_local / sk_step_select / sk_step_finish) the caller sums an exchange buffer over the processes between
+// the phases: x1 = [this process's share of the mean sketch | its gradient sums on I_{t-1}], x2 = [its sums of a_t at
+// the candidates]; both index lists are in ascending order so that position q means the same coordinate everywhere.
+
+// Phase 1 (workers): moments, error-compensated vector, sketches of this handle's workers, their sum.
+int phase_local(sk_state* s, const float* grads, float* x1) {
+    const sk::Params& P = s->P;
+    const bool vec = s->step_vec;
+    const bool sharded = x1 != nullptr;
+    cudaStream_t st = s->stream;
+    if (s->timing && s->recs.size() > 4096) { int rc = flush_timing(s); if (rc) return rc; }
+
+    sk::MomentArgs A = moment_args(s, grads);
     const bool windowed = vec && P.win_cw != 0 && s->variant == 0;   // the windowed kernel implements Algorithm 2 only
     const uint32_t wc = windowed ? std::min<uint32_t>((uint32_t)s->window_workers, P.n) : chunk_of(s);
     // With a second round the sketch kernel also leaves sum_w a^(w) per coordinate, so that each of the P*k exact
-    // values costs one gather instead of n (the windowed kernel does not: there every worker's value is gathered).
-    A.asum = (s->cand_mult > 1 && !windowed) ? s->asum : nullptr;
-    const float* asum = A.asum;
+    // values costs one gather instead of n (not the windowed kernel, and not a partitioned step, whose exact values
+    // are exchanged: there every local worker's value is gathered).
+    A.asum = (s->cand_mult > 1 && !windowed && !sharded) ? s->asum : nullptr;
+    s->asum_live = A.asum != nullptr;
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
+    if (sharded && s->k_prev) {      // I_{t-1} in ascending order, from its bitmap
+        StageTimer tm(s, 0);
+        tm.done(sk::launch_list_from_bitmap(s->bitmap, s->bitmap_bytes / 4, s->scan, s->I_prev, st));
+    }
     for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
         const uint32_t nw = std::min(wc, P.n - w0);
         {
@@ -148,39 +164,75 @@ int do_step(sk_state* s, const float* grads, float* x) {
     }
     {
         StageTimer tm(s, 3);
-        tm.done(sk::launch_sum_tables(P, s->tables, s->sum, st));
+        int l = sk::launch_sum_tables(P, s->tables, sharded ? x1 : s->sum, st);
+        if (sharded && s->variant == 0)      // h_t: this process's gradient sums on I_{t-1}, zero-padded to k
+            l += sk::launch_gather(s->I_prev, s->k_prev, P.k, s->gsum, x1 + tfloats, st);
+        tm.done(l);
     }
+    SK_CUDA(cudaGetLastError());
+    return SK_OK;
+}
+
+// Phase 2 (master): second moments on I_{t-1}, unsketch of every coordinate, selection of the candidates.
+int phase_select(sk_state* s, const float* x1, float* x2) {
+    const sk::Params& P = s->P;
+    const bool vec = s->step_vec;
+    const bool sharded = x1 != nullptr;
+    cudaStream_t st = s->stream;
+    sk::MomentArgs A = moment_args(s, nullptr);
+    sk::Params Q = P;                           // first selection: P*k of d (k without a second round)
+    Q.k = (uint32_t)s->cand_mult * P.k;
     {
         StageTimer tm(s, 4);
+        int l = 0;
+        if (sharded) {                          // the summed exchange buffer: mean sketch, then gradient sums on I_{t-1}
+            SK_CUDA(cudaMemcpyAsync(s->sum, x1, (uint64_t)P.r * P.cs * 4, cudaMemcpyDeviceToDevice, st));
+            if (s->variant == 0) l += sk::launch_scatter(s->I_prev, s->k_prev, x1 + (uint64_t)P.r * P.cs, s->gsum, st);
+        }
         // ranking keys; v and vhat on I_{t-1} are brought up to date on the way, from the sums in gsum
-        int l = sk::launch_unsketch_hist(P, A, s->sum, s->keys, s->hist, vec, s->sm_count, st);
-        sk::Params Q = P;
-        Q.k = (uint32_t)s->cand_mult * P.k;         // with a second round the first selection takes P*k candidates
+        l += sk::launch_unsketch_hist(P, A, s->sum, s->keys, s->hist, vec, s->sm_count, st);
         l += sk::launch_pick_bin(Q, s->hist, s->sel, 0, st);
         tm.done(l);
     }
-    if (s->cand_mult <= 1) {
-        {
-            StageTimer tm(s, 5);
-            tm.done(sk::launch_emit(P, s->keys, nullptr, s->sel, s->I, s->cand, s->hist2, s->sm_count, st));
-        }
+    uint32_t* list = s->cand_mult > 1 ? s->Ic : s->I;
+    {
+        StageTimer tm(s, 5);
+        tm.done(sk::launch_emit(Q, s->keys, nullptr, s->sel, list, s->cand, s->hist2, s->sm_count, st));
+    }
+    {
         StageTimer tm(s, 6);
-        tm.done(sk::launch_refine(P, s->sel, s->cand, s->cand2, s->hist2, s->I, s->sm_count, st));
-    } else {
-        // Second round (Section III-A): the P*k largest estimates become candidates, their exact values are
-        // fetched, and the k candidates of largest exact magnitude are kept (ties: smaller index).
-        sk::Params Q = P;                       // first selection: P*k of d (the threshold bin was picked for P*k)
-        Q.k = (uint32_t)s->cand_mult * P.k;
-        {
-            StageTimer tm(s, 5);
-            tm.done(sk::launch_emit(Q, s->keys, nullptr, s->sel, s->Ic, s->cand, s->hist2, s->sm_count, st));
+        int l = sk::launch_refine(Q, s->sel, s->cand, s->cand2, s->hist2, list, s->sm_count, st);
+        if (sharded) {                          // candidates in ascending order, and this process's sums of a_t there
+            l += sk::launch_sort_list(list, Q.k, s->cbitmap, s->bitmap_bytes / 4, s->scan, st);
+            l += sk::launch_gather_worker_sum(P, list, Q.k, s->e, x2, st);
         }
+        tm.done(l);
+    }
+    SK_CUDA(cudaGetLastError());
+    return SK_OK;
+}
+
+// Phase 3: second round on the exact values (P > 1), then the update of x and of the error-feedback residual.
+int phase_finish(sk_state* s, const float* x2, float* x) {
+    const sk::Params& P = s->P;
+    const bool sharded = x2 != nullptr;
+    cudaStream_t st = s->stream;
+    const float* asum = s->asum_live ? s->asum : nullptr;
+    const float* vhat = s->variant == 1 ? nullptr : s->vhat;
+    if (sharded) {                              // the summed exact values, placed at their coordinates
         StageTimer tm(s, 6);
-        int l = sk::launch_refine(Q, s->sel, s->cand, s->cand2, s->hist2, s->Ic, s->sm_count, st);
-        l += sk::launch_exact_keys(P, s->Ic, Q.k, s->variant == 1 ? nullptr : s->vhat, s->e, asum, s->keys2, s->hist,
-                                   s->sm_count, st);
+        uint32_t* list = s->cand_mult > 1 ? s->Ic : s->I;
+        tm.done(sk::launch_scatter(list, (uint32_t)s->cand_mult * P.k, x2, s->asum, st));
+        asum = s->asum;
+    }
+    if (s->cand_mult > 1) {
+        // Second round (Section III-A): the P*k largest estimates are candidates, their exact values are fetched,
+        // and the k candidates of largest exact magnitude are kept (ties: smaller index).
+        StageTimer tm(s, 6);
+        const uint32_t pk = (uint32_t)s->cand_mult * P.k;
+        int l = sk::launch_exact_keys(P, s->Ic, pk, vhat, s->e, asum, s->keys2, s->hist, s->sm_count, st);
         sk::Params Q2 = P;                      // second selection: k of the P*k candidates, keyed by exact value
-        Q2.d = Q.k;
+        Q2.d = pk;
         l += sk::launch_pick_bin(Q2, s->hist, s->sel, 0, st);
         l += sk::launch_emit(Q2, s->keys2, s->Ic, s->sel, s->I, s->cand, s->hist2, s->sm_count, st);
         l += sk::launch_refine(Q2, s->sel, s->cand, s->cand2, s->hist2, s->I, s->sm_count, st);
@@ -189,7 +241,7 @@ int do_step(sk_state* s, const float* grads, float* x) {
     {
         StageTimer tm(s, 7);     // the bitmap of I_{t-1} has served its purpose: clear it, then apply marks I_t
         int l = sk::launch_zero(s->bitmap, s->bitmap_bytes, st);
-        l += sk::launch_apply(P, s->I, s->variant == 1 ? nullptr : s->vhat, s->e, asum, x, s->bitmap, st);
+        l += sk::launch_apply(P, s->I, vhat, s->e, asum, x, s->bitmap, st);
         tm.done(l);
     }
     SK_CUDA(cudaGetLastError());
@@ -197,6 +249,24 @@ int do_step(sk_state* s, const float* grads, float* x) {
     s->k_prev = P.k;
     s->t += 1;
     if (s->timing) s->timed_steps += 1;
+    return SK_OK;
+}
+
+int do_step(sk_state* s, const float* grads, float* x) {
+    if (s->phase != 0) return fail(SK_ESTATE, "sk_step: a partitioned step is in progress (finish it with sk_step_finish)");
+    s->step_vec = (s->P.d % 4 == 0) && s->P.log2g >= 2 && ((uintptr_t)grads % 16 == 0) && ((uintptr_t)x % 16 == 0);
+    int rc = phase_local(s, grads, nullptr);
+    if (!rc) rc = phase_select(s, nullptr, nullptr);
+    if (!rc) rc = phase_finish(s, nullptr, x);
+    return rc;
+}
+
+// scratch of the partitioned step, allocated at its first use
+int shard_buffers(sk_state* s) {
+    if (s->cbitmap) return SK_OK;
+    SK_CUDA(cudaMalloc((void**)&s->cbitmap, s->bitmap_bytes));
+    SK_CUDA(cudaMalloc((void**)&s->scan, sk::scan_entries(s->bitmap_bytes / 4) * 4));
+    if (!s->asum) SK_CUDA(cudaMalloc((void**)&s->asum, ((uint64_t)s->P.d + 3) / 4 * 16));
     return SK_OK;
 }
 
@@ -239,7 +309,7 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     s->seed = seed;
     s->eps = eps;
     sk::Params& P = s->P;
-    P.d = (uint32_t)d; P.n = n; P.r = r; P.c = c; P.k = (uint32_t)k;
+    P.d = (uint32_t)d; P.n = n; P.n_all = n; P.r = r; P.c = c; P.k = (uint32_t)k;
     P.cs = (c + 31u) / 32u * 32u;
     P.beta1 = beta1; P.beta2 = beta2; P.lr = lr;
     uint32_t lg = 5;
@@ -291,7 +361,7 @@ void sk_destroy(sk_state* s) {
     if (s->stream) cudaStreamSynchronize(s->stream); else cudaDeviceSynchronize();
     for (void* p : {(void*)s->m, (void*)s->e, (void*)s->v, (void*)s->vhat, (void*)s->vstamp, (void*)s->tables,
                     (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->hist2, (void*)s->sel, (void*)s->cand, (void*)s->cand2,
-                    (void*)s->keys, (void*)s->gsum, (void*)s->asum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw, (void*)s->Ic, (void*)s->keys2,
+                    (void*)s->keys, (void*)s->gsum, (void*)s->asum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw, (void*)s->Ic, (void*)s->keys2, (void*)s->cbitmap, (void*)s->scan,
                     (void*)s->stage_grads, (void*)s->stage_x})
         if (p) cudaFree(p);
     for (const TimeRec& r : s->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -319,6 +389,44 @@ int sk_step_host(const float* grads_host, float* x_host, sk_state* s) {
     SK_CUDA(cudaMemcpyAsync(x_host, s->stage_x, (uint64_t)s->P.d * 4, cudaMemcpyDeviceToHost, s->stream));
     SK_CUDA(cudaStreamSynchronize(s->stream));
     return SK_OK;
+}
+
+uint64_t sk_exchange_floats(const sk_state* s, int which) {
+    if (!s) return 0;
+    if (which == 1) return (uint64_t)s->P.r * s->P.cs + (s->variant == 0 ? s->P.k : 0);
+    if (which == 2) return (uint64_t)s->cand_mult * s->P.k;
+    return 0;
+}
+
+int sk_step_local(const float* grads, float* exchange1, sk_state* s) {
+    if (!s || !grads || !exchange1) return fail(SK_EINVAL, "sk_step_local: null argument");
+    if (((uintptr_t)grads % 4) || ((uintptr_t)exchange1 % 16))
+        return fail(SK_EINVAL, "sk_step_local: grads must be 4-byte and exchange1 16-byte aligned");
+    if (s->phase != 0) return fail(SK_ESTATE, "sk_step_local: the previous partitioned step was not finished");
+    int rc = shard_buffers(s);
+    if (rc) return rc;
+    s->step_vec = (s->P.d % 4 == 0) && s->P.log2g >= 2 && ((uintptr_t)grads % 16 == 0);
+    rc = phase_local(s, grads, exchange1);
+    if (!rc) s->phase = 1;
+    return rc;
+}
+
+int sk_step_select(const float* exchange1, float* exchange2, sk_state* s) {
+    if (!s || !exchange1 || !exchange2) return fail(SK_EINVAL, "sk_step_select: null argument");
+    if (((uintptr_t)exchange1 % 16) || ((uintptr_t)exchange2 % 4))
+        return fail(SK_EINVAL, "sk_step_select: exchange1 must be 16-byte and exchange2 4-byte aligned");
+    if (s->phase != 1) return fail(SK_ESTATE, "sk_step_select: call sk_step_local first");
+    int rc = phase_select(s, exchange1, exchange2);
+    if (!rc) s->phase = 2;
+    return rc;
+}
+
+int sk_step_finish(const float* exchange2, float* x, sk_state* s) {
+    if (!s || !exchange2 || !x) return fail(SK_EINVAL, "sk_step_finish: null argument");
+    if (((uintptr_t)exchange2 | (uintptr_t)x) % 4) return fail(SK_EINVAL, "sk_step_finish: pointers must be 4-byte aligned");
+    if (s->phase != 2) return fail(SK_ESTATE, "sk_step_finish: call sk_step_select first");
+    s->phase = 0;
+    return phase_finish(s, exchange2, x);
 }
 
 int sk_set_stream(sk_state* s, void* stream) {
@@ -365,6 +473,12 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
                 return fail(SK_ENOMEM, "cudaMalloc of the candidate buffers failed: %s", cudaGetErrorString(cudaGetLastError()));
         }
         s->cand_mult = value;
+        return SK_OK;
+    }
+    if (!strcmp(key, "workers_total")) {
+        if (s->t != 0) return fail(SK_ESTATE, "workers_total can only be changed before the first step");
+        if (value < (int64_t)s->P.n || value >= (1ll << 31)) return fail(SK_EINVAL, "workers_total must be >= n");
+        s->P.n_all = (uint32_t)value;
         return SK_OK;
     }
     if (!strcmp(key, "variant")) {
@@ -420,6 +534,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     else if (!strcmp(key, "window_workers")) *value = s->window_workers;
     else if (!strcmp(key, "variant")) *value = s->variant;
     else if (!strcmp(key, "P")) *value = s->cand_mult;
+    else if (!strcmp(key, "workers_total")) *value = s->P.n_all;
     else if (!strcmp(key, "window_red_rows")) *value = s->window_red_rows;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;

@@ -21,6 +21,8 @@ struct Params {
     uint32_t win_panels;  // windowed family: windows per row = c / win_cw
     uint32_t k;
     float beta1, beta2, lr;
+    uint32_t n_all;     // workers the means are taken over: n, or the total over all processes when the workers are
+                        // partitioned (the handle then holds n of them)
 };
 
 // Device-resident selection state (one per handle).
@@ -90,5 +92,21 @@ int launch_v_materialize(const Params& P, const float* v, const uint32_t* vstamp
                          cudaStream_t st);
 int launch_masked_copy(const Params& P, const float* e, const uint32_t* bitmap, uint32_t workers, float* out,
                        cudaStream_t st);
+// ---- workers partitioned over processes (sk_shard.cu): canonical (ascending) index lists and the packing of what
+// the processes exchange
+constexpr uint32_t kScanWordsPerBlock = 1024;      // bitmap words one block of the compaction covers
+inline uint64_t scan_entries(uint64_t bitmap_words) { return (bitmap_words + kScanWordsPerBlock - 1) / kScanWordsPerBlock + 1; }
+// out <- the set bits of the bitmap as ascending coordinates; scan: scratch of scan_entries(words) uint32
+int launch_list_from_bitmap(const uint32_t* bitmap, uint64_t words, uint32_t* scan, uint32_t* out, cudaStream_t st);
+// sorts a list of distinct coordinates in place through a scratch bitmap of `words` words
+int launch_sort_list(uint32_t* list, uint32_t count, uint32_t* scratch_bitmap, uint64_t words, uint32_t* scan,
+                     cudaStream_t st);
+// out[q] = src[list[q]] for q < count, 0 for count <= q < padded
+int launch_gather(const uint32_t* list, uint32_t count, uint32_t padded, const float* src, float* out, cudaStream_t st);
+// dst[list[q]] = vals[q]
+int launch_scatter(const uint32_t* list, uint32_t count, const float* vals, float* dst, cudaStream_t st);
+// out[q] = sum over this handle's workers (in order) of e[w][list[q]]
+int launch_gather_worker_sum(const Params& P, const uint32_t* list, uint32_t count, const float* e, float* out,
+                             cudaStream_t st);
 
 }  // namespace sk

@@ -29,7 +29,7 @@ __device__ __forceinline__ float decay_owed_fast(float v, float beta2, uint32_t 
 
 // h = gsum / n ; v = beta2 v + (1-beta2) h^2, after the decay owed since `stamp`; `step` is t (1-based)
 __device__ __forceinline__ float second_moment_value(const Params& P, float v, uint32_t stamp, uint32_t step, float gsum) {
-    const float h = gsum / (float)P.n;
+    const float h = gsum / (float)P.n_all;
     return fmaf(P.beta2, decay_owed_fast(v, P.beta2, step - 1u - stamp), (1.0f - P.beta2) * h * h);
 }
 

@@ -421,7 +421,7 @@ k_exact_keys(const __grid_constant__ Params P, const uint32_t* __restrict__ C, u
         float abar = 0.0f;
         if (asum) abar = asum[j];
         else for (uint32_t w = 0; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
-        abar = abar / (float)P.n;
+        abar = abar / (float)P.n_all;
         const uint32_t key = key_of(vhat ? scale_est(abar, vhat[j]) : abar);
         keys2[q] = key;
         atomicAdd(&sh[key >> kHistShift], 1u);
@@ -451,7 +451,7 @@ k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const 
         for (uint32_t u = 0; u < 8; ++u) abar += a[u];
     }
     for (; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
-    abar = abar / (float)P.n;
+    abar = abar / (float)P.n_all;
     const float delta = vhat ? scale_est(abar, vhat[j]) : abar;
     x[j] = x[j] - P.lr * delta;
     atomicOr(&bitmap[j >> 5], 1u << (j & 31u));

@@ -215,11 +215,12 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
     }
 }
 
-// S = (S^(0) + S^(1) + ... + S^(n-1)) / n, workers added in index order (Algorithm 2, master side).
+// S = (S^(0) + S^(1) + ... + S^(n-1)) / n_all, workers added in index order (Algorithm 2, master side); with the
+// workers partitioned over processes this is the process's share of the mean.
 __global__ void __launch_bounds__(kThreads)
 k_sum_tables(const __grid_constant__ Params P, const float4* __restrict__ tables, float4* sum) {
     const uint32_t q4 = (P.r * P.cs) >> 2;
-    const float fn = (float)P.n;
+    const float fn = (float)P.n_all;
     for (uint32_t t = blockIdx.x * kThreads + threadIdx.x; t < q4; t += gridDim.x * kThreads) {
         float4 acc = __ldcs(tables + t);
         for (uint32_t w = 1; w < P.n; ++w) {

@@ -32,6 +32,11 @@ struct sk_state {
     float* gsum = nullptr;
     float* asum = nullptr;        // d, only with a second round: sum over the workers of a_t (worker order), written by the sketch kernel
     uint64_t bitmap_bytes = 0;
+    // one iteration in three phases (workers partitioned over processes): 0 idle, 1 after local, 2 after select
+    int phase = 0;
+    bool step_vec = false;        // this step runs the 128-bit kernels
+    bool asum_live = false;       // this step's sketch kernel filled asum
+    uint32_t *cbitmap = nullptr, *scan = nullptr;   // scratch of the partitioned step: candidate bitmap, block offsets
     sk::Select* sel = nullptr;
     sk::Cand *cand = nullptr, *cand2 = nullptr;
     float *stage_grads = nullptr, *stage_x = nullptr;
