@@ -17,8 +17,8 @@
  *     (v decays there); `v_keep=1` switches to "v unchanged off I_{t-1}" (the remark in Lemma 3's proof).
  *   - Algorithm 3 is read as a per-coordinate scale at query time:
  *     est_i = median_j( s_j(i) S[j,h_j(i)] ) / sqrt(vhat_i).
- *   - Delta_t holds the EXACT worker means at I_t, preconditioned (Section III-A "extract their exact
- *     values"); e_t^(i) is a_t^(i) with the coordinates of I_t set to zero (Lemma 3's proof).
+ *   - Delta_t holds the EXACT worker means at I_t, preconditioned (the second communication round of
+ *     Section III-A); e_t^(i) is a_t^(i) with the coordinates of I_t set to zero (Lemma 3's proof).
  *   - Even r: lower median.  Ties in top-k: the smaller index wins.
  *
  * ora_step also implements Algorithm 1 (parameter averaging) when the option "variant_pa" is set: per-worker

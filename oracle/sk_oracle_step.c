@@ -131,7 +131,7 @@ static inline void hash_at(const ora_state* s, uint32_t j, uint64_t i, uint32_t*
 
 static int ora_step_pa(ora_state* s, const float* grads, float* x);
 
-/* Second round of Section III-A ("In practice ..."): of the estimates take the P*k largest as candidates, fetch the
+/* Second round of Section III-A: of the estimates take the P*k largest as candidates, fetch the
  * EXACT values of the compressed vector there -- `exact[j]` is computed by the caller for the candidates only --
  * and keep the k candidates of largest exact magnitude (ties: smaller index).  With P = 1 this is plain Top-k of
  * the estimates.  `scale` is vhat for Algorithm 2 (exact value = mean_w a / sqrt(vhat)) or NULL for Algorithm 1. */
