@@ -52,6 +52,7 @@ def lib() -> C.CDLL:
         L.ora_destroy.restype = None; L.ora_destroy.argtypes = [vp]
         L.ora_set_hash.restype = None; L.ora_set_hash.argtypes = [vp, vp, vp]
         L.ora_set_option.restype = None; L.ora_set_option.argtypes = [vp, C.c_char_p, C.c_int]
+        L.ora_set_lr.restype = None; L.ora_set_lr.argtypes = [vp, f32]
         L.ora_step.restype = C.c_int; L.ora_step.argtypes = [vp, vp, vp]
         L.ora_field.restype = vp; L.ora_field.argtypes = [vp, C.c_char_p]
         L.ora_count.restype = u64; L.ora_count.argtypes = [vp, C.c_char_p]
@@ -120,7 +121,8 @@ class Oracle:
     """One SketchedAMSGrad (gradient averaging) optimiser; `step` advances it by one iteration."""
 
     def __init__(self, d, n, r, c, k, seed=0, log2g=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8,
-                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0, variant="ga", P=1):
+                 hash_idx=None, hash_sgn=None, v_keep=False, threads=1, window_lines=0, variant="ga", P=1,
+                 freeze_v=False):
         self.d, self.n, self.r, self.c, self.k, self.P = d, n, r, c, k, P
         self._h = lib().ora_create(d, n, r, c, k, seed, log2g, lr, beta1, beta2, eps)
         if not self._h:
@@ -142,6 +144,9 @@ class Oracle:
             if P < 1 or P * k > d:
                 raise ValueError("P must be >= 1 with P*k <= d")
             lib().ora_set_option(self._h, b"P", int(P))
+        if freeze_v and variant != "ga":
+            raise ValueError("freeze_v applies to Algorithm 2 (gradient averaging) only")
+        lib().ora_set_option(self._h, b"freeze_v", int(freeze_v))
         lib().ora_set_option(self._h, b"v_keep", int(v_keep))
         lib().ora_set_option(self._h, b"threads", int(threads))
 
@@ -152,6 +157,10 @@ class Oracle:
 
     def __del__(self):
         self.close()
+
+    def set_lr(self, lr: float) -> None:
+        """Step size alpha_t of the steps taken from now on."""
+        lib().ora_set_lr(self._h, float(lr))
 
     def step(self, grads: np.ndarray, x: np.ndarray) -> None:
         """grads: (n, d) float32, C-contiguous; x: (d,) float32, updated in place."""

@@ -71,6 +71,11 @@ void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn);
    the candidates of the last step are the uint32 field "cand"), "v_keep", "threads", "window_lines" (windowed hash family), "variant_pa" (1 = Algorithm 1, parameter averaging;
    per-worker v and vhat are then the fields "vw" and "vhatw", n*d each) */
 void ora_set_option(ora_state* s, const char* key, int value);
+/* "freeze_v" (Algorithm 2 only): h_t is not used and v, vhat keep the values they have (Section III-B: with the
+   variance term fixed the method becomes the fixed-preconditioner scheme it is compared with).
+   ora_set_lr: the step size alpha_t of the steps taken from now on; each step weights e_{t-1} by
+   alpha_{t-1}/alpha_t as Algorithms 1 and 2 print it (alpha_0 := alpha_1). */
+void ora_set_lr(ora_state* s, float lr);
 int  ora_step(ora_state* s, const float* grads /* n*d worker-major */, float* x /* d, in place */);
 
 /* field access: "m","e" (n*d) "v","vhat","est" (d) "tables" (n*r*c) "sum" (r*c) -> float*;

@@ -14,7 +14,9 @@ struct ora_state {
     uint64_t d, k, seed, t, k_prev;
     uint32_t n, r, c, log2g, window_lines;
     float lr, beta1, beta2, eps;
+    float lr_prev;           /* alpha_{t-1}: the step size of the last step taken (alpha_0 := alpha_1) */
     int v_keep, threads, variant_pa;
+    int freeze_v;            /* Algorithm 2 without h_t and without the update of v, vhat (Section III-B's remark) */
     uint32_t P;              /* candidate multiplier of the second round (Section III-A); 1 = no second round */
     uint32_t* cand;          /* the P*k candidates of the last step, ascending */
     float *vw, *vhatw;       /* parameter-averaging variant: per-worker v and vhat (n*d each) */
@@ -32,7 +34,7 @@ ora_state* ora_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k
     if ((c >> log2g) == 0 || d >= (1ULL << 32)) return NULL;
     ora_state* s = (ora_state*)calloc(1, sizeof(ora_state));
     s->d = d; s->n = n; s->r = r; s->c = c; s->k = k; s->seed = seed; s->log2g = log2g;
-    s->lr = lr; s->beta1 = beta1; s->beta2 = beta2; s->eps = eps;
+    s->lr = lr; s->lr_prev = lr; s->beta1 = beta1; s->beta2 = beta2; s->eps = eps;
     s->threads = 1;
     s->P = 1;
     s->m = (float*)calloc((size_t)n * d, sizeof(float));        /* m_0 = 0 */
@@ -60,8 +62,12 @@ void ora_destroy(ora_state* s) {
 
 void ora_set_hash(ora_state* s, const uint32_t* idx, const int8_t* sgn) { s->h_idx = idx; s->h_sgn = sgn; }
 
+/* alpha_t of the steps taken from now on; the step computes alpha_{t-1}/alpha_t from the last step's value */
+void ora_set_lr(ora_state* s, float lr) { s->lr = lr; }
+
 void ora_set_option(ora_state* s, const char* key, int value) {
     if (!strcmp(key, "v_keep")) s->v_keep = value;
+    else if (!strcmp(key, "freeze_v")) s->freeze_v = value;
     else if (!strcmp(key, "window_lines")) {
         /* only with g = 32 and at least one whole window in a row; otherwise left unchanged */
         if (value >= 0 && (value == 0 || (s->log2g == 5 && (uint64_t)32 * (uint64_t)value <= s->c)))
@@ -163,7 +169,7 @@ int ora_step(ora_state* s, const float* grads, float* x) {
     const uint64_t d = s->d, k = s->k;
     const uint32_t n = s->n, r = s->r, c = s->c;
     const double b1 = (double)s->beta1, b2 = (double)s->beta2, lr = (double)s->lr;
-    const double rho = 1.0;   /* alpha_{t-1}/alpha_t with a constant step size (Theorem 2's alpha_t) */
+    const double rho = (double)s->lr_prev / (double)s->lr;   /* alpha_{t-1}/alpha_t (Algorithm 2's sketch line) */
 #ifdef _OPENMP
     omp_set_num_threads(s->threads);
 #endif
@@ -177,8 +183,10 @@ int ora_step(ora_state* s, const float* grads, float* x) {
        v_t = beta2 v_{t-1} + (1-beta2) h_t^2 ; vhat_t = max(vhat_{t-1}, v_t)   (master side) */
     memset(s->mask, 0, (size_t)d);
     for (uint64_t t = 0; t < s->k_prev; ++t) s->mask[s->I_prev[t]] = 1;
+    /* freeze_v: h_t is not sent and v, vhat keep their initial values (the fixed-variance scheme the paper
+       compares with, Section III-B) */
 #pragma omp parallel for schedule(static)
-    for (uint64_t j = 0; j < d; ++j) {
+    for (uint64_t j = 0; j < (s->freeze_v ? 0 : d); ++j) {
         double h = 0.0;
         if (s->mask[j]) {
             for (uint32_t w = 0; w < n; ++w) h += (double)grads[(uint64_t)w * d + j];
@@ -250,6 +258,7 @@ int ora_step(ora_state* s, const float* grads, float* x) {
 
     memcpy(s->I_prev, s->I, (size_t)k * sizeof(uint32_t));
     s->k_prev = k;
+    s->lr_prev = s->lr;
     s->t += 1;
     return 0;
 }
@@ -267,7 +276,7 @@ static int ora_step_pa(ora_state* s, const float* grads, float* x) {
     const uint64_t d = s->d, k = s->k;
     const uint32_t n = s->n, r = s->r, c = s->c;
     const double b1 = (double)s->beta1, b2 = (double)s->beta2, lr = (double)s->lr;
-    const double rho = 1.0;
+    const double rho = (double)s->lr_prev / (double)s->lr;   /* alpha_{t-1}/alpha_t (Algorithm 1's sketch line) */
 #ifdef _OPENMP
     omp_set_num_threads(s->threads);
 #endif
@@ -324,6 +333,7 @@ static int ora_step_pa(ora_state* s, const float* grads, float* x) {
     }
     memcpy(s->I_prev, s->I, (size_t)k * sizeof(uint32_t));
     s->k_prev = k;
+    s->lr_prev = s->lr;
     s->t += 1;
     return 0;
 }

@@ -78,6 +78,29 @@ def test_auxiliary_sequence_identity_and_masking():
         assert np.array_equal(I, true_topk.astype(np.uint32))
 
 
+def test_auxiliary_sequence_identity_under_a_step_size_schedule():
+    # Section IV-A with alpha_t = alpha / sqrt(t): x_{t+1} - x~_{t+1} = alpha_t e_t needs e_{t-1} weighted by
+    # alpha_{t-1}/alpha_t in the sketched vector (Algorithm 1's sketch line)
+    d, n, k = 300, 3, 25
+    hi, hs = _identity(d)
+    o = oracle.Oracle(d, n, 1, d, k, hash_idx=hi, hash_sgn=hs, variant="pa", lr=0.05, beta1=0.9, beta2=0.99, eps=1e-6)
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal(d).astype(np.float32)
+    xt = x.astype(np.float64).copy()
+    worst = 0.0
+    for t in range(1, 11):
+        lr = np.float32(0.05 / np.sqrt(t))
+        o.set_lr(lr)
+        g = (rng.standard_normal((n, d)) * rng.uniform(0.01, 1.0, d)).astype(np.float32)
+        o.step(g, x)
+        m, vh = o.field("m").astype(np.float64), o.field("vhatw").astype(np.float64)
+        xt = xt - np.float64(lr) * (m / np.sqrt(vh)).mean(0)
+        want = np.float64(lr) * o.field("e").astype(np.float64).mean(0)
+        np.testing.assert_allclose(x.astype(np.float64) - xt, want, rtol=0, atol=2e-5)
+        worst = max(worst, np.abs(want).max())
+    assert worst > 1e-2
+
+
 def test_no_compression_averages_local_amsgrad_steps():
     # k = d and a lossless sketch: e stays 0 and x moves by the average of the workers' own AMSGrad directions
     # (Section II-A: parameter averaging is NOT AMSGrad on the averaged gradient).

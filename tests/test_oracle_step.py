@@ -29,6 +29,8 @@ EXAMPLES = {
     "B": dict(n=1, d=2, grads=[[1.0, 0.5]]),
     "C": dict(n=2, d=2, grads=[[1.0, 0.5], [3.0, -0.5]]),
     "D": dict(n=1, d=1, grads=[[1.0]], v_keep=True),
+    "G": dict(n=1, d=1, grads=[[1.0]], freeze_v=True),
+    "H": dict(n=1, d=2, grads=[[1.0, 0.5]], freeze_v=True, lrs=[0.1, 0.05, 0.025]),
 }
 
 
@@ -37,11 +39,14 @@ def test_worked_examples(ex):
     cfg = EXAMPLES[ex]
     n, d = cfg["n"], cfg["d"]
     hi, hs = _identity(d)
-    o = oracle.Oracle(d, n, 1, d, 1, hash_idx=hi, hash_sgn=hs, v_keep=cfg.get("v_keep", False), **HP)
+    o = oracle.Oracle(d, n, 1, d, 1, hash_idx=hi, hash_sgn=hs, v_keep=cfg.get("v_keep", False),
+                      freeze_v=cfg.get("freeze_v", False), **HP)
     g = np.array(cfg["grads"], np.float32)
     x = np.zeros(d, np.float32)
     checks = _golden()[ex]
     for t in range(1, max(c[0] for c in checks) + 1):
+        if "lrs" in cfg:
+            o.set_lr(cfg["lrs"][t - 1])
         o.step(g, x)
         for (tt, q, j, val) in checks:
             if tt != t:
@@ -124,7 +129,7 @@ def test_step_invariants(log2g):
 
 def test_lemma3_identity_and_contraction():
     # Lemma 3: x_t - x~_t = alpha vhat_{t-1}^{-1/2} e_{t-1}, with x~_{t+1} = x~_t - alpha vhat_t^{-1/2} mean_w m_t.
-    # Also "Delta_t is some coordinates of Delta~_t": ||Delta~ - Delta|| <= ||Delta~||, and when I_t is the true
+    # Also, Delta_t being a restriction of Delta~_t to I_t: ||Delta~ - Delta|| <= ||Delta~||, and when I_t is the true
     # top-k of Delta~_t (lossless sketch) the bound of Lemma 2 holds: <= sqrt(1-k/d) ||Delta~||.
     d, n, k = 400, 4, 40
     o, hp, hist = _run(d, n, 1, d, k, 12, 0, identity=True)
@@ -142,6 +147,73 @@ def test_lemma3_identity_and_contraction():
         assert np.linalg.norm(dtil - dsel) <= np.sqrt(1 - k / d) * np.linalg.norm(dtil) * (1 + 1e-6)
         true_topk = np.sort(np.argsort(-np.abs(dtil), kind="stable")[:k])
         assert np.array_equal(h["I"], true_topk.astype(np.uint32))
+
+
+def test_lemma3_identity_under_a_step_size_schedule():
+    # Lemma 3 with alpha_t = alpha / sqrt(t) (Theorem 2's choice): x_{t+1} - x~_{t+1} = alpha_t vhat_t^{-1/2} e_t with
+    # x~_{t+1} = x~_t - alpha_t vhat_t^{-1/2} mean_w m_t.  It holds only because e_{t-1} enters a_t weighted by
+    # alpha_{t-1}/alpha_t: with the weight dropped or inverted the two sides drift apart.
+    d, n, k, steps = 300, 3, 30, 12
+    hi, hs = _identity(d)
+    o = oracle.Oracle(d, n, 1, d, k, hash_idx=hi, hash_sgn=hs, lr=0.05, beta1=0.9, beta2=0.99, eps=1e-6)
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal(d).astype(np.float32)
+    xt = x.astype(np.float64).copy()
+    gaps = []
+    for t in range(1, steps + 1):
+        lr = np.float32(0.05 / np.sqrt(t))
+        o.set_lr(lr)
+        g = (rng.standard_normal((n, d)) * rng.uniform(0.01, 1.0, d)).astype(np.float32)
+        o.step(g, x)
+        vh = o.field("vhat").astype(np.float64)
+        xt = xt - np.float64(lr) * o.field("m").astype(np.float64).mean(0) / np.sqrt(vh)
+        want = np.float64(lr) * o.field("e").astype(np.float64).mean(0) / np.sqrt(vh)
+        np.testing.assert_allclose(x.astype(np.float64) - xt, want, rtol=0, atol=2e-5)
+        gaps.append(np.abs(want).max())
+    assert max(gaps) > 1e-2          # the identity is not vacuous: the residual term is thousands of tolerances large
+
+
+def test_constant_schedule_and_unit_weight_are_the_plain_step():
+    # alpha_{t-1}/alpha_t = 1: setting the same step size before every step changes nothing, bit for bit
+    d, n, r, c, k = 500, 2, 3, 64, 20
+    a = oracle.Oracle(d, n, r, c, k, seed=5, log2g=2, lr=0.01)
+    b = oracle.Oracle(d, n, r, c, k, seed=5, log2g=2, lr=0.01)
+    rng = np.random.default_rng(2)
+    xa = np.zeros(d, np.float32); xb = np.zeros(d, np.float32)
+    for t in range(5):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        b.set_lr(0.01)
+        a.step(g, xa); b.step(g, xb)
+        assert np.array_equal(xa, xb) and np.array_equal(a.field("e"), b.field("e"))
+
+
+def test_frozen_second_moments():
+    # freeze_v (Section III-B's remark): v and vhat never change; with vhat = s^2 everywhere the estimates, and hence
+    # the index sets and residuals, do not depend on s, and x moves 1/s as far (s a power of two: exactly)
+    d, n, r, c, k = 800, 3, 5, 128, 40
+    runs = {}
+    for s2 in (1.0, 4.0):
+        o = oracle.Oracle(d, n, r, c, k, seed=3, log2g=3, lr=0.25, eps=s2, freeze_v=True)
+        rng = np.random.default_rng(7)
+        x = np.zeros(d, np.float32)
+        sets = []
+        for t in range(6):
+            g = rng.standard_normal((n, d)).astype(np.float32)
+            o.step(g, x)
+            assert np.all(o.field("vhat") == np.float32(s2)) and np.all(o.field("v") == np.float32(s2))
+            sets.append(o.field("I").copy())
+        runs[s2] = (sets, x.copy(), o.field("e").copy())
+    for a, b in zip(runs[1.0][0], runs[4.0][0]):
+        assert np.array_equal(a, b)
+    assert np.array_equal(runs[1.0][2], runs[4.0][2])
+    np.testing.assert_allclose(runs[4.0][1], runs[1.0][1] / 2, rtol=3e-7, atol=0)
+    # and the moving-vhat run differs (the switch does something)
+    o = oracle.Oracle(d, n, r, c, k, seed=3, log2g=3, lr=0.25, eps=1.0)
+    rng = np.random.default_rng(7)
+    x = np.zeros(d, np.float32)
+    for t in range(6):
+        o.step(rng.standard_normal((n, d)).astype(np.float32), x)
+    assert np.any(o.field("vhat") > 1.0) and not np.array_equal(x, runs[1.0][1])
 
 
 def test_no_compression_reduces_to_distributed_amsgrad():
