@@ -48,16 +48,23 @@ typedef struct sk_state sk_state;
 sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, uint64_t seed,
                     float lr, float beta1, float beta2, float eps);
 
-/* One iteration of Algorithm 2 (the whole list above).  grads: device, n*d fp32, worker-major
- * (grads[w*d + j]), read only.  x: device, d fp32, updated in place.  Both must be 4-byte aligned; the
+/* One iteration of Algorithm 2 (the whole list above).  grads: device, n*d gradient entries, worker-major
+ * (grads[w*d + j]), read only: fp32, or bf16 when the option "grads_bf16" is 1 (the entries are widened exactly;
+ * everything else stays fp32).  x: device, d fp32, updated in place.  Both must be 4-byte aligned; the
  * vectorised kernels are used when d % 4 == 0 and both are 16-byte aligned, scalar kernels otherwise.
  * Asynchronous: returns after enqueueing on the handle's stream. */
-int sk_step(const float* grads, float* x, sk_state* state);
+int sk_step(const void* grads, float* x, sk_state* state);
+
+/* Step size alpha_t of the steps taken from now on (Algorithms 1 and 2 allow a schedule; Theorem 2 uses
+ * alpha/sqrt(t)).  Each step weights e_{t-1} by alpha_{t-1}/alpha_t, computed in fp64 from the two fp32 values
+ * and rounded to fp32, with alpha_{t-1} the step size of the last step taken (1 when they are equal).  Finite;
+ * a zero step size cannot precede or follow a different one.  Not inside a partitioned step. */
+int sk_set_lr(sk_state* state, float lr);
 
 /* Same step with HOST buffers: copies grads (n*d) to an internal device staging buffer and x (d) in,
  * runs the step, copies x back, and synchronises the stream.  Pinned host memory makes the copies faster
  * but is not required.  The staging buffers are allocated on first use and freed by sk_destroy. */
-int sk_step_host(const float* grads_host, float* x_host, sk_state* state);
+int sk_step_host(const void* grads_host, float* x_host, sk_state* state);
 
 /* ---- One iteration with the WORKERS PARTITIONED over several processes (one GPU each) -----------------------------
  * Every process creates a handle for its own n workers (same d, r, c, k, seed, hyper-parameters and options on all
@@ -83,7 +90,7 @@ int sk_step_host(const float* grads_host, float* x_host, sk_state* state);
  * synchronises.  Calls out of order return SK_ESTATE.  With one process the result equals sk_step's up to the
  * rounding of the sums. */
 uint64_t sk_exchange_floats(const sk_state* state, int which /* 1 or 2 */);
-int sk_step_local(const float* grads, float* exchange1, sk_state* state);
+int sk_step_local(const void* grads, float* exchange1, sk_state* state);
 int sk_step_select(const float* exchange1, float* exchange2, sk_state* state);
 int sk_step_finish(const float* exchange2, float* x, sk_state* state);
 
@@ -102,6 +109,11 @@ int sk_sync(sk_state* state);
  *                  estimates become candidates, their exact values are fetched from the workers' vectors, and the
  *                  k candidates of largest exact magnitude form I_t (ties: smaller index).  1 (default) = no second
  *                  round.  P*k <= d.  Only before the first step.  The candidates of the last step are field "cand".
+ *   "freeze_v"     1: Algorithm 2 without h_t and without the update of v and vhat, which keep the values they have
+ *                  (set them with sk_set "v", "vhat"): the fixed-variance scheme Section III-B reduces the method
+ *                  to.  0 (default) resumes the updates.  Gradient averaging only.  Any time between steps.
+ *   "grads_bf16"   1: the gradient arguments of sk_step, sk_step_host and sk_step_local hold bf16 entries
+ *                  (2 bytes each, same layout).  Default 0.  Any time between steps.
  *   "workers_total" number of workers the means are taken over, >= n; default n.  Set it on every handle of a
  *                  partitioned step (see sk_step_local) to the sum of their n.  Only before the first step.
  *   "variant"      0 (default) = gradient averaging, Algorithm 2; 1 = parameter averaging, Algorithm 1: every worker

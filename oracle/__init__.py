@@ -162,6 +162,10 @@ class Oracle:
         """Step size alpha_t of the steps taken from now on."""
         lib().ora_set_lr(self._h, float(lr))
 
+    def set_freeze_v(self, on: bool) -> None:
+        """Algorithm 2 without h_t and the update of v, vhat (on), or with them (off), from the next step."""
+        lib().ora_set_option(self._h, b"freeze_v", int(on))
+
     def step(self, grads: np.ndarray, x: np.ndarray) -> None:
         """grads: (n, d) float32, C-contiguous; x: (d,) float32, updated in place."""
         assert grads.dtype == np.float32 and grads.flags.c_contiguous and grads.size == self.n * self.d

@@ -13,7 +13,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsketched_amsgrad.so")
 
-EXPORTS = ["sk_create", "sk_step", "sk_step_host", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
+EXPORTS = ["sk_create", "sk_step", "sk_set_lr", "sk_step_host", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
            "sk_get_option", "sk_hash", "sk_get", "sk_set", "sk_algorithmic_bytes", "sk_get_timing", "sk_select_static",
            "sk_exchange_floats", "sk_step_local", "sk_step_select", "sk_step_finish", "sk_last_error", "sk_version"]
 STATIC_MAX_D = 262144
@@ -39,6 +39,7 @@ def lib() -> C.CDLL:
         L.sk_create.restype = vp
         L.sk_create.argtypes = [u64, u32, u32, u32, u64, u64, f32, f32, f32, f32]
         L.sk_step.restype = C.c_int; L.sk_step.argtypes = [vp, vp, vp]
+        L.sk_set_lr.restype = C.c_int; L.sk_set_lr.argtypes = [vp, f32]
         L.sk_step_host.restype = C.c_int; L.sk_step_host.argtypes = [vp, vp, vp]
         L.sk_destroy.restype = None; L.sk_destroy.argtypes = [vp]
         L.sk_set_stream.restype = C.c_int; L.sk_set_stream.argtypes = [vp, vp]
@@ -118,6 +119,10 @@ class SketchedAMSGrad:
     def step(self, grads, x) -> None:
         """grads: CUDA float32 tensor of n*d elements (worker-major); x: CUDA float32 tensor of d, in place."""
         _check(lib().sk_step(_ptr(grads), _ptr(x), self._h))
+
+    def set_lr(self, lr: float) -> None:
+        """Step size of the steps taken from now on; e_{t-1} is weighted by alpha_{t-1}/alpha_t (Algorithms 1, 2)."""
+        _check(lib().sk_set_lr(self._h, float(lr)))
 
     def step_host(self, grads, x) -> None:
         """Same step with host buffers (numpy arrays or CPU tensors, ideally pinned); x is updated in place."""

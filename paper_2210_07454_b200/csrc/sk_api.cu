@@ -111,11 +111,11 @@ int check_status(sk_state* s) {
     return SK_OK;
 }
 
-sk::MomentArgs moment_args(const sk_state* s, const float* grads) {
+sk::MomentArgs moment_args(const sk_state* s, const void* grads) {
     sk::MomentArgs A{};
-    A.grads = grads; A.m = s->m; A.e = s->e; A.tables = s->tables; A.gsum = s->gsum;
+    A.grads = grads; A.grad_bf16 = s->grads_bf16 ? 1u : 0u; A.m = s->m; A.e = s->e; A.tables = s->tables; A.gsum = s->gsum;
     A.v = s->v; A.vhat = s->vhat; A.vstamp = s->vstamp; A.bitmap = s->bitmap;
-    A.step = (uint32_t)(s->t + 1); A.members = s->k_prev ? 1u : 0u;
+    A.step = (uint32_t)(s->vclock + 1); A.members = s->k_prev ? 1u : 0u;
     A.vw = s->vw; A.vhatw = s->vhatw; A.variant = (uint32_t)s->variant;
     return A;
 }
@@ -126,7 +126,9 @@ sk::MomentArgs moment_args(const sk_state* s, const float* grads) {
 // the candidates]; both index lists are in ascending order so that position q means the same coordinate everywhere.
 
 // Phase 1 (workers): moments, error-compensated vector, sketches of this handle's workers, their sum.
-int phase_local(sk_state* s, const float* grads, float* x1) {
+int phase_local(sk_state* s, const void* grads, float* x1) {
+    // alpha_{t-1}/alpha_t weights e_{t-1} in the sketched vector (the sketch lines of Algorithms 1 and 2)
+    s->P.rho = (s->lr_prev == s->P.lr) ? 1.0f : (float)((double)s->lr_prev / (double)s->P.lr);
     const sk::Params& P = s->P;
     const bool vec = s->step_vec;
     const bool sharded = x1 != nullptr;
@@ -180,6 +182,7 @@ int phase_select(sk_state* s, const float* x1, float* x2) {
     const bool sharded = x1 != nullptr;
     cudaStream_t st = s->stream;
     sk::MomentArgs A = moment_args(s, nullptr);
+    if (s->freeze_v) A.members = 0;             // v, vhat stay as they are (Section III-B's fixed-variance remark)
     sk::Params Q = P;                           // first selection: P*k of d (k without a second round)
     Q.k = (uint32_t)s->cand_mult * P.k;
     {
@@ -247,12 +250,14 @@ int phase_finish(sk_state* s, const float* x2, float* x) {
     SK_CUDA(cudaGetLastError());
     std::swap(s->I, s->I_prev);      // I_prev now holds I_t
     s->k_prev = P.k;
+    s->lr_prev = P.lr;
+    if (!s->freeze_v || s->variant == 1) s->vclock += 1;
     s->t += 1;
     if (s->timing) s->timed_steps += 1;
     return SK_OK;
 }
 
-int do_step(sk_state* s, const float* grads, float* x) {
+int do_step(sk_state* s, const void* grads, float* x) {
     if (s->phase != 0) return fail(SK_ESTATE, "sk_step: a partitioned step is in progress (finish it with sk_step_finish)");
     s->step_vec = (s->P.d % 4 == 0) && s->P.log2g >= 2 && ((uintptr_t)grads % 16 == 0) && ((uintptr_t)x % 16 == 0);
     int rc = phase_local(s, grads, nullptr);
@@ -311,7 +316,8 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     sk::Params& P = s->P;
     P.d = (uint32_t)d; P.n = n; P.n_all = n; P.r = r; P.c = c; P.k = (uint32_t)k;
     P.cs = (c + 31u) / 32u * 32u;
-    P.beta1 = beta1; P.beta2 = beta2; P.lr = lr;
+    P.beta1 = beta1; P.beta2 = beta2; P.lr = lr; P.rho = 1.0f;
+    s->lr_prev = lr;
     uint32_t lg = 5;
     while ((1u << lg) > c) --lg;
     P.log2g = lg;
@@ -369,20 +375,21 @@ void sk_destroy(sk_state* s) {
     delete s;
 }
 
-int sk_step(const float* grads, float* x, sk_state* s) {
+int sk_step(const void* grads, float* x, sk_state* s) {
     if (!s || !grads || !x) return fail(SK_EINVAL, "sk_step: null argument");
     if (((uintptr_t)grads | (uintptr_t)x) % 4) return fail(SK_EINVAL, "sk_step: pointers must be 4-byte aligned");
     return do_step(s, grads, x);
 }
 
-int sk_step_host(const float* grads_host, float* x_host, sk_state* s) {
+int sk_step_host(const void* grads_host, float* x_host, sk_state* s) {
     if (!s || !grads_host || !x_host) return fail(SK_EINVAL, "sk_step_host: null argument");
     const uint64_t nd = (uint64_t)s->P.n * s->P.d;
+    const uint64_t gbytes = nd * (s->grads_bf16 ? 2 : 4);
     if (!s->stage_grads) {
         SK_CUDA(cudaMalloc((void**)&s->stage_grads, nd * 4));
         SK_CUDA(cudaMalloc((void**)&s->stage_x, (uint64_t)s->P.d * 4));
     }
-    SK_CUDA(cudaMemcpyAsync(s->stage_grads, grads_host, nd * 4, cudaMemcpyHostToDevice, s->stream));
+    SK_CUDA(cudaMemcpyAsync(s->stage_grads, grads_host, gbytes, cudaMemcpyHostToDevice, s->stream));
     SK_CUDA(cudaMemcpyAsync(s->stage_x, x_host, (uint64_t)s->P.d * 4, cudaMemcpyHostToDevice, s->stream));
     int rc = do_step(s, s->stage_grads, s->stage_x);
     if (rc) return rc;
@@ -398,7 +405,7 @@ uint64_t sk_exchange_floats(const sk_state* s, int which) {
     return 0;
 }
 
-int sk_step_local(const float* grads, float* exchange1, sk_state* s) {
+int sk_step_local(const void* grads, float* exchange1, sk_state* s) {
     if (!s || !grads || !exchange1) return fail(SK_EINVAL, "sk_step_local: null argument");
     if (((uintptr_t)grads % 4) || ((uintptr_t)exchange1 % 16))
         return fail(SK_EINVAL, "sk_step_local: grads must be 4-byte and exchange1 16-byte aligned");
@@ -427,6 +434,16 @@ int sk_step_finish(const float* exchange2, float* x, sk_state* s) {
     if (s->phase != 2) return fail(SK_ESTATE, "sk_step_finish: call sk_step_select first");
     s->phase = 0;
     return phase_finish(s, exchange2, x);
+}
+
+int sk_set_lr(sk_state* s, float lr) {
+    if (!s) return fail(SK_EINVAL, "null handle");
+    if (!std::isfinite(lr)) return fail(SK_EINVAL, "the step size must be finite");
+    if (lr == 0.0f && lr != s->P.lr) return fail(SK_EINVAL, "a zero step size has no ratio alpha_{t-1}/alpha_t");
+    if (s->phase != 0) return fail(SK_ESTATE, "the step size cannot change inside a partitioned step");
+    if (s->lr_prev == 0.0f && lr != 0.0f) return fail(SK_EINVAL, "a zero step size has no ratio alpha_{t-1}/alpha_t");
+    s->P.lr = lr;
+    return SK_OK;
 }
 
 int sk_set_stream(sk_state* s, void* stream) {
@@ -475,6 +492,17 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         s->cand_mult = value;
         return SK_OK;
     }
+    if (!strcmp(key, "freeze_v")) {
+        if (value != 0 && s->variant == 1) return fail(SK_EINVAL, "freeze_v applies to gradient averaging (Algorithm 2) only");
+        if (s->phase != 0) return fail(SK_ESTATE, "freeze_v cannot change inside a partitioned step");
+        s->freeze_v = value != 0;
+        return SK_OK;
+    }
+    if (!strcmp(key, "grads_bf16")) {
+        if (value != 0 && value != 1) return fail(SK_EINVAL, "grads_bf16 must be 0 or 1");
+        s->grads_bf16 = value != 0;
+        return SK_OK;
+    }
     if (!strcmp(key, "workers_total")) {
         if (s->t != 0) return fail(SK_ESTATE, "workers_total can only be changed before the first step");
         if (value < (int64_t)s->P.n || value >= (1ll << 31)) return fail(SK_EINVAL, "workers_total must be >= n");
@@ -484,6 +512,7 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
     if (!strcmp(key, "variant")) {
         if (s->t != 0) return fail(SK_ESTATE, "variant can only be changed before the first step");
         if (value != 0 && value != 1) return fail(SK_EINVAL, "variant must be 0 (gradient averaging) or 1 (parameter averaging)");
+        if (value == 1 && s->freeze_v) return fail(SK_EINVAL, "freeze_v applies to gradient averaging (Algorithm 2) only");
         if (value == 1 && !s->vw) {                   // v_0^(w) = vhat_0^(w) = eps on every worker (Algorithm 1)
             const uint64_t nd = (uint64_t)s->P.n * s->P.d;
             if (cudaMalloc((void**)&s->vw, nd * 4) != cudaSuccess || cudaMalloc((void**)&s->vhatw, nd * 4) != cudaSuccess)
@@ -535,6 +564,8 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     else if (!strcmp(key, "variant")) *value = s->variant;
     else if (!strcmp(key, "P")) *value = s->cand_mult;
     else if (!strcmp(key, "workers_total")) *value = s->P.n_all;
+    else if (!strcmp(key, "freeze_v")) *value = s->freeze_v;
+    else if (!strcmp(key, "grads_bf16")) *value = s->grads_bf16;
     else if (!strcmp(key, "window_red_rows")) *value = s->window_red_rows;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
@@ -557,11 +588,12 @@ int sk_hash(const sk_state* s, uint32_t row, uint64_t i0, uint64_t count, uint32
 uint64_t sk_algorithmic_bytes(const sk_state* s) {
     if (!s) return 0;
     const uint64_t n = s->P.n, d = s->P.d, r = s->P.r, c = s->P.c, k = s->P.k;
+    const uint64_t g = s->grads_bf16 ? 2 : 0;     // bytes saved per gradient entry when they arrive as bf16
     // second round: per candidate, its index, the n workers' values (and vhat) in, its exact value out
     const uint64_t second = s->cand_mult > 1 ? (uint64_t)s->cand_mult * k * (4 * n + (s->variant == 1 ? 8 : 12)) : 0;
     if (s->variant == 1)     // Algorithm 1: read g,m,v,vhat,e and write m,v,vhat,e; no master-side second moments
-        return 36 * n * d + 8 * n * r * c + 4 * r * c + 8 * n * k + 8 * k + second;
-    return 20 * n * d + 4 * d + 8 * n * r * c + 4 * r * c + 12 * n * k + 24 * k + second;
+        return (36 - g) * n * d + 8 * n * r * c + 4 * r * c + 8 * n * k + 8 * k + second;
+    return (20 - g) * n * d + 4 * d + 8 * n * r * c + 4 * r * c + 12 * n * k + 24 * k + second;
 }
 
 int sk_get_timing(sk_state* s, double* ms, uint64_t* launches) {

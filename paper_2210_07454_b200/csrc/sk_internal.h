@@ -21,6 +21,7 @@ struct Params {
     uint32_t win_panels;  // windowed family: windows per row = c / win_cw
     uint32_t k;
     float beta1, beta2, lr;
+    float rho;          // alpha_{t-1}/alpha_t, the weight of e_{t-1} in the sketched vector (1 for a constant step size)
     uint32_t n_all;     // workers the means are taken over: n, or the total over all processes when the workers are
                         // partitioned (the handle then holds n of them)
 };
@@ -41,7 +42,8 @@ struct Cand { uint32_t key, idx; };
 
 // Pointers of the moment + sketch kernel (all device memory).
 struct MomentArgs {
-    const float* grads;
+    const void* grads;       // n*d gradient entries, fp32 or (grad_bf16 != 0) bf16
+    uint32_t grad_bf16;
     float *m, *e, *tables;
     float* asum;             // d or nullptr: running sum over the workers of a_t, in worker order (second round of Section III-A)
     float* gsum;             // running gradient sums on I_{t-1} when the workers are processed in several launches

@@ -1,6 +1,7 @@
 // Master-side second-moment update of Algorithm 2 for one coordinate of I_{t-1}, shared by the kernels that
 // apply it.  Device-side only.
 #pragma once
+#include <cstdint>
 #include "sk_internal.h"
 
 namespace sk {
@@ -31,6 +32,21 @@ __device__ __forceinline__ float decay_owed_fast(float v, float beta2, uint32_t 
 __device__ __forceinline__ float second_moment_value(const Params& P, float v, uint32_t stamp, uint32_t step, float gsum) {
     const float h = gsum / (float)P.n_all;
     return fmaf(P.beta2, decay_owed_fast(v, P.beta2, step - 1u - stamp), (1.0f - P.beta2) * h * h);
+}
+
+// Gradient entries are stored as fp32 or as bf16 (the upper half of an fp32: widening is exact).
+// Four consecutive entries of quad index q (q-th group of four in the worker-major array):
+__device__ __forceinline__ float4 load_grad4(const void* grads, uint64_t q, uint32_t bf16) {
+    if (bf16) {
+        const uint2 raw = __ldcs((const uint2*)grads + q);
+        return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
+                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+    }
+    return __ldcs((const float4*)grads + q);
+}
+__device__ __forceinline__ float load_grad1(const void* grads, uint64_t q, uint32_t bf16) {
+    if (bf16) return __uint_as_float((uint32_t)((const uint16_t*)grads)[q] << 16);
+    return ((const float*)grads)[q];
 }
 
 }  // namespace sk

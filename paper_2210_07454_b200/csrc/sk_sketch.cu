@@ -52,10 +52,11 @@ k_masked_copy(const float* __restrict__ e, const uint32_t* __restrict__ bitmap, 
 #define SK_MOMENT(mm, aa, gg, mask)                                                     \
     mm.x = fmaf(b1, mm.x, omb1 * gg.x); mm.y = fmaf(b1, mm.y, omb1 * gg.y);             \
     mm.z = fmaf(b1, mm.z, omb1 * gg.z); mm.w = fmaf(b1, mm.w, omb1 * gg.w);             \
-    aa.x = mm.x + ((mask & 1u) ? 0.0f : aa.x); aa.y = mm.y + ((mask & 2u) ? 0.0f : aa.y); \
-    aa.z = mm.z + ((mask & 4u) ? 0.0f : aa.z); aa.w = mm.w + ((mask & 8u) ? 0.0f : aa.w);
+    aa.x = fmaf(rho, (mask & 1u) ? 0.0f : aa.x, mm.x); aa.y = fmaf(rho, (mask & 2u) ? 0.0f : aa.y, mm.y); \
+    aa.z = fmaf(rho, (mask & 4u) ? 0.0f : aa.z, mm.z); aa.w = fmaf(rho, (mask & 8u) ? 0.0f : aa.w, mm.w);
 
-// m = beta1 m + (1-beta1) g ; a = m + e (kept in the e buffer; e counts as 0 on I_{t-1}) ;
+// m = beta1 m + (1-beta1) g ; a = m + rho e (kept in the e buffer; e counts as 0 on I_{t-1}; rho = alpha_{t-1}/alpha_t,
+// and fmaf(1, e, m) is m + e to the bit) ;
 // S^(w)[row, h_row(j)] += s_row(j) a_j ; and on I_{t-1} the gradient sum that feeds v and vhat.
 // Vector form: one thread owns 4 consecutive coordinates and walks the workers w0..w0+nw-1, so the hashes are
 // evaluated once per coordinate quad and reused for every worker (all workers share h and s, or the sketches
@@ -63,12 +64,12 @@ k_masked_copy(const float* __restrict__ e, const uint32_t* __restrict__ bitmap, 
 template <int R>
 __global__ void __launch_bounds__(kThreads, 3)
 k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
-    const float4* __restrict__ grads = (const float4*)A.grads;
     float4* m = (float4*)A.m;
     float4* e = (float4*)A.e;
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
     const uint32_t d4 = P.d >> 2;
-    const float b1 = P.beta1, omb1 = 1.0f - P.beta1;
+    const float b1 = P.beta1, omb1 = 1.0f - P.beta1, rho = P.rho;
+    const uint32_t gb = A.grad_bf16;
     const uint64_t tstride = (uint64_t)P.r * P.cs;
     constexpr int RMAX = R > 0 ? R : (int)kMaxRows;
     const uint32_t trips = (d4 + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
@@ -86,7 +87,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
         const uint32_t wend = w0 + nw;
         for (; w + 2 <= wend; w += 2) {                  // two workers per trip: six 16-byte loads in flight
             const uint64_t q0 = (uint64_t)w * d4 + t, q1 = q0 + d4;
-            const float4 g0 = __ldcs(grads + q0), g1 = __ldcs(grads + q1);
+            const float4 g0 = load_grad4(A.grads, q0, gb), g1 = load_grad4(A.grads, q1, gb);
             float4 m0 = __ldcs(m + q0), m1 = __ldcs(m + q1);
             float4 a0 = __ldcs(e + q0), a1 = __ldcs(e + q1);
             SK_MOMENT(m0, a0, g0, mask)
@@ -108,7 +109,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
         }
         if (w < wend) {
             const uint64_t q0 = (uint64_t)w * d4 + t;
-            const float4 g0 = __ldcs(grads + q0);
+            const float4 g0 = load_grad4(A.grads, q0, gb);
             float4 m0 = __ldcs(m + q0);
             float4 a0 = __ldcs(e + q0);
             SK_MOMENT(m0, a0, g0, mask)
@@ -129,25 +130,25 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
 // Parameter averaging (Algorithm 1): every worker keeps its own v and vhat from its own gradient,
 //   m = beta1 m + (1-beta1) g ; v = beta2 v + (1-beta2) g^2 ; vhat = max(vhat, v) ; a = m / sqrt(vhat) + e,
 // and a is what is sketched.  Reads g, m, v, vhat, e and writes m, v, vhat, a: 36 bytes per worker-coordinate.
-__device__ __forceinline__ void pa_moment(float b1, float omb1, float b2, float omb2, float g, float& m, float& v,
-                                          float& vh, float& a, bool masked) {
+__device__ __forceinline__ void pa_moment(float b1, float omb1, float b2, float omb2, float rho, float g, float& m,
+                                          float& v, float& vh, float& a, bool masked) {
     m = fmaf(b1, m, omb1 * g);
     v = fmaf(b2, v, omb2 * g * g);
     vh = fmaxf(vh, v);
-    a = __fdiv_rn(m, __fsqrt_rn(vh)) + (masked ? 0.0f : a);
+    a = fmaf(rho, masked ? 0.0f : a, __fdiv_rn(m, __fsqrt_rn(vh)));
 }
 
 template <int R>
 __global__ void __launch_bounds__(kThreads, 3)
 k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
-    const float4* __restrict__ grads = (const float4*)A.grads;
     float4* m = (float4*)A.m;
     float4* e = (float4*)A.e;
     float4* vw = (float4*)A.vw;
     float4* vhw = (float4*)A.vhatw;
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
     const uint32_t d4 = P.d >> 2;
-    const float b1 = P.beta1, omb1 = 1.0f - P.beta1, b2 = P.beta2, omb2 = 1.0f - P.beta2;
+    const float b1 = P.beta1, omb1 = 1.0f - P.beta1, b2 = P.beta2, omb2 = 1.0f - P.beta2, rho = P.rho;
+    const uint32_t gb = A.grad_bf16;
     const uint64_t tstride = (uint64_t)P.r * P.cs;
     constexpr int RMAX = R > 0 ? R : (int)kMaxRows;
     const uint32_t trips = (d4 + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
@@ -161,12 +162,12 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
         if (A.asum && w0 > 0) as = ((const float4*)A.asum)[t];
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q0 = (uint64_t)w * d4 + t;
-            const float4 g0 = __ldcs(grads + q0);
+            const float4 g0 = load_grad4(A.grads, q0, gb);
             float4 m0 = __ldcs(m + q0), v0 = __ldcs(vw + q0), h0 = __ldcs(vhw + q0), a0 = __ldcs(e + q0);
-            pa_moment(b1, omb1, b2, omb2, g0.x, m0.x, v0.x, h0.x, a0.x, mask & 1u);
-            pa_moment(b1, omb1, b2, omb2, g0.y, m0.y, v0.y, h0.y, a0.y, mask & 2u);
-            pa_moment(b1, omb1, b2, omb2, g0.z, m0.z, v0.z, h0.z, a0.z, mask & 4u);
-            pa_moment(b1, omb1, b2, omb2, g0.w, m0.w, v0.w, h0.w, a0.w, mask & 8u);
+            pa_moment(b1, omb1, b2, omb2, rho, g0.x, m0.x, v0.x, h0.x, a0.x, mask & 1u);
+            pa_moment(b1, omb1, b2, omb2, rho, g0.y, m0.y, v0.y, h0.y, a0.y, mask & 2u);
+            pa_moment(b1, omb1, b2, omb2, rho, g0.z, m0.z, v0.z, h0.z, a0.z, mask & 4u);
+            pa_moment(b1, omb1, b2, omb2, rho, g0.w, m0.w, v0.w, h0.w, a0.w, mask & 8u);
             __stcs(m + q0, m0); __stcs(vw + q0, v0); __stcs(vhw + q0, h0); __stcs(e + q0, a0);
             float* t0 = A.tables + (uint64_t)w * tstride;
 #pragma unroll
@@ -181,7 +182,7 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
 // Scalar form: any d, any alignment, any group size.  One thread per coordinate.
 __global__ void __launch_bounds__(kThreads)
 k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
-    const float b1 = P.beta1, omb1 = 1.0f - P.beta1;
+    const float b1 = P.beta1, omb1 = 1.0f - P.beta1, rho = P.rho;
     const uint64_t tstride = (uint64_t)P.r * P.cs;
     for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads) {
         const bool member = A.members && ((A.bitmap[j >> 5] >> (j & 31u)) & 1u);
@@ -189,16 +190,16 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
         float as = (A.asum && w0 > 0) ? A.asum[j] : 0.0f;
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q = (uint64_t)w * P.d + j;
-            const float g = A.grads[q];
+            const float g = load_grad1(A.grads, q, A.grad_bf16);
             float mm, a;
             if (A.variant == 1) {
                 float vv = A.vw[q], vh = A.vhatw[q];
                 mm = A.m[q]; a = A.e[q];
-                pa_moment(b1, omb1, P.beta2, 1.0f - P.beta2, g, mm, vv, vh, a, member);
+                pa_moment(b1, omb1, P.beta2, 1.0f - P.beta2, rho, g, mm, vv, vh, a, member);
                 A.vw[q] = vv; A.vhatw[q] = vh;
             } else {
                 mm = fmaf(b1, A.m[q], omb1 * g);
-                a = mm + (member ? 0.0f : A.e[q]);
+                a = fmaf(rho, member ? 0.0f : A.e[q], mm);
             }
             gs += g;
             as += a;

@@ -16,6 +16,7 @@
 // every thread of the block takes part in every barrier the same number of times.
 #include "sk_internal.h"
 #include "sk_hash.cuh"
+#include "sk_moment.cuh"
 
 namespace sk {
 
@@ -43,8 +44,8 @@ __device__ __forceinline__ void bar_arrive(uint32_t id, uint32_t count) {
 #define SK_MOMENT(mm, aa, gg, mask)                                                     \
     mm.x = fmaf(b1, mm.x, omb1 * gg.x); mm.y = fmaf(b1, mm.y, omb1 * gg.y);             \
     mm.z = fmaf(b1, mm.z, omb1 * gg.z); mm.w = fmaf(b1, mm.w, omb1 * gg.w);             \
-    aa.x = mm.x + ((mask & 1u) ? 0.0f : aa.x); aa.y = mm.y + ((mask & 2u) ? 0.0f : aa.y); \
-    aa.z = mm.z + ((mask & 4u) ? 0.0f : aa.z); aa.w = mm.w + ((mask & 8u) ? 0.0f : aa.w);
+    aa.x = fmaf(rho, (mask & 1u) ? 0.0f : aa.x, mm.x); aa.y = fmaf(rho, (mask & 2u) ? 0.0f : aa.y, mm.y); \
+    aa.z = fmaf(rho, (mask & 4u) ? 0.0f : aa.z, mm.z); aa.w = fmaf(rho, (mask & 8u) ? 0.0f : aa.w, mm.w);
 
 // units of work item `item`: panel, and the half-open range [t_begin, t_end) of the panel's unit list
 __device__ __forceinline__ void item_range(const Params& P, uint32_t item, uint32_t slices, uint32_t units_total,
@@ -75,11 +76,11 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
 
     if (tid < kProducerThreads) {
         // ------------------------------------------------------------------------------------ producer
-        const float4* __restrict__ grads = (const float4*)A.grads;
         float4* m = (float4*)A.m;
         float4* e = (float4*)A.e;
         const uint32_t d4 = P.d >> 2;
-        const float b1 = P.beta1, omb1 = 1.0f - P.beta1;
+        const float b1 = P.beta1, omb1 = 1.0f - P.beta1, rho = P.rho;
+        const uint32_t gb = A.grad_bf16;
         const uint64_t tstride = (uint64_t)P.r * P.cs;
         uint32_t seq = 0;                                      // units produced by this block so far
         for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
@@ -106,7 +107,7 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                     uint32_t w = 0;
                     for (; w + 2 <= nw; w += 2) {
                         const uint64_t q0 = (uint64_t)(w0 + w) * d4 + t, q1 = q0 + d4;
-                        const float4 g0 = __ldcs(grads + q0), g1 = __ldcs(grads + q1);
+                        const float4 g0 = load_grad4(A.grads, q0, gb), g1 = load_grad4(A.grads, q1, gb);
                         float4 m0 = __ldcs(m + q0), m1 = __ldcs(m + q1);
                         float4 a0 = __ldcs(e + q0), a1 = __ldcs(e + q1);
                         SK_MOMENT(m0, a0, g0, mask)
@@ -127,7 +128,7 @@ k_moment_sketch_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                     }
                     if (w < nw) {
                         const uint64_t q0 = (uint64_t)(w0 + w) * d4 + t;
-                        const float4 g0 = __ldcs(grads + q0);
+                        const float4 g0 = load_grad4(A.grads, q0, gb);
                         float4 m0 = __ldcs(m + q0);
                         float4 a0 = __ldcs(e + q0);
                         SK_MOMENT(m0, a0, g0, mask)

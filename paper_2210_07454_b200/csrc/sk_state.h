@@ -10,6 +10,10 @@ struct TimeRec { int stage; cudaEvent_t a, b; };
 struct sk_state {
     sk::Params P{};
     uint64_t seed = 0, t = 0;
+    uint64_t vclock = 0;          // steps that updated v, vhat: the clock of the lazy decay stamps (t minus frozen steps)
+    float lr_prev = 0;            // alpha_{t-1}: the step size of the last step taken
+    bool freeze_v = false;        // Algorithm 2 without h_t and without the update of v, vhat
+    bool grads_bf16 = false;      // gradients are passed as bf16
     float eps = 0;
     uint32_t k_prev = 0;
     int sm_count = 148;

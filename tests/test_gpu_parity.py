@@ -28,13 +28,15 @@ def _workload(base, **over):
     return w
 
 
-def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga", P=1):
+def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga", P=1, freeze_v=False):
     b = _binding()
     gpu = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
                             eps=w.eps, log2g=log2g, window_lines=window_lines, variant=variant, P=P)
     lg = gpu.get_option("log2g")
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=lg, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
-                        eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"), variant=variant, P=P)
+                        eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"), variant=variant, P=P, freeze_v=freeze_v)
+    if freeze_v:
+        gpu.set_option("freeze_v", 1)
     return gpu, ora
 
 
@@ -73,15 +75,24 @@ def _exact_values(ora, e_before, variant):
 
 
 def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True, window_lines=None, variant="ga",
-               P=1):
-    gpu, ora = _pair(w, log2g, window_lines=window_lines, variant=variant, P=P)
+               P=1, lr_of=None, freeze_v=False, bf16=False):
+    """lr_of: step -> step size (a schedule); bf16: the GPU receives the gradients as bf16, the oracle the same
+    values widened to fp32."""
+    gpu, ora = _pair(w, log2g, window_lines=window_lines, variant=variant, P=P, freeze_v=freeze_v)
+    if bf16:
+        gpu.set_option("grads_bf16", 1)
     src = _source(w, cfg_id=cfg_id)
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
     diverged_at = None
     for t in range(1, steps + 1):
         g = src.grads(t)
-        g_host = g.cpu().numpy()
+        if bf16:
+            g = g.to(torch.bfloat16)
+        g_host = g.float().cpu().numpy()
+        if lr_of is not None:
+            gpu.set_lr(lr_of(t))
+            ora.set_lr(lr_of(t))
         if teacher and t > 1:
             force_state(gpu, ora, variant)
             x_gpu.copy_(torch.from_numpy(x_ref))
@@ -315,6 +326,89 @@ def test_second_round_option_errors():
         gpu.set_option("P", 1)                                # fixed after the first step
     with pytest.raises(b.SkError):
         gpu.select_static(torch.empty(10, dtype=torch.int32, device="cuda"))
+
+
+# ------------------------------------------- step-size schedule, frozen second moments, bf16 gradients (flags)
+def _inv_sqrt(t):
+    return float(np.float32(0.01 / np.sqrt(t)))             # Theorem 2's alpha_t = alpha / sqrt(t)
+
+
+FLAG_CASES = {
+    "schedule": dict(lr_of=_inv_sqrt),
+    "schedule_free_running": dict(lr_of=_inv_sqrt, teacher=False),
+    "schedule_growing_steps": dict(lr_of=lambda t: 1e-3 * 2 ** (t % 3)),     # ratios below and above one
+    "schedule_pa": dict(lr_of=_inv_sqrt, variant="pa"),
+    "schedule_windowed": dict(lr_of=_inv_sqrt, window_lines=4),
+    "schedule_second_round": dict(lr_of=_inv_sqrt, P=2),
+    "frozen": dict(freeze_v=True),
+    "frozen_schedule_second_round": dict(freeze_v=True, lr_of=_inv_sqrt, P=2),
+    "bf16": dict(bf16=True),
+    "bf16_pa": dict(bf16=True, variant="pa"),
+    "bf16_windowed": dict(bf16=True, window_lines=4),
+}
+
+
+@pytest.mark.parametrize("case", sorted(FLAG_CASES))
+def test_flags_c1_steps(case):
+    _run_steps(_workload("C1"), 8, **FLAG_CASES[case])
+
+
+@pytest.mark.parametrize("case", ["schedule", "bf16", "frozen"])
+def test_flags_scalar_path(case):
+    w = _workload("C1", name="E", steps=4, recipe="planted", d=10_007, n=3, r=5, c=1000, k=333)
+    _run_steps(w, 4, cfg_id=7, **FLAG_CASES[case])
+
+
+def test_frozen_second_moments_keep_v_and_its_decay_clock():
+    # v and vhat must not move while frozen (not even the lazy decay), and resume exactly where they were
+    w = _workload("C1", name="E", d=30_000, n=2, r=5, c=2048, k=300, steps=9)
+    gpu, ora = _pair(w)
+    src = _source(w, cfg_id=5)
+    x = src.x0()
+    x_ref = x.cpu().numpy().copy()
+    for t in range(1, 10):
+        frozen = 4 <= t <= 6
+        gpu.set_option("freeze_v", int(frozen))
+        ora.set_freeze_v(frozen)
+        g = src.grads(t)
+        v_before, vhat_before = gpu.get("v"), gpu.get("vhat")
+        gpu.step(g, x)
+        ora.step(g.cpu().numpy(), x_ref)
+        if np.setxor1d(gpu.get("I"), ora.field("I")).size:
+            break
+        if frozen:
+            assert np.array_equal(gpu.get("v"), v_before) and np.array_equal(gpu.get("vhat"), vhat_before)
+        np.testing.assert_allclose(gpu.get("v"), ora.field("v"), rtol=1e-5, atol=0)
+        close(gpu.get("vhat"), ora.field("vhat"), "vhat")
+    else:
+        return
+    pytest.fail("the index sets split before the frozen window was over")
+
+
+def test_flag_errors_and_bf16_host_step():
+    b = _binding()
+    gpu = b.SketchedAMSGrad(4000, 2, 3, 256, 20, lr=0.01)
+    with pytest.raises(b.SkError):
+        gpu.set_lr(float("nan"))
+    with pytest.raises(b.SkError):
+        gpu.set_lr(0.0)                                       # no ratio alpha_{t-1}/alpha_t with a zero step size
+    pa = b.SketchedAMSGrad(4000, 2, 3, 256, 20, variant="pa")
+    with pytest.raises(b.SkError):
+        pa.set_option("freeze_v", 1)                          # Algorithm 2 only
+    # host entry point with bf16 gradients against the device entry point
+    gpu.set_option("grads_bf16", 1)
+    other = b.SketchedAMSGrad(4000, 2, 3, 256, 20, lr=0.01)
+    other.set_option("grads_bf16", 1)
+    assert gpu.algorithmic_bytes() == other.algorithmic_bytes() == 18 * 2 * 4000 + 4 * 4000 + 8 * 2 * 3 * 256 \
+        + 4 * 3 * 256 + 12 * 2 * 20 + 24 * 20
+    g = (torch.randn((2, 4000), device="cuda") * 0.1).to(torch.bfloat16)
+    x_dev = torch.zeros(4000, device="cuda")
+    x_host = np.zeros(4000, np.float32)
+    gpu.step(g, x_dev)
+    other.step_host(g.cpu().view(torch.int16).numpy(), x_host)
+    gpu.sync()
+    assert np.array_equal(gpu.get("I"), other.get("I"))
+    np.testing.assert_allclose(x_host, x_dev.cpu().numpy(), rtol=1e-6, atol=1e-9)
 
 
 def test_worker_chunking_matches_single_pass():

@@ -84,7 +84,7 @@ def _exact_values(ora, e_before, variant):
     return a.mean(axis=0) / np.sqrt(ora.field("vhat").astype(np.float64))
 
 
-def _run(w, split, steps, variant="ga", P=1, window_lines=None, cfg_id=None):
+def _run(w, split, steps, variant="ga", P=1, window_lines=None, cfg_id=None, lr_of=None, bf16=False):
     from paper_2210_07454_b200.synthetic import GradientSource
     ranks = Ranks(w, split, variant=variant, P=P, window_lines=window_lines)
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=ranks.get_option("log2g"), lr=w.lr, beta1=w.beta1,
@@ -93,8 +93,16 @@ def _run(w, split, steps, variant="ga", P=1, window_lines=None, cfg_id=None):
     src = GradientSource(w, device="cuda", cfg_id=cfg_id)
     x_ref = src.x0().cpu().numpy().copy()
     xs = [src.x0() for _ in split]
+    for h in ranks.handles:
+        h.set_option("grads_bf16", int(bf16))
     for t in range(1, steps + 1):
         g = src.grads(t)
+        if bf16:
+            g = g.to(torch.bfloat16)
+        if lr_of is not None:
+            ora.set_lr(lr_of(t))
+            for h in ranks.handles:
+                h.set_lr(lr_of(t))
         if t > 1:                                   # teacher forcing
             force_state(ranks, ora, variant)
             for x in xs:
@@ -104,7 +112,7 @@ def _run(w, split, steps, variant="ga", P=1, window_lines=None, cfg_id=None):
         e_before = ora.field("e").astype(np.float64) if P > 1 else None
         ranks.step(g, xs)
         ranks.sync()
-        ora.step(g.cpu().numpy(), x_ref)
+        ora.step(g.float().cpu().numpy(), x_ref)
         for x in xs[1:]:
             assert torch.equal(x, xs[0]), "the replicas of x disagree"
         compare_step(ranks, ora, xs[0].cpu().numpy(), x_ref, x_before, w.lr, x_gpu_before=x_own, variant=variant,
@@ -125,6 +133,10 @@ def test_c1_second_round(P):
 def test_c1_parameter_averaging():
     _run(_workload(), (2, 2), 6, variant="pa")
     _run(_workload(), (3, 1), 3, variant="pa", P=2)
+
+
+def test_c1_schedule_and_bf16_gradients():
+    _run(_workload(), (2, 2), 6, P=2, lr_of=lambda t: float(np.float32(0.01 / np.sqrt(t))), bf16=True)
 
 
 CASES = {
