@@ -186,6 +186,7 @@ def main():
     ap.add_argument("--partition-workers", action="store_true",
                     help="split the workload's n workers over the processes (one step = three phases with two "
                          "all-reduces between them) instead of running one full replica per process")
+    ap.add_argument("--grads-bf16", action="store_true", help="pass the gradients as bf16 (18 B per worker-coordinate)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-timing", action="store_true")
     args = ap.parse_args()
@@ -217,6 +218,9 @@ def main():
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
                                   eps=w.eps, log2g=args.log2g, window_lines=args.window_lines, variant=args.variant,
                                   P=args.P, workers_total=n_all if args.partition_workers else None)
+    if args.grads_bf16:
+        opt.set_option("grads_bf16", 1)
+    gbytes = 2 if args.grads_bf16 else 4
     step = opt.step
     if args.partition_workers:
         from paper_2210_07454_b200.partitioned import PartitionedStep
@@ -230,9 +234,11 @@ def main():
         opt.set_option("sketch_ctas_per_sm", args.sketch_ctas)
     # gradient buffers rotate so that no step finds its inputs in L2 (each set is far larger than L2 anyway)
     free_b, _ = torch.cuda.mem_get_info()
-    set_bytes = 4 * w.n * w.d
+    set_bytes = gbytes * w.n * w.d
     nsets = args.grad_sets if args.grad_sets > 0 else int(max(2, min(4, (free_b * 0.5) // set_bytes)))
     gsets = [src.grads(t + 1) for t in range(nsets)]
+    if args.grads_bf16:
+        gsets = [g.to(torch.bfloat16) for g in gsets]
     x = src.x0()
     torch.cuda.synchronize()
 
@@ -272,7 +278,7 @@ def main():
     # dominant kernel: moments + sketch.  Algorithmic bytes per launch: 20 B per worker-coordinate streamed
     # (read g, m, e; write m, e) plus the worker tables it fills (4 B per bucket).
     k1_launches = max(1, stage_launches[2])
-    k1_bytes_step = (20 if args.variant == "ga" else 36) * w.n * w.d + 4 * w.n * w.r * w.c
+    k1_bytes_step = ((20 if args.variant == "ga" else 36) - (4 - gbytes)) * w.n * w.d + 4 * w.n * w.r * w.c
     roofline = None
     if not args.no_stage_timing and stage_ms[2] > 0:
         k1_ms = stage_ms[2] / k1_launches
@@ -280,7 +286,8 @@ def main():
         achieved = k1_bytes / (k1_ms * 1e-3) / 1e9
         sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2210_07454_b200", "csrc", "sk_sketch.cu"), "rb").read()).hexdigest()
         traffic = None
-        if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"] and args.variant == "ga":
+        if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"] and args.variant == "ga" \
+                and not args.grads_bf16:
             traffic = NCU_TRAFFIC["bytes_per_worker_coord"] * w.n * w.d * args.steps / k1_launches
         roofline = {"bound": "hbm", "kernel": "k_moment_sketch_v4" if args.variant == "ga" else "k_moment_sketch_pa_v4", "achieved": achieved, "peak": peak,
                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
@@ -290,7 +297,7 @@ def main():
     # end to end through the host entry point: pinned host gradients in, x back out, every step
     e2e = None
     if args.e2e_steps > 0:
-        hg = torch.empty((w.n, w.d), dtype=torch.float32, pin_memory=True)
+        hg = torch.empty((w.n, w.d), dtype=gsets[0].dtype, pin_memory=True)
         hg.copy_(gsets[0])
         hx = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
         hx.copy_(x)
@@ -313,7 +320,7 @@ def main():
         torch.cuda.synchronize()
         dt = reduce_max(time.perf_counter() - t0, world, dev)
         e2e = {"value": units * args.e2e_steps / dt / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": 4 * w.n * w.d + 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
+               "h2d_bytes_per_step": gbytes * w.n * w.d + 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
                "ms_per_step": 1e3 * dt / args.e2e_steps, "steps": args.e2e_steps}
 
     if rank != 0:
@@ -330,7 +337,8 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "strong" if args.partition_workers else "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "d": w.d, "n": n_all, "r": w.r, "c": w.c, "k": w.k,
+            "config": {"gradient_storage": "bf16" if args.grads_bf16 else "f32",
+                       "workload": w.name, "d": w.d, "n": n_all, "r": w.r, "c": w.c, "k": w.k,
                        "recipe": w.recipe, "variant": args.variant, "P": args.P, "hash_group": 1 << opt.get_option("log2g"),
                        "window_lines": opt.get_option("window_lines"),
                        "worker_chunk": opt.get_option("worker_chunk"),

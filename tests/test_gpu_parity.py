@@ -28,7 +28,7 @@ def _workload(base, **over):
     return w
 
 
-def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga", P=1, freeze_v=False):
+def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga", P=1, freeze_v=False, options=None):
     b = _binding()
     gpu = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
                             eps=w.eps, log2g=log2g, window_lines=window_lines, variant=variant, P=P)
@@ -37,6 +37,8 @@ def _pair(w, log2g=None, threads=8, window_lines=None, variant="ga", P=1, freeze
                         eps=w.eps, threads=threads, window_lines=gpu.get_option("window_lines"), variant=variant, P=P, freeze_v=freeze_v)
     if freeze_v:
         gpu.set_option("freeze_v", 1)
+    for key, value in (options or {}).items():
+        gpu.set_option(key, value)
     return gpu, ora
 
 
@@ -75,10 +77,10 @@ def _exact_values(ora, e_before, variant):
 
 
 def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=True, window_lines=None, variant="ga",
-               P=1, lr_of=None, freeze_v=False, bf16=False):
+               P=1, lr_of=None, freeze_v=False, bf16=False, options=None):
     """lr_of: step -> step size (a schedule); bf16: the GPU receives the gradients as bf16, the oracle the same
     values widened to fp32."""
-    gpu, ora = _pair(w, log2g, window_lines=window_lines, variant=variant, P=P, freeze_v=freeze_v)
+    gpu, ora = _pair(w, log2g, window_lines=window_lines, variant=variant, P=P, freeze_v=freeze_v, options=options)
     if bf16:
         gpu.set_option("grads_bf16", 1)
     src = _source(w, cfg_id=cfg_id)
