@@ -31,7 +31,7 @@ DEFAULT_WORKLOAD = "C3"      # d = 25.6M: the size the headline metric is quoted
 # valid only for the kernel source it was taken on (sha256 of sk_sketch.cu); otherwise reported as null.
 # Capture: C3 at half size (profiles/c3_half_moment_sketch_ncu_full.md): 1.2539 GB read + 0.7941 GB written for
 # 1.024e8 worker-coordinates; the traffic grows in proportion to n*d, so it is scaled to the timed launch.
-NCU_TRAFFIC = {"sha256": "d7fcc51852afaab3c176519dbf7d85174eb2aa934de0f0ce02f90c93e0957250",
+NCU_TRAFFIC = {"sha256": "cd14dd6dd7a210877101af2dfc87ea7a5287a14c43fb18384c0f38fa36f03594",
                "bytes_per_worker_coord": 20.00}
 
 
@@ -287,7 +287,7 @@ def main():
         sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2210_07454_b200", "csrc", "sk_sketch.cu"), "rb").read()).hexdigest()
         traffic = None
         if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"] and args.variant == "ga" \
-                and not args.grads_bf16:
+                and not args.grads_bf16 and args.P == 1 and not opt.get_option("window_lines"):
             traffic = NCU_TRAFFIC["bytes_per_worker_coord"] * w.n * w.d * args.steps / k1_launches
         roofline = {"bound": "hbm", "kernel": "k_moment_sketch_v4" if args.variant == "ga" else "k_moment_sketch_pa_v4", "achieved": achieved, "peak": peak,
                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
