@@ -483,27 +483,43 @@ inline int grid_for(uint64_t items, int sm_count, int per_sm) {
 
 }  // namespace
 
+// Persistent grids are sized to what is resident at once (registers and shared memory decide): one block more per
+// SM than fits would run as a second, nearly empty wave after the first.
+template <typename K>
+int resident_per_sm(K kernel, int fallback) {
+    int nb = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, kThreads, 0) != cudaSuccess || nb < 1) {
+        cudaGetLastError();
+        return fallback;
+    }
+    return nb;
+}
+
+#define SK_ROWS_CASE(KERNEL, RR, ...)                                                                      \
+    { auto kfn = KERNEL<RR, true>;                                                                         \
+      kfn<<<grid_for(items, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(__VA_ARGS__); } break;
 #define SK_ROWS_SWITCH(KERNEL, ...)                                                                        \
     switch (P.r) {                                                                                         \
-        case 1: KERNEL<1, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 2: KERNEL<2, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 3: KERNEL<3, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 4: KERNEL<4, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 5: KERNEL<5, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 6: KERNEL<6, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 7: KERNEL<7, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 8: KERNEL<8, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                            \
-        case 10: KERNEL<10, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                          \
-        default: KERNEL<0, true><<<grid, kThreads, 0, st>>>(__VA_ARGS__); break;                           \
+        case 1: SK_ROWS_CASE(KERNEL, 1, __VA_ARGS__)                                                       \
+        case 2: SK_ROWS_CASE(KERNEL, 2, __VA_ARGS__)                                                       \
+        case 3: SK_ROWS_CASE(KERNEL, 3, __VA_ARGS__)                                                       \
+        case 4: SK_ROWS_CASE(KERNEL, 4, __VA_ARGS__)                                                       \
+        case 5: SK_ROWS_CASE(KERNEL, 5, __VA_ARGS__)                                                       \
+        case 6: SK_ROWS_CASE(KERNEL, 6, __VA_ARGS__)                                                       \
+        case 7: SK_ROWS_CASE(KERNEL, 7, __VA_ARGS__)                                                       \
+        case 8: SK_ROWS_CASE(KERNEL, 8, __VA_ARGS__)                                                       \
+        case 10: SK_ROWS_CASE(KERNEL, 10, __VA_ARGS__)                                                     \
+        default: SK_ROWS_CASE(KERNEL, 0, __VA_ARGS__)                                                      \
     }
 
 int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum, uint32_t* keys, uint32_t* hist,
                          bool vec, int sm_count, cudaStream_t st) {
     if (!vec) {
-        k_unsketch_hist<0, false><<<grid_for(P.d, sm_count, 6), kThreads, 0, st>>>(P, A, sum, keys, hist);
+        auto kfn = k_unsketch_hist<0, false>;
+        kfn<<<grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P, A, sum, keys, hist);
         return 1;
     }
-    const int grid = grid_for(P.d >> 2, sm_count, 6);
+    const uint64_t items = P.d >> 2;
     SK_ROWS_SWITCH(k_unsketch_hist, P, A, sum, keys, hist)
     return 1;
 }
@@ -515,16 +531,21 @@ int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cud
 
 int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, Select* sel, uint32_t* I_out, Cand* cand,
                 uint32_t* hist2, int sm_count, cudaStream_t st) {
-    if (P.d % 4 == 0 && !idx_map)
-        k_emit<true><<<grid_for((P.d >> 2) / 4 + 1, sm_count, 8), kThreads, 0, st>>>(P.d, keys, nullptr, sel, I_out, cand, hist2);
-    else
-        k_emit<false><<<grid_for(P.d, sm_count, 8), kThreads, 0, st>>>(P.d, keys, idx_map, sel, I_out, cand, hist2);
+    if (P.d % 4 == 0 && !idx_map) {
+        auto kfn = k_emit<true>;
+        kfn<<<grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P.d, keys, nullptr, sel, I_out,
+                                                                                                   cand, hist2);
+    } else {
+        auto kfn = k_emit<false>;
+        kfn<<<grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P.d, keys, idx_map, sel, I_out, cand, hist2);
+    }
     return 1;
 }
 
 int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const float* vhat, const float* e,
                       const float* asum, uint32_t* keys2, uint32_t* hist, int sm_count, cudaStream_t st) {
-    k_exact_keys<<<grid_for(count, sm_count, 8), kThreads, 0, st>>>(P, C, count, vhat, e, asum, keys2, hist);
+    k_exact_keys<<<grid_for(count, sm_count, resident_per_sm(k_exact_keys, 4)), kThreads, 0, st>>>(P, C, count, vhat, e, asum,
+                                                                                                  keys2, hist);
     return 1;
 }
 
