@@ -13,6 +13,9 @@
  *   x_j      -= lr * mean_w a_t^(w)_j / sqrt(vhat_t,j)   for j in I_t           (exact values, Section III-A)
  *   e_t^(w)   = a_t^(w) off I_t, 0 on I_t                                       (error feedback)
  * v_0 = vhat_0 = eps (an initial value, not a denominator term), m_0 = e_0 = 0, I_0 = empty.
+ * Options widen this to the rest of the method: Algorithm 1 ("variant"), the second selection round of
+ * Section III-A ("P"), a step-size schedule (sk_set_lr), frozen second moments ("freeze_v"), bf16 gradients
+ * ("grads_bf16"), and the workers partitioned over several GPUs (sk_step_local / _select / _finish).
  *
  * Conventions for every entry point:
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are ordinary memory.
@@ -159,7 +162,9 @@ int sk_set(sk_state* state, const char* field, const void* buf, uint64_t bytes);
 
 /* Bytes one step must move by the method's own definition, used as the roofline numerator:
  * 20*n*d (read g,m,e; write m,e) + 4*d (vhat) + 8*n*r*c + 4*r*c (worker tables written and read, aggregate
- * written) + 12*n*k + 24*k (sparse gathers and updates on I_{t-1} and I_t). */
+ * written) + 12*n*k + 24*k (sparse gathers and updates on I_{t-1} and I_t).  Algorithm 1: 36*n*d (g, m, v, vhat, e
+ * in; m, v, vhat, e out) and no master-side second moments.  bf16 gradients: 2 bytes less per worker-coordinate.
+ * Second round: P*k*(4n + 12) more (candidate index, the n workers' values and vhat in, the exact value out). */
 uint64_t sk_algorithmic_bytes(const sk_state* state);
 
 /* Stage timing (option "timing" = 1).  Stages: 0 zero tables, 1 unused (the second moments on I_{t-1} are updated
@@ -180,7 +185,8 @@ int sk_get_timing(sk_state* state, double* ms, uint64_t* launches);
  * all its scratch (histograms, ranking keys, candidate lists; about 5 MB) lives in one file-scope device array
  * inside the library, which every GPU that loads the library holds until the process exits.
  *   - Limit: d <= SK_STATIC_MAX_D; larger handles are rejected with SK_EINVAL and a message naming the limit.
- *     SK_ESTATE if the handle has not taken a step yet.
+ *     SK_ESTATE if the handle has not taken a step yet, or runs a second round (P > 1), whose exact values
+ *     this entry point does not fetch.
  *   - The first call on a device resolves the device address of the scratch array (once per device, with that
  *     device current).  Make that first call before starting any stream capture.
  *   - Every call, from every handle and stream, shares the one array, and the array keeps the previous call's
