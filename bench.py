@@ -186,6 +186,8 @@ def main():
     ap.add_argument("--partition-workers", action="store_true",
                     help="split the workload's n workers over the processes (one step = three phases with two "
                          "all-reduces between them) instead of running one full replica per process")
+    ap.add_argument("--sum-sketch", action="store_true",
+                    help="NOT the headline path: one sketch of the worker sum instead of n sketches and their sum")
     ap.add_argument("--grads-bf16", action="store_true", help="pass the gradients as bf16 (18 B per worker-coordinate)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stage-timing", action="store_true")
@@ -218,6 +220,8 @@ def main():
     opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2,
                                   eps=w.eps, log2g=args.log2g, window_lines=args.window_lines, variant=args.variant,
                                   P=args.P, workers_total=n_all if args.partition_workers else None)
+    if args.sum_sketch:
+        opt.set_option("sum_sketch", 1)
     if args.grads_bf16:
         opt.set_option("grads_bf16", 1)
     gbytes = 2 if args.grads_bf16 else 4
@@ -278,7 +282,8 @@ def main():
     # dominant kernel: moments + sketch.  Algorithmic bytes per launch: 20 B per worker-coordinate streamed
     # (read g, m, e; write m, e) plus the worker tables it fills (4 B per bucket).
     k1_launches = max(1, stage_launches[2])
-    k1_bytes_step = ((20 if args.variant == "ga" else 36) - (4 - gbytes)) * w.n * w.d + 4 * w.n * w.r * w.c
+    k1_bytes_step = ((20 if args.variant == "ga" else 36) - (4 - gbytes)) * w.n * w.d \
+        + 4 * (1 if args.sum_sketch else w.n) * w.r * w.c
     roofline = None
     if not args.no_stage_timing and stage_ms[2] > 0:
         k1_ms = stage_ms[2] / k1_launches
@@ -287,7 +292,7 @@ def main():
         sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2210_07454_b200", "csrc", "sk_sketch.cu"), "rb").read()).hexdigest()
         traffic = None
         if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"] and args.variant == "ga" \
-                and not args.grads_bf16 and args.P == 1 and not opt.get_option("window_lines"):
+                and not args.grads_bf16 and not args.sum_sketch and args.P == 1 and not opt.get_option("window_lines"):
             traffic = NCU_TRAFFIC["bytes_per_worker_coord"] * w.n * w.d * args.steps / k1_launches
         roofline = {"bound": "hbm", "kernel": "k_moment_sketch_v4" if args.variant == "ga" else "k_moment_sketch_pa_v4", "achieved": achieved, "peak": peak,
                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
@@ -337,7 +342,8 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "strong" if args.partition_workers else "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"gradient_storage": "bf16" if args.grads_bf16 else "f32",
+            "config": {"sketches": "one, of the worker sum (linearity; not the headline path)" if args.sum_sketch
+                       else "one per worker, then summed", "gradient_storage": "bf16" if args.grads_bf16 else "f32",
                        "workload": w.name, "d": w.d, "n": n_all, "r": w.r, "c": w.c, "k": w.k,
                        "recipe": w.recipe, "variant": args.variant, "P": args.P, "hash_group": 1 << opt.get_option("log2g"),
                        "window_lines": opt.get_option("window_lines"),

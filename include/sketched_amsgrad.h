@@ -112,6 +112,12 @@ int sk_sync(sk_state* state);
  *                  estimates become candidates, their exact values are fetched from the workers' vectors, and the
  *                  k candidates of largest exact magnitude form I_t (ties: smaller index).  1 (default) = no second
  *                  round.  P*k <= d.  Only before the first step.  The candidates of the last step are field "cand".
+ *   "sum_sketch"   1: the n per-worker sketches and their sum are replaced by ONE sketch of the worker sum,
+ *                  S((1/n) sum_w a^(w)), which equals (1/n) sum_w S(a^(w)) because the sketch is linear (Section II-C;
+ *                  the two differ only in the rounding of fp32 sums).  The per-worker tables are then not formed
+ *                  (sk_get "tables" fails) -- they are what a worker would transmit, so this is for a single GPU
+ *                  holding all workers, or for the local share of a partitioned step.  Default 0: n sketches.
+ *                  Uses the reduction kernel (not the shared-memory windows).  Any time between steps.
  *   "freeze_v"     1: Algorithm 2 without h_t and without the update of v and vhat, which keep the values they have
  *                  (set them with sk_set "v", "vhat"): the fixed-variance scheme Section III-B reduces the method
  *                  to.  0 (default) resumes the updates.  Gradient averaging only.  Any time between steps.

@@ -136,7 +136,8 @@ int phase_local(sk_state* s, const void* grads, float* x1) {
     if (s->timing && s->recs.size() > 4096) { int rc = flush_timing(s); if (rc) return rc; }
 
     sk::MomentArgs A = moment_args(s, grads);
-    const bool windowed = vec && P.win_cw != 0 && s->variant == 0;   // the windowed kernel implements Algorithm 2 only
+    // the windowed kernel implements Algorithm 2 with one table per worker only
+    const bool windowed = vec && P.win_cw != 0 && s->variant == 0 && !s->sum_sketch;
     const uint32_t wc = windowed ? std::min<uint32_t>((uint32_t)s->window_workers, P.n) : chunk_of(s);
     // With a second round the sketch kernel also leaves sum_w a^(w) per coordinate, so that each of the P*k exact
     // values costs one gather instead of n (not the windowed kernel, and not a partitioned step, whose exact values
@@ -144,13 +145,19 @@ int phase_local(sk_state* s, const void* grads, float* x1) {
     A.asum = (s->cand_mult > 1 && !windowed && !sharded) ? s->asum : nullptr;
     s->asum_live = A.asum != nullptr;
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
+    float* sum_out = sharded ? x1 : s->sum;
+    if (s->sum_sketch) {             // one sketch of the worker sum, accumulated straight into the aggregate
+        A.sum_table = sum_out;
+        StageTimer tm(s, 0);
+        tm.done(sk::launch_zero(sum_out, tfloats * 4, st));
+    }
     if (sharded && s->k_prev) {      // I_{t-1} in ascending order, from its bitmap
         StageTimer tm(s, 0);
         tm.done(sk::launch_list_from_bitmap(s->bitmap, s->bitmap_bytes / 4, s->scan, s->I_prev, st));
     }
     for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
         const uint32_t nw = std::min(wc, P.n - w0);
-        {
+        if (!s->sum_sketch) {
             StageTimer tm(s, 0);
             tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats * 4, st));
         }
@@ -166,7 +173,7 @@ int phase_local(sk_state* s, const void* grads, float* x1) {
     }
     {
         StageTimer tm(s, 3);
-        int l = sk::launch_sum_tables(P, s->tables, sharded ? x1 : s->sum, st);
+        int l = s->sum_sketch ? 0 : sk::launch_sum_tables(P, s->tables, sum_out, st);
         if (sharded && s->variant == 0)      // h_t: this process's gradient sums on I_{t-1}, zero-padded to k
             l += sk::launch_gather(s->I_prev, s->k_prev, P.k, s->gsum, x1 + tfloats, st);
         tm.done(l);
@@ -492,6 +499,12 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         s->cand_mult = value;
         return SK_OK;
     }
+    if (!strcmp(key, "sum_sketch")) {
+        if (value != 0 && value != 1) return fail(SK_EINVAL, "sum_sketch must be 0 or 1");
+        if (s->phase != 0) return fail(SK_ESTATE, "sum_sketch cannot change inside a partitioned step");
+        s->sum_sketch = value != 0;
+        return SK_OK;
+    }
     if (!strcmp(key, "freeze_v")) {
         if (value != 0 && s->variant == 1) return fail(SK_EINVAL, "freeze_v applies to gradient averaging (Algorithm 2) only");
         if (s->phase != 0) return fail(SK_ESTATE, "freeze_v cannot change inside a partitioned step");
@@ -565,6 +578,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     else if (!strcmp(key, "P")) *value = s->cand_mult;
     else if (!strcmp(key, "workers_total")) *value = s->P.n_all;
     else if (!strcmp(key, "freeze_v")) *value = s->freeze_v;
+    else if (!strcmp(key, "sum_sketch")) *value = s->sum_sketch;
     else if (!strcmp(key, "grads_bf16")) *value = s->grads_bf16;
     else if (!strcmp(key, "window_red_rows")) *value = s->window_red_rows;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
@@ -589,11 +603,12 @@ uint64_t sk_algorithmic_bytes(const sk_state* s) {
     if (!s) return 0;
     const uint64_t n = s->P.n, d = s->P.d, r = s->P.r, c = s->P.c, k = s->P.k;
     const uint64_t g = s->grads_bf16 ? 2 : 0;     // bytes saved per gradient entry when they arrive as bf16
+    const uint64_t tables = s->sum_sketch ? 8 * r * c : 8 * n * r * c + 4 * r * c;   // one table instead of n + 1
     // second round: per candidate, its index, the n workers' values (and vhat) in, its exact value out
     const uint64_t second = s->cand_mult > 1 ? (uint64_t)s->cand_mult * k * (4 * n + (s->variant == 1 ? 8 : 12)) : 0;
     if (s->variant == 1)     // Algorithm 1: read g,m,v,vhat,e and write m,v,vhat,e; no master-side second moments
-        return (36 - g) * n * d + 8 * n * r * c + 4 * r * c + 8 * n * k + 8 * k + second;
-    return (20 - g) * n * d + 4 * d + 8 * n * r * c + 4 * r * c + 12 * n * k + 24 * k + second;
+        return (36 - g) * n * d + tables + 8 * n * k + 8 * k + second;
+    return (20 - g) * n * d + 4 * d + tables + 12 * n * k + 24 * k + second;
 }
 
 int sk_get_timing(sk_state* s, double* ms, uint64_t* launches) {

@@ -45,6 +45,8 @@ struct MomentArgs {
     const void* grads;       // n*d gradient entries, fp32 or (grad_bf16 != 0) bf16
     uint32_t grad_bf16;
     float *m, *e, *tables;
+    float* sum_table;        // not nullptr: sketch the worker sum of a_t once into this r x cs table (already divided by
+                             // n_all) instead of one table per worker -- the sketch is linear (Section II-C)
     float* asum;             // d or nullptr: running sum over the workers of a_t, in worker order (second round of Section III-A)
     float* gsum;             // running gradient sums on I_{t-1} when the workers are processed in several launches
     float *v, *vhat;

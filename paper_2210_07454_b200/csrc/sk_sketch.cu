@@ -55,6 +55,28 @@ k_masked_copy(const float* __restrict__ e, const uint32_t* __restrict__ bitmap, 
     aa.x = fmaf(rho, (mask & 1u) ? 0.0f : aa.x, mm.x); aa.y = fmaf(rho, (mask & 2u) ? 0.0f : aa.y, mm.y); \
     aa.z = fmaf(rho, (mask & 4u) ? 0.0f : aa.z, mm.z); aa.w = fmaf(rho, (mask & 8u) ? 0.0f : aa.w, mm.w);
 
+// Option: S_t = (1/n) sum_w S(a^(w)) = S((1/n) sum_w a^(w)) because the sketch is linear (Section II-C), so one sketch
+// of the worker sum replaces the n per-worker sketches and their sum.  `as` is the sum over this launch's workers.
+// The exact values of Section III-A's second round are read from asum = sum_w a^(w): each launch adds its workers'
+// sum to what the earlier launches of the step left there.
+__device__ __forceinline__ void store_worker_sum(const MomentArgs& A, uint32_t t, float4 as, uint32_t w0) {
+    if (w0 > 0) {
+        const float4 prev = ((const float4*)A.asum)[t];
+        as.x += prev.x; as.y += prev.y; as.z += prev.z; as.w += prev.w;
+    }
+    ((float4*)A.asum)[t] = as;
+}
+
+template <int RMAX>
+__device__ __forceinline__ void sketch_of_sum(const Params& P, const MomentArgs& A, uint32_t r, const Quad (&h)[RMAX],
+                                              float4 as) {
+    const float fn = (float)P.n_all;
+    as.x = as.x / fn; as.y = as.y / fn; as.z = as.z / fn; as.w = as.w / fn;
+#pragma unroll
+    for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+        if (row < r) red_add_v4(A.sum_table + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], as));
+}
+
 // m = beta1 m + (1-beta1) g ; a = m + rho e (kept in the e buffer; e counts as 0 on I_{t-1}; rho = alpha_{t-1}/alpha_t,
 // and fmaf(1, e, m) is m + e to the bit) ;
 // S^(w)[row, h_row(j)] += s_row(j) a_j ; and on I_{t-1} the gradient sum that feeds v and vhat.
@@ -81,8 +103,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
         const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
         float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);     // running gradient sum in worker order (used on I_{t-1})
         if (mask && w0 > 0) gs = ((const float4*)A.gsum)[t];
-        float4 as = make_float4(0.f, 0.f, 0.f, 0.f);     // running sum of a in worker order: the exact values of
-        if (A.asum && w0 > 0) as = ((const float4*)A.asum)[t];   // Section III-A's second round reads them from it
+        float4 as = make_float4(0.f, 0.f, 0.f, 0.f);     // sum of a over this launch's workers, in worker order
         uint32_t w = w0;
         const uint32_t wend = w0 + nw;
         for (; w + 2 <= wend; w += 2) {                  // two workers per trip: six 16-byte loads in flight
@@ -100,12 +121,14 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             __stcs(e + q0, a0); __stcs(e + q1, a1);
             float* t0 = A.tables + (uint64_t)w * tstride;
             float* t1 = t0 + tstride;
+            if (!A.sum_table) {
 #pragma unroll
-            for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
-                if (row < r) {
-                    red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
-                    red_add_v4(t1 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a1));
-                }
+                for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+                    if (row < r) {
+                        red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+                        red_add_v4(t1 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a1));
+                    }
+            }
         }
         if (w < wend) {
             const uint64_t q0 = (uint64_t)w * d4 + t;
@@ -118,12 +141,15 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             __stcs(m + q0, m0);
             __stcs(e + q0, a0);
             float* t0 = A.tables + (uint64_t)w * tstride;
+            if (!A.sum_table) {
 #pragma unroll
-            for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
-                if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+                for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+                    if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+            }
         }
         if (mask) ((float4*)A.gsum)[t] = gs;             // consumed by the key pass (or by the next launch)
-        if (A.asum) ((float4*)A.asum)[t] = as;
+        if (A.sum_table) sketch_of_sum<RMAX>(P, A, r, h, as);
+        if (A.asum) store_worker_sum(A, t, as, w0);
     }
 }
 
@@ -158,8 +184,7 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
         quad_hashes<RMAX>(P, r, t < d4 ? t : d4 - 1, h);
         if (t >= d4) continue;
         const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
-        float4 as = make_float4(0.f, 0.f, 0.f, 0.f);     // running sum of a in worker order
-        if (A.asum && w0 > 0) as = ((const float4*)A.asum)[t];
+        float4 as = make_float4(0.f, 0.f, 0.f, 0.f);     // sum of a over this launch's workers, in worker order
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q0 = (uint64_t)w * d4 + t;
             const float4 g0 = load_grad4(A.grads, q0, gb);
@@ -170,12 +195,15 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
             pa_moment(b1, omb1, b2, omb2, rho, g0.w, m0.w, v0.w, h0.w, a0.w, mask & 8u);
             __stcs(m + q0, m0); __stcs(vw + q0, v0); __stcs(vhw + q0, h0); __stcs(e + q0, a0);
             float* t0 = A.tables + (uint64_t)w * tstride;
+            if (!A.sum_table) {
 #pragma unroll
-            for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
-                if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+                for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+                    if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+            }
             as.x += a0.x; as.y += a0.y; as.z += a0.z; as.w += a0.w;
         }
-        if (A.asum) ((float4*)A.asum)[t] = as;
+        if (A.sum_table) sketch_of_sum<RMAX>(P, A, r, h, as);
+        if (A.asum) store_worker_sum(A, t, as, w0);
     }
 }
 
@@ -187,7 +215,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
     for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads) {
         const bool member = A.members && ((A.bitmap[j >> 5] >> (j & 31u)) & 1u);
         float gs = (member && w0 > 0) ? A.gsum[j] : 0.0f;
-        float as = (A.asum && w0 > 0) ? A.asum[j] : 0.0f;
+        float as = 0.0f;                             // sum of a over this launch's workers
         for (uint32_t w = w0; w < w0 + nw; ++w) {
             const uint64_t q = (uint64_t)w * P.d + j;
             const float g = load_grad1(A.grads, q, A.grad_bf16);
@@ -205,14 +233,22 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
             as += a;
             A.m[q] = mm;
             A.e[q] = a;
-            for (uint32_t row = 0; row < P.r; ++row) {
+            for (uint32_t row = 0; row < P.r && !A.sum_table; ++row) {
                 uint32_t b; float s;
                 coord_hash(P, P.row_key[row], j, b, s);
                 atomicAdd(A.tables + (uint64_t)w * tstride + (uint64_t)row * P.cs + b, s * a);
             }
         }
         if (member && A.variant == 0) A.gsum[j] = gs;
-        if (A.asum) A.asum[j] = as;
+        if (A.asum) A.asum[j] = (w0 > 0 ? A.asum[j] : 0.0f) + as;
+        if (A.sum_table) {
+            const float share = as / (float)P.n_all;
+            for (uint32_t row = 0; row < P.r; ++row) {
+                uint32_t b; float s;
+                coord_hash(P, P.row_key[row], j, b, s);
+                atomicAdd(A.sum_table + (uint64_t)row * P.cs + b, s * share);
+            }
+        }
     }
 }
 

@@ -12,6 +12,7 @@ struct sk_state {
     uint64_t seed = 0, t = 0;
     uint64_t vclock = 0;          // steps that updated v, vhat: the clock of the lazy decay stamps (t minus frozen steps)
     float lr_prev = 0;            // alpha_{t-1}: the step size of the last step taken
+    bool sum_sketch = false;      // sketch the worker sum once instead of one table per worker (linearity)
     bool freeze_v = false;        // Algorithm 2 without h_t and without the update of v, vhat
     bool grads_bf16 = false;      // gradients are passed as bf16
     float eps = 0;

@@ -413,6 +413,54 @@ def test_flag_errors_and_bf16_host_step():
     np.testing.assert_allclose(x_host, x_dev.cpu().numpy(), rtol=1e-6, atol=1e-9)
 
 
+# -------------------------------------------- one sketch of the worker sum instead of n sketches (option sum_sketch)
+SUM_SKETCH = {
+    "c1": dict(),
+    "c1_second_round": dict(P=2),
+    "c1_pa": dict(variant="pa"),
+    "c1_windowed_family": dict(window_lines=4),                 # the family, with the reduction kernel
+    "c1_schedule_bf16": dict(lr_of=_inv_sqrt, bf16=True),
+    "chunked_workers": dict(over=dict(d=30_000, n=7, r=16, c=1001, k=300), options={"worker_chunk": 3}),
+    "chunked_workers_second_round": dict(over=dict(d=40_000, n=6, r=5, c=2048, k=400), options={"worker_chunk": 4}, P=3),
+    "scalar_path": dict(over=dict(d=10_007, n=3, r=5, c=1000, k=333)),
+}
+
+
+@pytest.mark.parametrize("case", sorted(SUM_SKETCH))
+def test_sketch_of_the_worker_sum(case):
+    cfg = dict(SUM_SKETCH[case])
+    over = cfg.pop("over", None)
+    options = dict(cfg.pop("options", {}), sum_sketch=1)
+    w = _workload("C1", name="E", steps=4, recipe="planted", **over) if over else _workload("C1")
+    _run_steps(w, 4, cfg_id=7 if over else None, options=options, check_tables=False, **cfg)
+
+
+def test_sketch_of_the_worker_sum_integer_inputs_bit_exact():
+    d, n, r, c, k = 200_000, 4, 5, 4096, 1000
+    b = _binding()
+    gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0)
+    gpu.set_option("sum_sketch", 1)
+    ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=gpu.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
+                        threads=8)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    x = torch.zeros(d, device="cuda")
+    x_ref = np.zeros(d, np.float32)
+    for step in range(2):
+        g = torch.randint(-8, 9, (n, d), generator=gen, device="cuda").float()
+        gpu.step(g, x)
+        gpu.sync()
+        ora.step(g.cpu().numpy(), x_ref)
+        assert np.array_equal(gpu.get("sum"), ora.field("sum"))       # n = 4: every quotient and sum is exact
+        assert np.array_equal(gpu.get("I"), ora.field("I"))
+        assert np.array_equal(gpu.get("e"), ora.field("e"))
+        if step == 0:                                                  # vhat = 1 still: the update is exact too
+            assert np.array_equal(x.cpu().numpy(), x_ref)
+        x.copy_(torch.from_numpy(x_ref))
+    with pytest.raises(b.SkError):
+        gpu.get("tables")                                              # not formed in this mode
+    assert gpu.algorithmic_bytes() == 20 * n * d + 4 * d + 8 * r * c + 12 * n * k + 24 * k
+
+
 def test_worker_chunking_matches_single_pass():
     w = _workload("C1", name="E", d=40_000, n=6, r=5, c=2048, k=400)
     b = _binding()

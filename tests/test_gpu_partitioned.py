@@ -135,6 +135,35 @@ def test_c1_parameter_averaging():
     _run(_workload(), (3, 1), 3, variant="pa", P=2)
 
 
+def test_c1_sketch_of_the_local_worker_sum():
+    # each process sketches the sum of its own workers once: the exchanged share of the mean sketch is the same vector
+    from paper_2210_07454_b200 import synthetic  # noqa: F401
+    w = _workload()
+    from paper_2210_07454_b200.synthetic import GradientSource
+    ranks = Ranks(w, (3, 1), P=2)
+    for h in ranks.handles:
+        h.set_option("sum_sketch", 1)
+    ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=ranks.get_option("log2g"), lr=w.lr, beta1=w.beta1,
+                        beta2=w.beta2, eps=w.eps, threads=8, P=2)
+    src = GradientSource(w, device="cuda")
+    x_ref = src.x0().cpu().numpy().copy()
+    xs = [src.x0() for _ in ranks.handles]
+    for t in range(1, 5):
+        g = src.grads(t)
+        if t > 1:
+            force_state(ranks, ora, "ga")
+            for x in xs:
+                x.copy_(torch.from_numpy(x_ref))
+        x_before = x_ref.astype(np.float64).copy()
+        x_own = xs[0].cpu().numpy().copy()
+        e_before = ora.field("e").astype(np.float64)
+        ranks.step(g, xs)
+        ranks.sync()
+        ora.step(g.cpu().numpy(), x_ref)
+        compare_step(ranks, ora, xs[0].cpu().numpy(), x_ref, x_before, w.lr, check_tables=False, x_gpu_before=x_own,
+                     exact_ref=_exact_values(ora, e_before, "ga"))
+
+
 def test_c1_schedule_and_bf16_gradients():
     _run(_workload(), (2, 2), 6, P=2, lr_of=lambda t: float(np.float32(0.01 / np.sqrt(t))), bf16=True)
 
