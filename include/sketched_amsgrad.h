@@ -65,8 +65,11 @@ int sk_step(const void* grads, float* x, sk_state* state);
 int sk_set_lr(sk_state* state, float lr);
 
 /* Same step with HOST buffers: copies grads (n*d) to an internal device staging buffer and x (d) in,
- * runs the step, copies x back, and synchronises the stream.  Pinned host memory makes the copies faster
- * but is not required.  The staging buffers are allocated on first use and freed by sk_destroy. */
+ * runs the step, copies x back, and synchronises the stream.  The gradients are copied in up to four pieces of
+ * whole workers on an internal copy stream and the sketch kernel starts on each piece as it arrives, so most of
+ * the kernel time hides behind the transfer; with pageable memory the copies simply serialise.  Pinned host
+ * memory makes the copies faster but is not required.  The staging buffers, the copy stream and its events are
+ * created on first use and released by sk_destroy. */
 int sk_step_host(const void* grads_host, float* x_host, sk_state* state);
 
 /* ---- One iteration with the WORKERS PARTITIONED over several processes (one GPU each) -----------------------------

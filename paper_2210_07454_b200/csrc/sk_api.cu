@@ -126,14 +126,19 @@ sk::MomentArgs moment_args(const sk_state* s, const void* grads) {
 // the candidates]; both index lists are in ascending order so that position q means the same coordinate everywhere.
 
 // Phase 1 (workers): moments, error-compensated vector, sketches of this handle's workers, their sum.
-int phase_local(sk_state* s, const void* grads, float* x1) {
+// [wbeg, wend): the workers this call covers; a step may take the phase in several calls over ascending worker ranges
+// (the host-buffer step does, one call per gradient piece that has arrived): the first call opens the phase, the
+// one that reaches the last worker closes it.
+int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, uint32_t wend = 0xFFFFFFFFu) {
     // alpha_{t-1}/alpha_t weights e_{t-1} in the sketched vector (the sketch lines of Algorithms 1 and 2)
     s->P.rho = (s->lr_prev == s->P.lr) ? 1.0f : (float)((double)s->lr_prev / (double)s->P.lr);
     const sk::Params& P = s->P;
     const bool vec = s->step_vec;
     const bool sharded = x1 != nullptr;
     cudaStream_t st = s->stream;
-    if (s->timing && s->recs.size() > 4096) { int rc = flush_timing(s); if (rc) return rc; }
+    wend = std::min(wend, P.n);
+    const bool first = wbeg == 0, last = wend == P.n;
+    if (first && s->timing && s->recs.size() > 4096) { int rc = flush_timing(s); if (rc) return rc; }
 
     sk::MomentArgs A = moment_args(s, grads);
     // the windowed kernel implements Algorithm 2 with one table per worker only
@@ -146,17 +151,17 @@ int phase_local(sk_state* s, const void* grads, float* x1) {
     s->asum_live = A.asum != nullptr;
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     float* sum_out = sharded ? x1 : s->sum;
-    if (s->sum_sketch) {             // one sketch of the worker sum, accumulated straight into the aggregate
-        A.sum_table = sum_out;
+    if (s->sum_sketch) A.sum_table = sum_out;
+    if (s->sum_sketch && first) {    // one sketch of the worker sum, accumulated straight into the aggregate
         StageTimer tm(s, 0);
         tm.done(sk::launch_zero(sum_out, tfloats * 4, st));
     }
-    if (sharded && s->k_prev) {      // I_{t-1} in ascending order, from its bitmap
+    if (sharded && s->k_prev && first) {      // I_{t-1} in ascending order, from its bitmap
         StageTimer tm(s, 0);
         tm.done(sk::launch_list_from_bitmap(s->bitmap, s->bitmap_bytes / 4, s->scan, s->I_prev, st));
     }
-    for (uint32_t w0 = 0; w0 < P.n; w0 += wc) {
-        const uint32_t nw = std::min(wc, P.n - w0);
+    for (uint32_t w0 = wbeg; w0 < wend; w0 += wc) {
+        const uint32_t nw = std::min(wc, wend - w0);
         if (!s->sum_sketch) {
             StageTimer tm(s, 0);
             tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats * 4, st));
@@ -171,7 +176,7 @@ int phase_local(sk_state* s, const void* grads, float* x1) {
             tm.done(sk::launch_moment_sketch(P, A, w0, nw, vec, s->sm_count * (int)s->sketch_ctas_per_sm, st));
         }
     }
-    {
+    if (last) {
         StageTimer tm(s, 3);
         int l = s->sum_sketch ? 0 : sk::launch_sum_tables(P, s->tables, sum_out, st);
         if (sharded && s->variant == 0)      // h_t: this process's gradient sums on I_{t-1}, zero-padded to k
@@ -377,6 +382,11 @@ void sk_destroy(sk_state* s) {
                     (void*)s->keys, (void*)s->gsum, (void*)s->asum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw, (void*)s->Ic, (void*)s->keys2, (void*)s->cbitmap, (void*)s->scan,
                     (void*)s->stage_grads, (void*)s->stage_x})
         if (p) cudaFree(p);
+    if (s->copy_stream) {
+        cudaStreamSynchronize(s->copy_stream);
+        cudaStreamDestroy(s->copy_stream);
+        for (cudaEvent_t ev : s->copy_done) if (ev) cudaEventDestroy(ev);
+    }
     for (const TimeRec& r : s->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (cudaEvent_t e : s->free_events) cudaEventDestroy(e);
     delete s;
@@ -391,14 +401,40 @@ int sk_step(const void* grads, float* x, sk_state* s) {
 int sk_step_host(const void* grads_host, float* x_host, sk_state* s) {
     if (!s || !grads_host || !x_host) return fail(SK_EINVAL, "sk_step_host: null argument");
     const uint64_t nd = (uint64_t)s->P.n * s->P.d;
-    const uint64_t gbytes = nd * (s->grads_bf16 ? 2 : 4);
     if (!s->stage_grads) {
         SK_CUDA(cudaMalloc((void**)&s->stage_grads, nd * 4));
         SK_CUDA(cudaMalloc((void**)&s->stage_x, (uint64_t)s->P.d * 4));
     }
-    SK_CUDA(cudaMemcpyAsync(s->stage_grads, grads_host, gbytes, cudaMemcpyHostToDevice, s->stream));
-    SK_CUDA(cudaMemcpyAsync(s->stage_x, x_host, (uint64_t)s->P.d * 4, cudaMemcpyHostToDevice, s->stream));
-    int rc = do_step(s, s->stage_grads, s->stage_x);
+    if (s->phase != 0) return fail(SK_ESTATE, "sk_step_host: a partitioned step is in progress");
+    if (!s->copy_stream) {
+        SK_CUDA(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
+        for (cudaEvent_t& ev : s->copy_done) SK_CUDA(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    }
+    // The gradients arrive in up to kHostPieces pieces of whole workers on a copy stream of their own, and the sketch
+    // kernel starts on a piece as soon as it is there, so all but the last piece's kernel hides behind the transfer;
+    // x, which only the last stage needs, follows the gradients.
+    const uint32_t n = s->P.n;
+    const uint32_t per = (n + sk_state::kHostPieces - 1) / sk_state::kHostPieces;
+    const uint64_t wbytes = (uint64_t)s->P.d * (s->grads_bf16 ? 2 : 4);
+    SK_CUDA(cudaEventRecord(s->copy_done[sk_state::kHostPieces], s->stream));        // earlier work on the handle's stream
+    SK_CUDA(cudaStreamWaitEvent(s->copy_stream, s->copy_done[sk_state::kHostPieces], 0));
+    s->step_vec = (s->P.d % 4 == 0) && s->P.log2g >= 2;                               // the staging buffers are aligned
+    uint32_t piece = 0;
+    for (uint32_t w = 0; w < n; w += per, ++piece) {
+        const uint32_t we = std::min(n, w + per);
+        SK_CUDA(cudaMemcpyAsync((char*)s->stage_grads + w * wbytes, (const char*)grads_host + w * wbytes, (we - w) * wbytes,
+                                cudaMemcpyHostToDevice, s->copy_stream));
+        SK_CUDA(cudaEventRecord(s->copy_done[piece], s->copy_stream));
+        SK_CUDA(cudaStreamWaitEvent(s->stream, s->copy_done[piece], 0));
+        int rc = phase_local(s, s->stage_grads, nullptr, w, we);
+        if (rc) return rc;
+    }
+    SK_CUDA(cudaMemcpyAsync(s->stage_x, x_host, (uint64_t)s->P.d * 4, cudaMemcpyHostToDevice, s->copy_stream));
+    SK_CUDA(cudaEventRecord(s->copy_done[sk_state::kHostPieces], s->copy_stream));
+    int rc = phase_select(s, nullptr, nullptr);
+    if (rc) return rc;
+    SK_CUDA(cudaStreamWaitEvent(s->stream, s->copy_done[sk_state::kHostPieces], 0));
+    rc = phase_finish(s, nullptr, s->stage_x);
     if (rc) return rc;
     SK_CUDA(cudaMemcpyAsync(x_host, s->stage_x, (uint64_t)s->P.d * 4, cudaMemcpyDeviceToHost, s->stream));
     SK_CUDA(cudaStreamSynchronize(s->stream));

@@ -45,6 +45,10 @@ struct sk_state {
     sk::Select* sel = nullptr;
     sk::Cand *cand = nullptr, *cand2 = nullptr;
     float *stage_grads = nullptr, *stage_x = nullptr;
+    // host-buffer step: the gradients are copied in pieces on a stream of their own (one event per piece, one for x)
+    static constexpr uint32_t kHostPieces = 4;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t copy_done[kHostPieces + 1] = {};
     // timing
     std::vector<TimeRec> recs;
     std::vector<cudaEvent_t> free_events;
