@@ -328,6 +328,27 @@ def main():
                "h2d_bytes_per_step": gbytes * w.n * w.d + 4 * w.d, "d2h_bytes_per_step": 4 * w.d,
                "ms_per_step": 1e3 * dt / args.e2e_steps, "steps": args.e2e_steps}
 
+    # the same through the sparse-return host step (Section III-B's pattern: parameters stay on the device, host
+    # gradients in, k indices and values back); reported beside e2e, not instead of it
+    e2e_sparse = None
+    if args.e2e_steps > 0 and not args.partition_workers:
+        import numpy as np
+        idx = np.empty(w.k, np.uint32)
+        val = np.empty(w.k, np.float32)
+        opt.set("x", x)
+        opt.step_host_sparse(hg, idx, val)
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            opt.step_host_sparse(hg, idx, val)
+        torch.cuda.synchronize()
+        dt = reduce_max(time.perf_counter() - t0, world, dev)
+        e2e_sparse = {"value": units * args.e2e_steps / dt / 1e9, "unit": UNIT,
+                      "h2d_bytes_per_step": gbytes * w.n * w.d, "d2h_bytes_per_step": 8 * w.k,
+                      "ms_per_step": 1e3 * dt / args.e2e_steps, "steps": args.e2e_steps,
+                      "api": "sk_step_host_sparse: parameters resident on the device, sparse update returned"}
+
     if rank != 0:
         return
     cpu = None
@@ -357,7 +378,7 @@ def main():
                               "frac": b_alg / (ms_step * 1e-3) / 1e9 / peak},
             "roofline": roofline,
             "stage_ms_per_step": {nm: stage_ms[q] / max(1, nsteps) for q, nm in enumerate(binding.STAGE_NAMES)},
-            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+            "cpu_baseline": cpu, "e2e": e2e, "e2e_sparse_return": e2e_sparse, "gpu_launches": int(launches), "clocks": clocks}
     print(json.dumps(line), flush=True)
 
 

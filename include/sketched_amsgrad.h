@@ -72,6 +72,15 @@ int sk_set_lr(sk_state* state, float lr);
  * created on first use and released by sk_destroy. */
 int sk_step_host(const void* grads_host, float* x_host, sk_state* state);
 
+/* Host-buffer step in the method's own exchange pattern (Section III-B: what the master returns is the sparse update,
+ * k values and their positions): the parameters stay on the device (field "x": set it once with sk_set, read it with
+ * sk_get; zero until set), the gradients come from the host as for sk_step_host, and what goes back is
+ * idx_host[q] = the k coordinates of I_t (in no particular order) and values_host[q] = the new value of x there, so
+ * that a host copy of the parameters is brought up to date with x[idx_host[q]] = values_host[q].  Both HOST, k
+ * entries.  8*k bytes return instead of 4*d, and x is not sent at all.  Synchronises the stream.
+ * sk_step_host overwrites the same device-resident parameters with its x_host. */
+int sk_step_host_sparse(const void* grads_host, uint32_t* idx_host, float* values_host, sk_state* state);
+
 /* ---- One iteration with the WORKERS PARTITIONED over several processes (one GPU each) -----------------------------
  * Every process creates a handle for its own n workers (same d, r, c, k, seed, hyper-parameters and options on all
  * of them), sets the option "workers_total" to the number of workers over all processes, and keeps a replica of x.
@@ -164,6 +173,7 @@ int sk_hash(const sk_state* state, uint32_t row, uint64_t i0, uint64_t count,
  *   "I"       k uint32  I_t of the last step, ascending (get);  set: installs I_{t-1} for the next step
  *   "vw","vhatw" n*d  per-worker second moments (parameter-averaging variant only; "v","vhat" are then unavailable)
  *   "cand"    P*k uint32  candidates of the last step's second round, ascending (get only; empty when P = 1)
+ *   "x"       d    the device-resident parameters of the host-buffer steps (see sk_step_host_sparse)
  *   "t"       1 uint64  number of steps taken
  * Both calls synchronise the stream. */
 int sk_get(sk_state* state, const char* field, void* buf, uint64_t bytes);

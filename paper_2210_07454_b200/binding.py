@@ -13,7 +13,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsketched_amsgrad.so")
 
-EXPORTS = ["sk_create", "sk_step", "sk_set_lr", "sk_step_host", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
+EXPORTS = ["sk_create", "sk_step", "sk_set_lr", "sk_step_host", "sk_step_host_sparse", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
            "sk_get_option", "sk_hash", "sk_get", "sk_set", "sk_algorithmic_bytes", "sk_get_timing", "sk_select_static",
            "sk_exchange_floats", "sk_step_local", "sk_step_select", "sk_step_finish", "sk_last_error", "sk_version"]
 STATIC_MAX_D = 262144
@@ -41,6 +41,7 @@ def lib() -> C.CDLL:
         L.sk_step.restype = C.c_int; L.sk_step.argtypes = [vp, vp, vp]
         L.sk_set_lr.restype = C.c_int; L.sk_set_lr.argtypes = [vp, f32]
         L.sk_step_host.restype = C.c_int; L.sk_step_host.argtypes = [vp, vp, vp]
+        L.sk_step_host_sparse.restype = C.c_int; L.sk_step_host_sparse.argtypes = [vp, vp, vp, vp]
         L.sk_destroy.restype = None; L.sk_destroy.argtypes = [vp]
         L.sk_set_stream.restype = C.c_int; L.sk_set_stream.argtypes = [vp, vp]
         L.sk_sync.restype = C.c_int; L.sk_sync.argtypes = [vp]
@@ -84,7 +85,7 @@ def _nbytes(t) -> int:
 class SketchedAMSGrad:
     """Handle over ``sk_create`` / ``sk_step`` / ``sk_destroy`` and the auxiliary calls."""
 
-    _FIELD_SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "tables": "nrc", "sum": "rc",
+    _FIELD_SHAPES = {"m": "nd", "e": "nd", "v": "d", "vhat": "d", "est": "d", "x": "d", "tables": "nrc", "sum": "rc",
                      "vw": "nd", "vhatw": "nd"}
 
     def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None,
@@ -127,6 +128,11 @@ class SketchedAMSGrad:
     def step_host(self, grads, x) -> None:
         """Same step with host buffers (numpy arrays or CPU tensors, ideally pinned); x is updated in place."""
         _check(lib().sk_step_host(_ptr(grads), _ptr(x), self._h))
+
+    def step_host_sparse(self, grads, idx_out, values_out) -> None:
+        """Host gradients in, sparse update out (k indices of I_t and the new values of x there); the parameters stay
+        on the device (field "x").  idx_out: k uint32, values_out: k float32, host arrays."""
+        _check(lib().sk_step_host_sparse(_ptr(grads), _ptr(idx_out), _ptr(values_out), self._h))
 
     # -- one iteration in three phases, the workers partitioned over processes (see partitioned.py) ----
     def exchange_floats(self, which: int) -> int:

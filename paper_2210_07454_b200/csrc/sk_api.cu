@@ -287,11 +287,11 @@ int shard_buffers(sk_state* s) {
     return SK_OK;
 }
 
-enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_VW, F_VHATW, F_CAND, F_BAD };
+enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_VW, F_VHATW, F_CAND, F_X, F_BAD };
 
 Field field_of(const char* name) {
-    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t", "vw", "vhatw", "cand"};
-    for (int q = 0; q < 12; ++q) if (!strcmp(name, names[q])) return (Field)q;
+    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t", "vw", "vhatw", "cand", "x"};
+    for (int q = 0; q < 13; ++q) if (!strcmp(name, names[q])) return (Field)q;
     return F_BAD;
 }
 
@@ -380,7 +380,7 @@ void sk_destroy(sk_state* s) {
     for (void* p : {(void*)s->m, (void*)s->e, (void*)s->v, (void*)s->vhat, (void*)s->vstamp, (void*)s->tables,
                     (void*)s->sum, (void*)s->I, (void*)s->I_prev, (void*)s->hist, (void*)s->hist2, (void*)s->sel, (void*)s->cand, (void*)s->cand2,
                     (void*)s->keys, (void*)s->gsum, (void*)s->asum, (void*)s->bitmap, (void*)s->vw, (void*)s->vhatw, (void*)s->Ic, (void*)s->keys2, (void*)s->cbitmap, (void*)s->scan,
-                    (void*)s->stage_grads, (void*)s->stage_x})
+                    (void*)s->stage_grads, (void*)s->stage_x, (void*)s->stage_vals})
         if (p) cudaFree(p);
     if (s->copy_stream) {
         cudaStreamSynchronize(s->copy_stream);
@@ -398,21 +398,29 @@ int sk_step(const void* grads, float* x, sk_state* s) {
     return do_step(s, grads, x);
 }
 
-int sk_step_host(const void* grads_host, float* x_host, sk_state* s) {
-    if (!s || !grads_host || !x_host) return fail(SK_EINVAL, "sk_step_host: null argument");
+// staging buffers of the host-buffer steps; stage_x doubles as the device-resident parameters (field "x")
+static int ensure_stage(sk_state* s) {
+    if (s->stage_grads) return SK_OK;
     const uint64_t nd = (uint64_t)s->P.n * s->P.d;
-    if (!s->stage_grads) {
-        SK_CUDA(cudaMalloc((void**)&s->stage_grads, nd * 4));
-        SK_CUDA(cudaMalloc((void**)&s->stage_x, (uint64_t)s->P.d * 4));
-    }
-    if (s->phase != 0) return fail(SK_ESTATE, "sk_step_host: a partitioned step is in progress");
+    SK_CUDA(cudaMalloc((void**)&s->stage_grads, nd * 4));
+    SK_CUDA(cudaMalloc((void**)&s->stage_x, (uint64_t)s->P.d * 4));
+    SK_CUDA(cudaMalloc((void**)&s->stage_vals, (uint64_t)s->P.k * 4));
+    SK_CUDA(cudaMemsetAsync(s->stage_x, 0, (uint64_t)s->P.d * 4, s->stream));
+    return SK_OK;
+}
+
+// The step on host gradients up to (not including) the copy back.  x_host != nullptr: x is sent after the gradients
+// (only the last stage reads it); nullptr: the parameters already on the device (field "x") are used.
+static int host_step(sk_state* s, const void* grads_host, const float* x_host) {
+    if (s->phase != 0) return fail(SK_ESTATE, "a partitioned step is in progress");
+    int rc = ensure_stage(s);
+    if (rc) return rc;
     if (!s->copy_stream) {
         SK_CUDA(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
         for (cudaEvent_t& ev : s->copy_done) SK_CUDA(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
     }
     // The gradients arrive in up to kHostPieces pieces of whole workers on a copy stream of their own, and the sketch
-    // kernel starts on a piece as soon as it is there, so all but the last piece's kernel hides behind the transfer;
-    // x, which only the last stage needs, follows the gradients.
+    // kernel starts on a piece as soon as it is there, so all but the last piece's kernel hides behind the transfer.
     const uint32_t n = s->P.n;
     const uint32_t per = (n + sk_state::kHostPieces - 1) / sk_state::kHostPieces;
     const uint64_t wbytes = (uint64_t)s->P.d * (s->grads_bf16 ? 2 : 4);
@@ -426,17 +434,36 @@ int sk_step_host(const void* grads_host, float* x_host, sk_state* s) {
                                 cudaMemcpyHostToDevice, s->copy_stream));
         SK_CUDA(cudaEventRecord(s->copy_done[piece], s->copy_stream));
         SK_CUDA(cudaStreamWaitEvent(s->stream, s->copy_done[piece], 0));
-        int rc = phase_local(s, s->stage_grads, nullptr, w, we);
+        rc = phase_local(s, s->stage_grads, nullptr, w, we);
         if (rc) return rc;
     }
-    SK_CUDA(cudaMemcpyAsync(s->stage_x, x_host, (uint64_t)s->P.d * 4, cudaMemcpyHostToDevice, s->copy_stream));
-    SK_CUDA(cudaEventRecord(s->copy_done[sk_state::kHostPieces], s->copy_stream));
-    int rc = phase_select(s, nullptr, nullptr);
+    if (x_host) {
+        SK_CUDA(cudaMemcpyAsync(s->stage_x, x_host, (uint64_t)s->P.d * 4, cudaMemcpyHostToDevice, s->copy_stream));
+        SK_CUDA(cudaEventRecord(s->copy_done[sk_state::kHostPieces], s->copy_stream));
+    }
+    rc = phase_select(s, nullptr, nullptr);
     if (rc) return rc;
-    SK_CUDA(cudaStreamWaitEvent(s->stream, s->copy_done[sk_state::kHostPieces], 0));
-    rc = phase_finish(s, nullptr, s->stage_x);
+    if (x_host) SK_CUDA(cudaStreamWaitEvent(s->stream, s->copy_done[sk_state::kHostPieces], 0));
+    return phase_finish(s, nullptr, s->stage_x);
+}
+
+int sk_step_host(const void* grads_host, float* x_host, sk_state* s) {
+    if (!s || !grads_host || !x_host) return fail(SK_EINVAL, "sk_step_host: null argument");
+    int rc = host_step(s, grads_host, x_host);
     if (rc) return rc;
     SK_CUDA(cudaMemcpyAsync(x_host, s->stage_x, (uint64_t)s->P.d * 4, cudaMemcpyDeviceToHost, s->stream));
+    SK_CUDA(cudaStreamSynchronize(s->stream));
+    return SK_OK;
+}
+
+int sk_step_host_sparse(const void* grads_host, uint32_t* idx_host, float* values_host, sk_state* s) {
+    if (!s || !grads_host || !idx_host || !values_host) return fail(SK_EINVAL, "sk_step_host_sparse: null argument");
+    int rc = host_step(s, grads_host, nullptr);
+    if (rc) return rc;
+    const uint64_t kb = (uint64_t)s->P.k * 4;
+    sk::launch_gather(s->I_prev, s->P.k, s->P.k, s->stage_x, s->stage_vals, s->stream);   // I_prev holds I_t now
+    SK_CUDA(cudaMemcpyAsync(idx_host, s->I_prev, kb, cudaMemcpyDeviceToHost, s->stream));
+    SK_CUDA(cudaMemcpyAsync(values_host, s->stage_vals, kb, cudaMemcpyDeviceToHost, s->stream));
     SK_CUDA(cudaStreamSynchronize(s->stream));
     return SK_OK;
 }

@@ -44,7 +44,7 @@ struct sk_state {
     uint32_t *cbitmap = nullptr, *scan = nullptr;   // scratch of the partitioned step: candidate bitmap, block offsets
     sk::Select* sel = nullptr;
     sk::Cand *cand = nullptr, *cand2 = nullptr;
-    float *stage_grads = nullptr, *stage_x = nullptr;
+    float *stage_grads = nullptr, *stage_x = nullptr, *stage_vals = nullptr;
     // host-buffer step: the gradients are copied in pieces on a stream of their own (one event per piece, one for x)
     static constexpr uint32_t kHostPieces = 4;
     cudaStream_t copy_stream = nullptr;

@@ -576,6 +576,34 @@ def test_host_step_matches_device_step():
     close(xh, xa.cpu().numpy(), "x via host entry point")
 
 
+def test_sparse_host_step_matches_device_step():
+    # parameters resident on the device, host gradients in, (index, new value) pairs out: applying the pairs to a
+    # host copy of x must reproduce the device step, step after step
+    w = _workload("C1", name="E", d=40_000, n=5, r=5, c=2048, k=400)
+    b = _binding()
+    src = _source(w, cfg_id=4)
+    dev = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=2, lr=w.lr)
+    host = b.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=2, lr=w.lr)
+    x_dev = src.x0()
+    x_host = x_dev.cpu().numpy().copy()
+    host.set("x", x_host)
+    idx = np.empty(w.k, np.uint32)
+    val = np.empty(w.k, np.float32)
+    for t in range(1, 5):
+        g = src.grads(t)
+        dev.step(g, x_dev)
+        host.step_host_sparse(g.cpu().numpy(), idx, val)
+        dev.sync()
+        assert np.array_equal(np.sort(idx), host.get("I")) and np.array_equal(host.get("I"), dev.get("I"))
+        x_host[idx] = val
+        np.testing.assert_allclose(x_host, x_dev.cpu().numpy(), rtol=1e-6, atol=1e-9)
+        assert np.array_equal(host.get("x"), x_host)           # the device-resident parameters are the same vector
+    # the dense host step shares those parameters
+    xh = x_host.copy()
+    host.step_host(src.grads(5).cpu().numpy(), xh)
+    assert np.array_equal(host.get("x"), xh)
+
+
 def test_argument_errors():
     b = _binding()
     with pytest.raises(b.SkError):
