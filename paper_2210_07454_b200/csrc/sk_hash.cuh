@@ -91,7 +91,10 @@ __device__ __forceinline__ void quad_hashes(const Params& P, uint32_t r, uint32_
                         const uint32_t src = (lane & ~7u) + j;
                         const uint32_t ohi = __shfl_sync(0xFFFFFFFFu, hi, src);
                         const uint32_t olo = __shfl_sync(0xFFFFFFFFu, lo, src);
-                        h[k + j] = quad_from_draw(P, ((uint64_t)ohi << 32) | olo, i, wbase);
+                        // g = 32 written out: block = floor(hi * G / 2^32), permutation = the next 5 bits
+                        const uint32_t o = i & 31u, perm = (ohi * P.G) >> 27;
+                        h[k + j].off = wbase + (__umulhi(ohi, P.G) << 5) + ((o ^ perm) & ~3u);
+                        h[k + j].p3sgn = (perm & 3u) | (((olo >> o) & 0xFu) << 2);
                     }
             }
         }

@@ -66,7 +66,9 @@ __device__ __forceinline__ uint32_t key_of(float est) { return __float_as_uint(e
 // of magnitude inside the tolerance within which the selected set is defined -- and it is a deterministic
 // function of (med, vhat), which is all the selection needs.  Denormal vhat takes the exact path.
 __device__ __forceinline__ uint32_t key_rank(float med, float vhat) {
-    return key_of(vhat > 1e-30f ? med * rsqrtf(vhat) : scale_est(med, vhat));
+    float rs;                                         // one MUFU: vhat is a normal number on this branch
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rs) : "f"(vhat));
+    return key_of(vhat > 1e-30f ? med * rs : scale_est(med, vhat));
 }
 
 // medians of the 4 coordinates 4t..4t+3 (vector form, g >= 4).  All lanes of the warp call this together.
