@@ -251,20 +251,58 @@ __device__ __forceinline__ void block_append(uint32_t n_a, uint32_t n_b, uint32_
 
 // ---- pass B over the stored keys: emit above the threshold bin, collect the threshold bin, histogram its next
 // 12 key bits ---------------------------------------------------------------------------------------------------
+// Appends go through per-warp staging buffers in shared memory: a warp reserves room in the global list with one
+// atomic per kWarpBuf entries and copies them out coalesced, so the pass needs no block-wide barrier per tile.
+constexpr uint32_t kWarpBuf = 128;
+
+template <typename T>
+__device__ __forceinline__ void warp_flush(T* buf, uint32_t& fill, uint32_t* counter, T* list) {
+    __syncwarp();
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t base = 0;
+    if (lane == 0 && fill) base = atomicAdd(counter, fill);
+    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+    for (uint32_t q = lane; q < fill; q += 32) list[base + q] = buf[q];
+    __syncwarp();
+    fill = 0;
+}
+
+// where this lane's `mine` entries of the warp's `total` go: into the staging buffer (flushed first if they do not
+// fit), or straight into the list when one tile yields more than a buffer holds
+template <typename T>
+__device__ __forceinline__ T* warp_reserve(T* buf, uint32_t& fill, uint32_t* counter, T* list, uint32_t total,
+                                           uint32_t excl) {
+    if (total == 0) return buf;
+    if (fill + total > kWarpBuf) warp_flush(buf, fill, counter, list);
+    if (total > kWarpBuf) {
+        uint32_t base = 0;
+        if ((threadIdx.x & 31u) == 0) base = atomicAdd(counter, total);
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        return list + base + excl;
+    }
+    T* dst = buf + fill + excl;
+    fill += total;
+    return dst;
+}
+
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx_map, Select* sel, uint32_t* I_out,
        Cand* cand, uint32_t* hist2) {
     // idx_map (scalar form only): keys[t] belongs to coordinate idx_map[t] instead of t (second round on a candidate list)
     __shared__ uint32_t sh2[kHistBins];
+    __shared__ uint32_t wb_out[kThreads / 32][kWarpBuf];
+    __shared__ Cand wb_cand[kThreads / 32][kWarpBuf];
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh2[b] = 0;
     __syncthreads();
     const uint32_t bin = sel->bin;
-    constexpr uint32_t U = 4;                                   // key loads in flight per thread and block-wide append
+    const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
+    uint32_t fill_out = 0, fill_cand = 0;                       // the same in every lane of the warp
+    constexpr uint32_t U = 4;                                   // key loads in flight per thread
     const uint32_t items = VEC ? (d >> 2) : d;
     const uint32_t tile = U * kThreads;
     const uint32_t trips = (items + gridDim.x * tile - 1) / (gridDim.x * tile);
-    for (uint32_t it = 0; it < trips; ++it) {
+    for (uint32_t it = 0; it < trips; ++it) {                   // uniform trip count: warps stay whole
         const uint32_t t0 = (it * gridDim.x + blockIdx.x) * tile + threadIdx.x;
         uint32_t kq[U][4], nk[U];
 #pragma unroll
@@ -292,8 +330,18 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
                     if (b == bin) { atomicAdd(&sh2[(kq[u][q] >> 7) & (kHistBins - 1u)], 1u); ++n_cand; }
                     n_out += b > bin;
                 }
-        uint32_t po, pc;
-        block_append(n_out, n_cand, &sel->cnt_out, &sel->cnt_cand, po, pc);   // <= 16 per thread, <= 4096 per block
+        const uint32_t packed = n_out | (n_cand << 16);         // each <= 16 per thread, <= 512 per warp
+        uint32_t incl = packed;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= (uint32_t)off) incl += o;
+        }
+        const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        if (total == 0) continue;
+        const uint32_t excl = incl - packed;
+        uint32_t* po = warp_reserve(wb_out[wid], fill_out, &sel->cnt_out, I_out, total & 0xFFFFu, excl & 0xFFFFu);
+        Cand* pc = warp_reserve(wb_cand[wid], fill_cand, &sel->cnt_cand, cand, total >> 16, excl >> 16);
 #pragma unroll
         for (uint32_t u = 0; u < U; ++u) {
             const uint32_t t = t0 + u * kThreads;
@@ -302,11 +350,13 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
             for (uint32_t q = 0; q < 4; ++q)
                 if (q < nk[u]) {
                     const uint32_t b = kq[u][q] >> kHistShift;
-                    if (b > bin) I_out[po++] = idx0 + q;
-                    else if (b == bin) { cand[pc].key = kq[u][q]; cand[pc].idx = idx0 + q; ++pc; }
+                    if (b > bin) *po++ = idx0 + q;
+                    else if (b == bin) { pc->key = kq[u][q]; pc->idx = idx0 + q; ++pc; }
                 }
         }
     }
+    warp_flush(wb_out[wid], fill_out, &sel->cnt_out, I_out);
+    warp_flush(wb_cand[wid], fill_cand, &sel->cnt_cand, cand);
     __syncthreads();
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
         if (sh2[b]) atomicAdd(&hist2[b], sh2[b]);
