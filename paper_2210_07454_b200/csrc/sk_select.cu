@@ -296,6 +296,8 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh2[b] = 0;
     __syncthreads();
     const uint32_t bin = sel->bin;
+    const uint32_t thr_lo = bin << kHistShift;                  // first key of the threshold bin
+    const uint32_t thr_hi = (bin + 1u) << kHistShift;           // first key above it (2^31 for the last bin: no key)
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     uint32_t fill_out = 0, fill_cand = 0;                       // the same in every lane of the warp
     constexpr uint32_t U = 4;                                   // key loads in flight per thread
@@ -320,16 +322,19 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
                 }
             }
         }
-        uint32_t n_out = 0, n_cand = 0;
+        // counting is branch-free: almost every key is below the threshold bin
+        uint32_t n_out = 0, n_ge = 0;
 #pragma unroll
         for (uint32_t u = 0; u < U; ++u)
+            if (nk[u]) {
 #pragma unroll
-            for (uint32_t q = 0; q < 4; ++q)
-                if (q < nk[u]) {
-                    const uint32_t b = kq[u][q] >> kHistShift;
-                    if (b == bin) { atomicAdd(&sh2[(kq[u][q] >> 7) & (kHistBins - 1u)], 1u); ++n_cand; }
-                    n_out += b > bin;
-                }
+                for (uint32_t q = 0; q < 4; ++q)
+                    if (VEC || q == 0) {
+                        n_out += kq[u][q] >= thr_hi;
+                        n_ge += kq[u][q] >= thr_lo;
+                    }
+            }
+        const uint32_t n_cand = n_ge - n_out;
         const uint32_t packed = n_out | (n_cand << 16);         // each <= 16 per thread, <= 512 per warp
         uint32_t incl = packed;
 #pragma unroll
@@ -342,16 +347,21 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
         const uint32_t excl = incl - packed;
         uint32_t* po = warp_reserve(wb_out[wid], fill_out, &sel->cnt_out, I_out, total & 0xFFFFu, excl & 0xFFFFu);
         Cand* pc = warp_reserve(wb_cand[wid], fill_cand, &sel->cnt_cand, cand, total >> 16, excl >> 16);
+        if (packed == 0) continue;                              // this lane has nothing to append
 #pragma unroll
         for (uint32_t u = 0; u < U; ++u) {
+            if (!nk[u]) continue;
             const uint32_t t = t0 + u * kThreads;
-            const uint32_t idx0 = VEC ? (t << 2) : ((idx_map && nk[u]) ? idx_map[t] : t);
+            const uint32_t idx0 = VEC ? (t << 2) : (idx_map ? idx_map[t] : t);
 #pragma unroll
             for (uint32_t q = 0; q < 4; ++q)
-                if (q < nk[u]) {
-                    const uint32_t b = kq[u][q] >> kHistShift;
-                    if (b > bin) *po++ = idx0 + q;
-                    else if (b == bin) { pc->key = kq[u][q]; pc->idx = idx0 + q; ++pc; }
+                if (VEC || q == 0) {
+                    const uint32_t key = kq[u][q];
+                    if (key >= thr_hi) *po++ = idx0 + q;
+                    else if (key >= thr_lo) {
+                        atomicAdd(&sh2[(key >> 7) & (kHistBins - 1u)], 1u);
+                        pc->key = key; pc->idx = idx0 + q; ++pc;
+                    }
                 }
         }
     }
