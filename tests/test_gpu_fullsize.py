@@ -110,3 +110,33 @@ def test_first_step_full_then_properties(name):
     np.testing.assert_allclose(gpu.get("v")[sample], want, rtol=1e-5)
     e = gpu.get("e")
     assert not e[:, I2].any()
+
+
+def test_c2_hundred_free_running_steps_keep_the_invariants():
+    # no reference: what must hold at every step whatever the data (Algorithm 2 and the proof of Lemma 3)
+    from paper_2210_07454_b200 import binding, synthetic
+    w = synthetic.WORKLOADS["C2"]
+    src = synthetic.GradientSource(w, device="cuda")
+    gpu = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
+    x = src.x0()
+    gsets = [src.grads(t) for t in (1, 2, 3)]
+    vhat_prev = gpu.get("vhat")
+    I_prev = np.zeros(0, np.uint32)
+    for t in range(1, 101):
+        x_before = x.clone() if t % 10 == 0 else None
+        gpu.step(gsets[t % 3], x)
+        if t % 10:
+            continue
+        gpu.sync()                                            # also reads the device status word
+        I = gpu.get("I")
+        assert I.size == w.k and np.all(np.diff(I.astype(np.int64)) > 0) and I[-1] < w.d
+        changed = torch.nonzero(x != x_before).flatten().cpu().numpy()
+        assert np.isin(changed, I).all()                      # x moves on I_t only
+        assert bool(torch.isfinite(x).all())
+        vhat = gpu.get("vhat")
+        assert np.all(vhat >= vhat_prev) and np.all(vhat >= np.float32(w.eps))
+        vhat_prev = vhat
+        e = gpu.get("e")
+        assert not e[:, I].any() and np.isfinite(e).all()     # the residual vanishes on I_t
+        I_prev = I
+    assert gpu.get("t")[0] == 100
