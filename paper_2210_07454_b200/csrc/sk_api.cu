@@ -143,11 +143,14 @@ int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, ui
     sk::MomentArgs A = moment_args(s, grads);
     // the windowed kernel implements Algorithm 2 with one table per worker only
     const bool windowed = vec && P.win_cw != 0 && s->variant == 0 && !s->sum_sketch;
-    const uint32_t wc = windowed ? std::min<uint32_t>((uint32_t)s->window_workers, P.n) : chunk_of(s);
+    const bool own = windowed && s->window_kernel == 1;      // accumulation by ownership: one warp per worker
+    const uint32_t wc = own ? std::min<uint32_t>(std::min<uint32_t>((uint32_t)s->window_workers, sk::kOwnMaxWorkers), P.n)
+                      : windowed ? std::min<uint32_t>(std::min<uint32_t>((uint32_t)s->window_workers, sk::kWinMaxWorkers), P.n)
+                                 : chunk_of(s);
     // With a second round the sketch kernel also leaves sum_w a^(w) per coordinate, so that each of the P*k exact
     // values costs one gather instead of n (not the windowed kernel, and not a partitioned step, whose exact values
     // are exchanged: there every local worker's value is gathered).
-    A.asum = (s->cand_mult > 1 && !windowed && !sharded) ? s->asum : nullptr;
+    A.asum = ((s->cand_mult > 1 || s->always_asum) && (!windowed || own) && !sharded) ? s->asum : nullptr;
     s->asum_live = A.asum != nullptr;
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     float* sum_out = sharded ? x1 : s->sum;
@@ -168,7 +171,8 @@ int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, ui
         }
         StageTimer tm(s, 2);     // moments + sketch; also leaves the gradient sums on I_{t-1} in gsum
         if (windowed) {
-            const int l = sk::launch_moment_sketch_win(P, A, w0, nw, (uint32_t)s->window_red_rows, s->sm_count, st);
+            const int l = own ? sk::launch_moment_sketch_own(P, A, w0, nw, s->sm_count, st)
+                              : sk::launch_moment_sketch_win(P, A, w0, nw, (uint32_t)s->window_red_rows, s->sm_count, st);
             if (l < 0) return fail(SK_ECUDA, "the windowed sketch kernel does not fit in shared memory (window_lines=%lld, r=%u)",
                                    (long long)s->window_lines, P.r);
             tm.done(l);
@@ -553,10 +557,10 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         if (s->t != 0) return fail(SK_ESTATE, "P can only be changed before the first step");
         if (value < 1 || (uint64_t)value * s->P.k > s->P.d) return fail(SK_EINVAL, "P must be >= 1 with P*k <= d");
         if (value > 1) {
-            if (s->Ic) { cudaFree(s->Ic); cudaFree(s->keys2); cudaFree(s->asum); s->Ic = s->keys2 = nullptr; s->asum = nullptr; }
+            if (s->Ic) { cudaFree(s->Ic); cudaFree(s->keys2); s->Ic = s->keys2 = nullptr; }
             const uint64_t pk = (uint64_t)value * s->P.k;
             if (cudaMalloc((void**)&s->Ic, pk * 4) != cudaSuccess || cudaMalloc((void**)&s->keys2, pk * 4) != cudaSuccess ||
-                cudaMalloc((void**)&s->asum, ((uint64_t)s->P.d + 3) / 4 * 16) != cudaSuccess)
+                (!s->asum && cudaMalloc((void**)&s->asum, ((uint64_t)s->P.d + 3) / 4 * 16) != cudaSuccess))
                 return fail(SK_ENOMEM, "cudaMalloc of the candidate buffers failed: %s", cudaGetErrorString(cudaGetLastError()));
         }
         s->cand_mult = value;
@@ -609,8 +613,21 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         return SK_OK;
     }
     if (!strcmp(key, "window_workers")) {
-        if (value < 1 || value > (int64_t)sk::kWinMaxWorkers) return fail(SK_EINVAL, "window_workers must be in 1..4");
+        if (value < 1 || value > (int64_t)sk::kOwnMaxWorkers) return fail(SK_EINVAL, "window_workers must be in 1..8");
         s->window_workers = value;
+        return SK_OK;
+    }
+    if (!strcmp(key, "window_kernel")) {
+        if (value != 0 && value != 1) return fail(SK_EINVAL, "window_kernel must be 0 (producer/consumer roles) or 1 (ownership)");
+        s->window_kernel = value;
+        return SK_OK;
+    }
+    if (!strcmp(key, "worker_sum")) {
+        if (value != 0 && value != 1) return fail(SK_EINVAL, "worker_sum must be 0 or 1");
+        if (s->phase != 0) return fail(SK_ESTATE, "worker_sum cannot change inside a partitioned step");
+        if (value && !s->asum && cudaMalloc((void**)&s->asum, ((uint64_t)s->P.d + 3) / 4 * 16) != cudaSuccess)
+            return fail(SK_ENOMEM, "cudaMalloc of the worker-sum buffer failed: %s", cudaGetErrorString(cudaGetLastError()));
+        s->always_asum = value;
         return SK_OK;
     }
     if (!strcmp(key, "worker_chunk")) {
@@ -637,6 +654,8 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     if (!strcmp(key, "log2g")) *value = s->P.log2g;
     else if (!strcmp(key, "window_lines")) *value = s->window_lines;
     else if (!strcmp(key, "window_workers")) *value = s->window_workers;
+    else if (!strcmp(key, "window_kernel")) *value = s->window_kernel;
+    else if (!strcmp(key, "worker_sum")) *value = s->always_asum;
     else if (!strcmp(key, "variant")) *value = s->variant;
     else if (!strcmp(key, "P")) *value = s->cand_mult;
     else if (!strcmp(key, "workers_total")) *value = s->P.n_all;

@@ -69,6 +69,11 @@ int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint
 constexpr uint32_t kWinMaxWorkers = 4;
 int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, uint32_t r_red,
                              int sm_count, cudaStream_t st);
+// windowed hash family, accumulation by ownership (one warp per worker, block-owned windows): at most kOwnMaxWorkers
+// workers per launch; fills A.asum when it is set; -1 if it cannot run
+constexpr uint32_t kOwnMaxWorkers = 8;
+int launch_moment_sketch_own(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, int sm_count,
+                             cudaStream_t st);
 int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStream_t st);
 // A.members != 0: also apply the second-moment update on I_{t-1} (bitmap, gsum, v, vstamp, vhat of A)
 int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum, uint32_t* keys, uint32_t* hist,
