@@ -116,6 +116,7 @@ sk::MomentArgs moment_args(const sk_state* s, const void* grads) {
     A.grads = grads; A.grad_bf16 = s->grads_bf16 ? 1u : 0u; A.m = s->m; A.e = s->e; A.tables = s->tables; A.gsum = s->gsum;
     A.v = s->v; A.vhat = s->vhat; A.vstamp = s->vstamp; A.bitmap = s->bitmap;
     A.step = (uint32_t)(s->vclock + 1); A.members = s->k_prev ? 1u : 0u;
+    A.gsum_on = (A.members && !s->freeze_v && s->variant == 0) ? 1u : 0u;
     A.vw = s->vw; A.vhatw = s->vhatw; A.variant = (uint32_t)s->variant;
     return A;
 }
@@ -363,6 +364,7 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     cudaMemset(s->bitmap, 0, s->bitmap_bytes);                          // I_0 is empty
     cudaMemset(s->m, 0, nd * 4); cudaMemset(s->e, 0, nd * 4);           // m_0 = e_0 = 0
     cudaMemset(s->vstamp, 0, d * 4);
+    cudaMemset(s->gsum, 0, d_pad * 4);
     cudaMemset(s->tables, 0, (uint64_t)n * tf * 4); cudaMemset(s->sum, 0, tf * 4);
     cudaMemset(s->hist, 0, sk::kHistBins * 4); cudaMemset(s->hist2, 0, sk::kHistBins * 4);
     cudaMemset(s->sel, 0, sizeof(sk::Select));

@@ -48,12 +48,14 @@ struct MomentArgs {
     float* sum_table;        // not nullptr: sketch the worker sum of a_t once into this r x cs table (already divided by
                              // n_all) instead of one table per worker -- the sketch is linear (Section II-C)
     float* asum;             // d or nullptr: running sum over the workers of a_t, in worker order (second round of Section III-A)
-    float* gsum;             // running gradient sums on I_{t-1} when the workers are processed in several launches
+    float* gsum;             // gradient sums on I_{t-1}, per coordinate.  Zero between steps: the key pass clears what it
+                             // consumes, so a kernel may either overwrite a member's quad or add to it
     float *v, *vhat;
     uint32_t* vstamp;        // step at which v[j] was last brought up to date
     const uint32_t* bitmap;  // membership of I_{t-1}: bit j of word j/32
     uint32_t step;           // t (1-based)
     uint32_t members;        // 0 when I_{t-1} is empty
+    uint32_t gsum_on;        // the gradient sums on I_{t-1} are wanted (members != 0, Algorithm 2, v not frozen)
     // parameter-averaging variant (Algorithm 1): per-worker second moments, n*d each; variant = 1
     float *vw, *vhatw;
     uint32_t variant;        // 0 = gradient averaging (Algorithm 2), 1 = parameter averaging (Algorithm 1)

@@ -152,6 +152,7 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
                     ((float4*)A.v)[t] = vv;
                     ((uint4*)A.vstamp)[t] = vs;
                     ((float4*)A.vhat)[t] = vh;
+                    ((float4*)A.gsum)[t] = make_float4(0.f, 0.f, 0.f, 0.f);   // consumed: the sums start from zero next step
                 }
                 uint4 k4;
                 k4.x = key_rank(med.x, vh.x); k4.y = key_rank(med.y, vh.y);
@@ -170,6 +171,7 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
                 float vv = A.v[t];
                 uint32_t vs = A.vstamp[t];
                 update_member(P, A, A.gsum[t], vv, vs, vh);
+                A.gsum[t] = 0.0f;
                 A.v[t] = vv; A.vstamp[t] = vs; A.vhat[t] = vh;
             }
             const uint32_t key = key_rank(median1(P, sum, t), vh);

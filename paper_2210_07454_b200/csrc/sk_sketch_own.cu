@@ -17,8 +17,8 @@
 //     for fewer rows the groups take turns).
 // The group hashes of a unit (r x 32 draws) are evaluated once per block into a double-buffered shared stage.
 // sum_w a^(w) (used by the update of x) is formed through a shared stage of the unit's a_t values, in worker
-// order; the gradient sums on I_{t-1} are re-read from global memory by one warp per 128 coordinates, in worker
-// order (about 1 % of the coordinates, mostly L2 hits).
+// order; the gradient sums on I_{t-1} (about 1 % of the coordinates) are formed with 16-byte reductions into the
+// gsum array, which is zero between steps because the key pass clears what it consumes.
 #include "sk_internal.h"
 #include "sk_hash.cuh"
 #include "sk_moment.cuh"
@@ -115,8 +115,6 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
     const uint32_t grp = lane >> 3, o = (lane & 7u) * 4u;          // this lane's group in the chunk, offset inside it
     const uint32_t sgn_mul = 1u << (28u - o);
     float* mywin = win + (size_t)wid * r * cw;
-    uint32_t duty = 0;                                             // chunks whose gradient sums this warp forms
-    for (uint32_t c = 0; c < kChunksPerUnit; ++c) if (c % nw == wid) duty |= 1u << c;
 
     auto fill_hashes = [&](uint32_t unit, uint32_t buf) {
         for (uint32_t hq = tid; hq < r * kGroupsPerUnit; hq += nthreads) {
@@ -185,14 +183,8 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
                         __syncwarp();
                     }
             }
-            if (mask && ((duty >> c) & 1u)) {                      // gradient sums on I_{t-1}, workers in order
-                float4 gs = w0 > 0 ? ((const float4*)A.gsum)[t] : zero4;
-                for (uint32_t w = 0; w < nw; ++w) {
-                    const float4 g = load_grad4(A.grads, (uint64_t)(w0 + w) * d4 + t, gb);
-                    gs.x += g.x; gs.y += g.y; gs.z += g.z; gs.w += g.w;
-                }
-                ((float4*)A.gsum)[t] = gs;
-            }
+            // gradient sums on I_{t-1}: every worker's warp adds its quad (gsum is zero between steps)
+            if (A.gsum_on && mask) red_add_v4(A.gsum + 4u * (size_t)t, k.g);
         }
         __syncthreads();            // every warp is done with this unit's hashes, windows and a_t stage
 
@@ -275,9 +267,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
     const uint32_t grp = lane >> 3, o = (lane & 7u) * 4u;          // this lane's group in the chunk, offset inside it
     const uint32_t sgn_mul = 1u << (28u - o);
-    const uint32_t members = A.members;
-    uint32_t duty = 0;                                             // chunks whose gradient sums this warp forms
-    for (uint32_t c = 0; c < kChunksPerUnit; ++c) if (c % nw == wid) duty |= 1u << c;
+    const uint32_t members = A.members, gsum_on = A.gsum_on;
 
     // per-lane shared addresses: the window row of sub-step i, and the stage entry of (row = group + i, group of chunk 0)
     const uint32_t sm_win = (uint32_t)__cvta_generic_to_shared(win);
@@ -322,7 +312,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
         SK_MOMENT(mm, aa, gg, mask)                                                                                 \
         __stcs(m4 + (tc_), mm); __stcs(e4 + (tc_), aa);                                                             \
         if (ASUM) sts128(ast_lane + (c_) * 512u, aa);                                                               \
-        _Pragma("unroll") for (uint32_t i = 0; i < r; ++i) {                                                        \
+        _Pragma("unroll") for (uint32_t i = 0; i < r; ++i) {                                   \
             const uint32_t addr = wrow[i] + ((h[i].x ^ o) & ~3u) * 4u;                                              \
             float4 cur = lds128(addr);                                                                              \
             const uint32_t t3 = h[i].y * sgn_mul, t2 = t3 * 2u, t1 = t3 * 4u, t0 = t3 * 8u;                         \
@@ -337,14 +327,8 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
             sts128(addr, cur);                                                                                      \
             __syncwarp();                        /* the next sub-step's lanes may read what these wrote */          \
         }                                                                                                           \
-        if (mask && ((duty >> (c_)) & 1u)) {     /* gradient sums on I_{t-1}, workers in order */                   \
-            float4 gs = w0 > 0 ? ((const float4*)A.gsum)[tc_] : zero4;                                              \
-            for (uint32_t w = 0; w < nw; ++w) {                                                                     \
-                const float4 g = load_grad4(A.grads, (uint64_t)(w0 + w) * d4 + (tc_), gb);                          \
-                gs.x += g.x; gs.y += g.y; gs.z += g.z; gs.w += g.w;                                                 \
-            }                                                                                                       \
-            ((float4*)A.gsum)[tc_] = gs;                                                                            \
-        }                                                                                                           \
+        /* gradient sums on I_{t-1}: every worker's warp adds its quad (gsum is zero between steps) */            \
+        if (gsum_on && mask) red_add_v4(A.gsum + 4u * (size_t)(tc_), gg);                                           \
         hs_c += 32u;                                                                                                \
     }
 
