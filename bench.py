@@ -176,8 +176,6 @@ def main():
                     help="ga = gradient averaging (Algorithm 2, the headline path); pa = parameter averaging (Algorithm 1)")
     ap.add_argument("--window-lines", type=int, default=None, help="windowed hash family: lines per window (0 = plain)")
     ap.add_argument("--window-workers", type=int, default=0, help="workers per launch of the windowed sketch kernel")
-    ap.add_argument("--window-red-rows", type=int, default=-1, help="rows the windowed kernel sketches by L2 reductions")
-    ap.add_argument("--window-kernel", type=int, default=-1, help="windowed sketch kernel: 1 = ownership, 0 = producer/consumer")
     ap.add_argument("--worker-sum", type=int, default=-1, help="1: the sketch kernel leaves the worker sum of a_t for the update of x")
     ap.add_argument("--worker-chunk", type=int, default=0)
     ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
@@ -234,12 +232,8 @@ def main():
     opt.set_option("worker_chunk", args.worker_chunk)
     if args.window_workers:
         opt.set_option("window_workers", args.window_workers)
-    if args.window_red_rows >= 0:
-        opt.set_option("window_red_rows", args.window_red_rows)
     if args.sketch_ctas:
         opt.set_option("sketch_ctas_per_sm", args.sketch_ctas)
-    if args.window_kernel >= 0:
-        opt.set_option("window_kernel", args.window_kernel)
     if args.worker_sum >= 0:
         opt.set_option("worker_sum", args.worker_sum)
     # gradient buffers rotate so that no step finds its inputs in L2 (each set is far larger than L2 anyway)

@@ -143,9 +143,12 @@ int sk_sync(sk_state* state);
  *                  of the exact values on I_t.  Only before the first step; allocates 8*n*d bytes.
  *   "window_lines" L > 0 selects the windowed variant of the hash family (needs g = 32, 32*L <= c): units of
  *                  1024 coordinates map into one aligned window of 32*L buckets per row, which lets the sketch
- *                  kernel accumulate in shared memory.  0 (default) = plain family.  Only before the first step.
- *   "window_workers" (1..4) workers per launch and "window_red_rows" (0..4) rows sketched by L2 reductions
- *                  instead of shared-memory windows, both for the windowed kernel only.
+ *                  kernel accumulate in shared memory, one warp per worker.  Default: 8 when g = 32 and c >= 256,
+ *                  else 0 (plain family; also what "log2g" < 5 selects).  Only before the first step.
+ *   "window_workers" (1..8) workers per launch of the shared-memory sketch kernel (one warp each); default 8.
+ *   "worker_sum"   1: the sketch kernel also stores sum_w a^(w) per coordinate (4*d bytes more written, allocated
+ *                  when first enabled), and the update of x reads one value per index of I_t instead of n.
+ *                  Default 0.  Any time between steps.
  *   "worker_chunk" workers whose tables are accumulated concurrently by the sketch kernel (0 = automatic,
  *                  sized so that the concurrently updated tables stay resident in L2).
  *   "sketch_ctas_per_sm" grid size of the plain sketch kernel in blocks per SM (default 64: one tile per block).

@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsketched_amsgrad.so")
-SOURCES = ["sk_api.cu", "sk_sketch.cu", "sk_sketch_win.cu", "sk_sketch_own.cu", "sk_select.cu", "sk_static.cu", "sk_shard.cu"]
+SOURCES = ["sk_api.cu", "sk_sketch.cu", "sk_sketch_own.cu", "sk_select.cu", "sk_static.cu", "sk_shard.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
 

@@ -17,6 +17,8 @@ namespace {
 
 thread_local std::string g_err;
 
+constexpr uint32_t kDefaultWindowLines = 8;
+
 int fail(int code, const char* fmt, ...) {
     char buf[512];
     va_list ap;
@@ -144,14 +146,12 @@ int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, ui
     sk::MomentArgs A = moment_args(s, grads);
     // the windowed kernel implements Algorithm 2 with one table per worker only
     const bool windowed = vec && P.win_cw != 0 && s->variant == 0 && !s->sum_sketch;
-    const bool own = windowed && s->window_kernel == 1;      // accumulation by ownership: one warp per worker
-    const uint32_t wc = own ? std::min<uint32_t>(std::min<uint32_t>((uint32_t)s->window_workers, sk::kOwnMaxWorkers), P.n)
-                      : windowed ? std::min<uint32_t>(std::min<uint32_t>((uint32_t)s->window_workers, sk::kWinMaxWorkers), P.n)
+    const uint32_t wc = windowed ? std::min<uint32_t>(std::min<uint32_t>((uint32_t)s->window_workers, sk::kOwnMaxWorkers), P.n)
                                  : chunk_of(s);
     // With a second round the sketch kernel also leaves sum_w a^(w) per coordinate, so that each of the P*k exact
     // values costs one gather instead of n (not the windowed kernel, and not a partitioned step, whose exact values
     // are exchanged: there every local worker's value is gathered).
-    A.asum = ((s->cand_mult > 1 || s->always_asum) && (!windowed || own) && !sharded) ? s->asum : nullptr;
+    A.asum = ((s->cand_mult > 1 || s->always_asum) && !sharded) ? s->asum : nullptr;
     s->asum_live = A.asum != nullptr;
     const uint64_t tfloats = (uint64_t)P.r * P.cs;
     float* sum_out = sharded ? x1 : s->sum;
@@ -172,8 +172,7 @@ int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, ui
         }
         StageTimer tm(s, 2);     // moments + sketch; also leaves the gradient sums on I_{t-1} in gsum
         if (windowed) {
-            const int l = own ? sk::launch_moment_sketch_own(P, A, w0, nw, s->sm_count, st)
-                              : sk::launch_moment_sketch_win(P, A, w0, nw, (uint32_t)s->window_red_rows, s->sm_count, st);
+            const int l = sk::launch_moment_sketch_own(P, A, w0, nw, s->sm_count, st);
             if (l < 0) return fail(SK_ECUDA, "the windowed sketch kernel does not fit in shared memory (window_lines=%lld, r=%u)",
                                    (long long)s->window_lines, P.r);
             tm.done(l);
@@ -338,6 +337,9 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     uint32_t lg = 5;
     while ((1u << lg) > c) --lg;
     P.log2g = lg;
+    // default family: groups of 32 confined to windows of kDefaultWindowLines lines, which lets the sketch accumulate
+    // on chip; rows too short for one window keep the plain family
+    if (lg == 5 && c >= 32u * kDefaultWindowLines) s->window_lines = kDefaultWindowLines;
     refresh_hash(s);
 
     const uint64_t nd = (uint64_t)n * d, tf = (uint64_t)r * P.cs;
@@ -609,19 +611,9 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         s->variant = value;
         return SK_OK;
     }
-    if (!strcmp(key, "window_red_rows")) {
-        if (value < 0 || value > 4) return fail(SK_EINVAL, "window_red_rows must be in 0..4");
-        s->window_red_rows = value;
-        return SK_OK;
-    }
     if (!strcmp(key, "window_workers")) {
         if (value < 1 || value > (int64_t)sk::kOwnMaxWorkers) return fail(SK_EINVAL, "window_workers must be in 1..8");
         s->window_workers = value;
-        return SK_OK;
-    }
-    if (!strcmp(key, "window_kernel")) {
-        if (value != 0 && value != 1) return fail(SK_EINVAL, "window_kernel must be 0 (producer/consumer roles) or 1 (ownership)");
-        s->window_kernel = value;
         return SK_OK;
     }
     if (!strcmp(key, "worker_sum")) {
@@ -656,7 +648,6 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     if (!strcmp(key, "log2g")) *value = s->P.log2g;
     else if (!strcmp(key, "window_lines")) *value = s->window_lines;
     else if (!strcmp(key, "window_workers")) *value = s->window_workers;
-    else if (!strcmp(key, "window_kernel")) *value = s->window_kernel;
     else if (!strcmp(key, "worker_sum")) *value = s->always_asum;
     else if (!strcmp(key, "variant")) *value = s->variant;
     else if (!strcmp(key, "P")) *value = s->cand_mult;
@@ -664,7 +655,6 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     else if (!strcmp(key, "freeze_v")) *value = s->freeze_v;
     else if (!strcmp(key, "sum_sketch")) *value = s->sum_sketch;
     else if (!strcmp(key, "grads_bf16")) *value = s->grads_bf16;
-    else if (!strcmp(key, "window_red_rows")) *value = s->window_red_rows;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
     else if (!strcmp(key, "sketch_ctas_per_sm")) *value = s->sketch_ctas_per_sm;

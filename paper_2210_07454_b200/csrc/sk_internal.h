@@ -67,10 +67,6 @@ int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st);
 int launch_set_bits(const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st);
 int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,
                          cudaStream_t st);
-// windowed hash family: shared-memory accumulation, at most kWinMaxWorkers workers per launch; -1 if it cannot run
-constexpr uint32_t kWinMaxWorkers = 4;
-int launch_moment_sketch_win(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, uint32_t r_red,
-                             int sm_count, cudaStream_t st);
 // windowed hash family, accumulation by ownership (one warp per worker, block-owned windows): at most kOwnMaxWorkers
 // workers per launch; fills A.asum when it is set; -1 if it cannot run
 constexpr uint32_t kOwnMaxWorkers = 8;

@@ -26,8 +26,6 @@ struct sk_state {
     int64_t variant = 0;          // 0 = gradient averaging (Algorithm 2), 1 = parameter averaging (Algorithm 1)
     float *vw = nullptr, *vhatw = nullptr;   // per-worker v, vhat of the parameter-averaging variant (n*d each)
     int64_t window_workers = 8;
-    int64_t window_red_rows = 0;
-    int64_t window_kernel = 1;    // 1: accumulation by ownership (sk_sketch_own.cu); 0: producer/consumer roles (sk_sketch_win.cu)
     int64_t always_asum = 0;      // the sketch kernel leaves sum_w a^(w) for the update of x even without a second round
     int64_t sketch_ctas_per_sm = 64;
     bool timing = false;

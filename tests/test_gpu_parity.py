@@ -49,18 +49,19 @@ def test_hash_bit_exact(log2g, c):
     b = _binding()
     d, r = 300_000, 7
     gpu = b.SketchedAMSGrad(d, 1, r, c, 1, seed=12345, log2g=log2g)
+    L = gpu.get_option("window_lines")               # groups of 32 come with the windowed family by default
     idx = torch.empty(d, dtype=torch.int32, device="cuda")
     sgn = torch.empty(d, dtype=torch.int8, device="cuda")
     for row in range(r):
         gpu.hash(row, 0, d, idx, sgn)
         gpu.sync()
-        wb, ws = oracle.hash_family(12345, log2g, c, row, 0, d)
+        wb, ws = oracle.hash_family(12345, log2g, c, row, 0, d, window_lines=L)
         assert np.array_equal(idx.cpu().numpy().view(np.uint32), wb)
         assert np.array_equal(sgn.cpu().numpy(), ws)
     # far end of the coordinate range
     gpu.hash(3, 2**32 - 1000, 1000, idx, sgn)
     gpu.sync()
-    wb, ws = oracle.hash_family(12345, log2g, c, 3, 2**32 - 1000, 1000)
+    wb, ws = oracle.hash_family(12345, log2g, c, 3, 2**32 - 1000, 1000, window_lines=L)
     assert np.array_equal(idx[:1000].cpu().numpy().view(np.uint32), wb)
     assert np.array_equal(sgn[:1000].cpu().numpy(), ws)
 
@@ -167,17 +168,19 @@ def test_windowed_edge_cases(case):
     _run_steps(w, 3, cfg_id=8, window_lines=L)
 
 
-@pytest.mark.parametrize("red_rows", [0, 1, 3, 4])
-def test_windowed_rows_split_between_reductions_and_windows(red_rows):
-    # the windowed kernel sketches the first rows by L2 reductions and the rest in shared-memory windows;
-    # every split must give the same tables
-    w = _workload("C1", name="E", d=1024 * 21 + 64, n=5, r=5, c=4096, k=300, steps=2, recipe="planted")
+@pytest.mark.parametrize("workers,worker_sum", [(1, 0), (2, 1), (3, 0), (5, 1), (8, 0)])
+def test_windowed_worker_chunks_and_worker_sum(workers, worker_sum):
+    # the ownership kernel runs one warp per worker: every split of the workers into launches (block sizes of
+    # 32 .. 256 threads, running sums carried over launches), with and without the worker sum of a_t that the update
+    # of x can read, must give the same step
+    w = _workload("C1", name="E", d=1024 * 21 + 64, n=5, r=5, c=4096, k=300, steps=3, recipe="planted")
     gpu, ora = _pair(w, window_lines=8)
-    gpu.set_option("window_red_rows", red_rows)
+    gpu.set_option("window_workers", workers)
+    gpu.set_option("worker_sum", worker_sum)
     src = _source(w, cfg_id=8)
     x = src.x0()
     x_ref = x.cpu().numpy().copy()
-    for t in (1, 2):
+    for t in (1, 2, 3):
         g = src.grads(t)
         if t > 1:
             force_state(gpu, ora)
@@ -298,7 +301,7 @@ def test_second_round_integer_inputs_are_bit_exact(chunk):
     b = _binding()
     gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0, P=P)
     ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=gpu.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
-                        threads=8, P=P)
+                        threads=8, P=P, window_lines=gpu.get_option("window_lines"))
     gpu.set_option("worker_chunk", chunk)            # workers in several launches: the running sums carry over
     gen = torch.Generator(device="cuda").manual_seed(5)
     x = torch.zeros(d, device="cuda")
@@ -441,7 +444,7 @@ def test_sketch_of_the_worker_sum_integer_inputs_bit_exact():
     gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0)
     gpu.set_option("sum_sketch", 1)
     ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=gpu.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
-                        threads=8)
+                        threads=8, window_lines=gpu.get_option("window_lines"))
     gen = torch.Generator(device="cuda").manual_seed(5)
     x = torch.zeros(d, device="cuda")
     x_ref = np.zeros(d, np.float32)
@@ -485,7 +488,7 @@ def test_integer_inputs_are_bit_exact():
     b = _binding()
     gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0)
     ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=gpu.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
-                        threads=8)
+                        threads=8, window_lines=gpu.get_option("window_lines"))
     gen = torch.Generator(device="cuda").manual_seed(5)
     x = torch.zeros(d, device="cuda")
     x_ref = np.zeros(d, np.float32)
@@ -556,7 +559,8 @@ def test_checkpoint_roundtrip():
     assert np.array_equal(a.get("I"), c2.get("I"))
     close(xb.cpu().numpy(), xa.cpu().numpy(), "x after resume")
     close(c2.get("e"), a.get("e"), "e after resume", groups_axis=0)
-    assert np.array_equal(c2.get("v"), a.get("v"))
+    # the gradient sums behind v are accumulated in arrival order (as the sketch tables are): equal to rounding
+    np.testing.assert_allclose(c2.get("v"), a.get("v"), rtol=1e-6, atol=0)
 
 
 def test_host_step_matches_device_step():

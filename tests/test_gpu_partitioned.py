@@ -144,7 +144,7 @@ def test_c1_sketch_of_the_local_worker_sum():
     for h in ranks.handles:
         h.set_option("sum_sketch", 1)
     ora = oracle.Oracle(w.d, w.n, w.r, w.c, w.k, seed=w.seed, log2g=ranks.get_option("log2g"), lr=w.lr, beta1=w.beta1,
-                        beta2=w.beta2, eps=w.eps, threads=8, P=2)
+                        beta2=w.beta2, eps=w.eps, threads=8, P=2, window_lines=ranks.get_option("window_lines"))
     src = GradientSource(w, device="cuda")
     x_ref = src.x0().cpu().numpy().copy()
     xs = [src.x0() for _ in ranks.handles]
@@ -195,7 +195,7 @@ def test_integer_inputs_are_bit_exact_and_equal_the_unpartitioned_step():
     w = synthetic.Workload("E", d, n, r, c, k, 1, "planted", seed=9, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0)
     ranks = Ranks(w, (1, 2, 1), P=P)
     ora = oracle.Oracle(d, n, r, c, k, seed=9, log2g=ranks.get_option("log2g"), lr=0.5, beta1=0.0, beta2=0.5, eps=1.0,
-                        threads=8, P=P)
+                        threads=8, P=P, window_lines=ranks.get_option("window_lines"))
     gen = torch.Generator(device="cuda").manual_seed(5)
     xs = [torch.zeros(d, device="cuda") for _ in range(3)]
     x_ref = np.zeros(d, np.float32)
