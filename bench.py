@@ -27,12 +27,16 @@ METRIC = "sketched_amsgrad_step_throughput"
 UNIT = "Gcoord/s"
 DEFAULT_WORKLOAD = "C3"      # d = 25.6M: the size the headline metric is quoted on
 
-# DRAM traffic of the dominant kernel (moments + sketch) from an ncu capture, in bytes per worker-coordinate,
-# valid only for the kernel source it was taken on (sha256 of sk_sketch.cu); otherwise reported as null.
-# Capture: C3 at half size (profiles/c3_half_moment_sketch_ncu_full.md): 1.2539 GB read + 0.7941 GB written for
-# 1.024e8 worker-coordinates; the traffic grows in proportion to n*d, so it is scaled to the timed launch.
-NCU_TRAFFIC = {"sha256": "0bdcf8570d0f285945aa41d187337492869ba658f80dc563b760b74395264035",
-               "bytes_per_worker_coord": 20.00}
+# DRAM traffic of the dominant kernel (moments + sketch) from an ncu capture, in bytes per worker-coordinate, valid
+# only for the kernel source it was taken on (sha256 of the file); otherwise reported as null.  The traffic grows in
+# proportion to n*d, so the capture (C3 at half size, see profiles/) is scaled to the timed launch.
+NCU_TRAFFIC = {
+    # shared-memory ownership kernel (windowed hash family, the default path)
+    "k_moment_sketch_own": {"file": "sk_sketch_own.cu", "sha256": None, "bytes_per_worker_coord": None},
+    # L2-reduction kernel (plain hash family): 1.2539 GB read + 0.7941 GB written for 1.024e8 worker-coordinates
+    "k_moment_sketch_v4": {"file": "sk_sketch.cu", "sha256": "0bdcf8570d0f285945aa41d187337492869ba658f80dc563b760b74395264035",
+                           "bytes_per_worker_coord": 20.00},
+}
 
 
 def _peaks():
@@ -47,7 +51,7 @@ def _peaks():
 
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -57,12 +61,22 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                          "-lms", "50", "-i", str(self.gpu)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def _stamp(text: str):
+        import datetime
+        try:
+            return datetime.datetime.strptime(text, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
+    def stop(self, windows=()):
+        """windows: (t0, t1) wall-clock intervals (time.time()) of the timed repetitions; returns the summary over the
+        samples inside them (all samples if none fall inside) and the median SM clock of every window."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
@@ -72,21 +86,30 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, mx, reasons = [], [], set()
+        rows, mx = [], []
         for line in out.splitlines():
-            f = [s.strip() for s in line.split(",")]
+            f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
             try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
+                rows.append((self._stamp(f[0]), float(f[1]), [v.lower().startswith("active") for v in f[5:9]]))
+                mx.append(float(f[2]))
             except ValueError:
                 continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                if val.lower().startswith("active"):
+        inside = [r for r in rows if r[0] is not None and any(a <= r[0] <= b for a, b in windows)]
+        use = inside if inside else rows
+        reasons = set()
+        for _, _, flags in use:
+            for name, on in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), flags):
+                if on:
                     reasons.add(name)
-        busy = [v for v in sm if v >= 0.5 * max(sm)] if sm else []
-        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        per_rep = []
+        for a, b in windows:
+            v = [r[1] for r in rows if r[0] is not None and a <= r[0] <= b]
+            per_rep.append(statistics.median(v) if v else None)
+        return {"sm_mhz": statistics.median([r[1] for r in use]) if use else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(rows), "samples_in_timed_region": len(inside),
+                "sm_mhz_per_repetition": per_rep}
 
 
 def _dist():
@@ -117,17 +140,27 @@ def reduce_sum(value: float, world: int, device) -> float:
     return float(t.item())
 
 
-def cpu_oracle_rate(w, scale: int, steps: int, threads: int, variant: str = "ga", P: int = 1):
-    """Times the CPU oracle, as it stands, on `steps` steps of the workload scaled down by `scale`."""
+def default_family(c: int):
+    """The library's default hash family for a row of c buckets: groups of 32 in windows of 8 lines when a row holds a
+    window, else the plain family with the largest group that fits (restated here for the oracle's arguments)."""
+    lg = 5
+    while (1 << lg) > c:
+        lg -= 1
+    return lg, (8 if lg == 5 and c >= 256 else 0)
+
+
+def cpu_oracle_rate(w, scale: int, steps: int, threads: int, variant: str = "ga", P: int = 1, family=None):
+    """Times the CPU oracle, as it stands, on `steps` steps of the workload scaled down by `scale`.
+    family: (log2g, window_lines) of the hash family (default: the library's default for the scaled row length)."""
     import oracle
     from paper_2210_07454_b200 import synthetic
     ws = synthetic.scaled(w, scale) if scale > 1 else w
     src = synthetic.GradientSource(ws, device="cpu", cfg_id=int(w.name[1]) if w.name[1:2].isdigit() else 9)
-    lg = 5
-    while (1 << lg) > ws.c:
-        lg -= 1
+    lg, wl = family if family is not None else default_family(ws.c)
+    if scale > 1 and (wl * 32 > ws.c or (1 << lg) > ws.c):
+        lg, wl = default_family(ws.c)
     o = oracle.Oracle(ws.d, ws.n, ws.r, ws.c, ws.k, seed=ws.seed, log2g=lg, lr=ws.lr, beta1=ws.beta1, beta2=ws.beta2,
-                      eps=ws.eps, threads=threads, variant=variant, P=P)
+                      eps=ws.eps, threads=threads, variant=variant, P=P, window_lines=wl)
     x = src.x0().numpy()
     grads = [src.grads(t).numpy() for t in range(1, min(steps, 2) + 1)]
     times = []
@@ -135,18 +168,39 @@ def cpu_oracle_rate(w, scale: int, steps: int, threads: int, variant: str = "ga"
         t0 = time.perf_counter()
         o.step(grads[t % len(grads)], x)
         times.append(time.perf_counter() - t0)
-    sample = (f"{steps} step(s) of {w.name} scaled 1/{scale} (d={ws.d}, n={ws.n}, r={ws.r}, c={ws.c}, k={ws.k}), "
-              f"gcc -O2 OpenMP oracle")
+    o.close()
+    size = "at full size" if scale == 1 else f"scaled 1/{scale}"
+    sample = (f"{steps} step(s) of {w.name} {size} (d={ws.d}, n={ws.n}, r={ws.r}, c={ws.c}, k={ws.k}), "
+              f"gcc -O2 OpenMP oracle, {threads} thread(s)")
     return ws, times, sample
 
 
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def run_reference(args, w):
+    """The reference arm: there is no reference code, so it is the CPU oracle itself on all host cores.  Each step is
+    one oracle step of the workload; at full size when the whole run then stays within a few minutes (probed on a
+    1/16-size step first), else at the smallest power-of-two reduction that does."""
     world, rank, _ = _dist()
     if rank != 0:
         return
     threads = os.cpu_count() or 1
-    scale = args.ref_scale
     total = args.steps + args.warmup
+    scale = args.ref_scale
+    if scale <= 0:                                    # automatic: full size if (steps + warmup) oracle steps fit the budget
+        _, probe, _ = cpu_oracle_rate(w, 16, 2, threads, args.variant, args.P)
+        full_step = 16.0 * probe[-1]
+        scale = 1
+        while total * full_step / scale > 200.0 and scale < 64:
+            scale *= 2
     ws, times, sample = cpu_oracle_rate(w, scale, total, threads, args.variant, args.P)
     timed = times[args.warmup:]
     ms = 1e3 * sum(timed) / len(timed)
@@ -155,11 +209,47 @@ def run_reference(args, w):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k,
-                       "sampled_as": f"each step is one oracle step at 1/{scale} size"},
+                       "sampled_as": "each step is one oracle step at full size" if scale == 1
+                       else f"each step is one oracle step at 1/{scale} size", "same_config": scale == 1,
+                       "cpu": cpu_model()},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def quick_step_roofline(name: str, dev, peak: float, steps: int = 5, reps: int = 3):
+    """A short run of another workload with the default options: step time (median of `reps` loops of `steps` steps
+    after 3 warm-up steps, two rotating gradient sets, both far larger than L2) and its fraction of the roofline."""
+    import torch
+    from paper_2210_07454_b200 import binding, synthetic
+    w = synthetic.WORKLOADS[name]
+    src = synthetic.GradientSource(w, device=dev, cfg_id=int(w.name[1]))
+    opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
+    gsets = [src.grads(1), src.grads(2)]
+    x = src.x0()
+    for t in range(3):
+        opt.step(gsets[t % 2], x)
+    opt.sync()
+    ms = []
+    for _ in range(reps):
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for t in range(steps):
+            opt.step(gsets[t % 2], x)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms.append(ev0.elapsed_time(ev1) / steps)
+    opt.sync()
+    ms_step = statistics.median(ms)
+    b_alg = opt.algorithmic_bytes()
+    out = {"d": w.d, "n": w.n, "r": w.r, "c": w.c, "k": w.k, "ms_per_step": ms_step, "steps": steps, "repetitions": reps,
+           "value": w.n * w.d / (ms_step * 1e-3) / 1e9, "unit": UNIT, "algorithmic_bytes": b_alg,
+           "achieved_gbs": b_alg / (ms_step * 1e-3) / 1e9, "frac": b_alg / (ms_step * 1e-3) / 1e9 / peak}
+    del opt, gsets, x, src
+    torch.cuda.empty_cache()
+    return out
 
 
 def main():
@@ -180,7 +270,9 @@ def main():
     ap.add_argument("--worker-chunk", type=int, default=0)
     ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--ref-scale", type=int, default=16)
+    ap.add_argument("--ref-scale", type=int, default=0, help="reference arm: 1/SCALE size per step (0 = full size if it fits the time budget)")
+    ap.add_argument("--reps", type=int, default=10, help="repetitions of the --steps long timed loop; the median is reported")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the short C4 and C5 runs reported beside the headline")
     ap.add_argument("--scale", type=int, default=1, help="run the workload at 1/SCALE size (profiling captures)")
     ap.add_argument("--grad-sets", type=int, default=0, help="rotating gradient sets (0 = as many as fit, 2..4)")
     ap.add_argument("--partition-workers", action="store_true",
@@ -210,6 +302,9 @@ def main():
     dev = torch.device("cuda", local)
     if world > 1:
         import torch.distributed as dist
+        if args.partition_workers:                   # the communicator's set-up lines (ranks, transports) go to stderr
+            os.environ.setdefault("NCCL_DEBUG", "INFO")
+            os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
         dist.init_process_group("nccl", device_id=dev)
 
     n_all = w.n
@@ -258,18 +353,28 @@ def main():
         import torch.distributed as dist
         dist.barrier()
     torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for t in range(args.steps):
-        step(gsets[(args.warmup + t) % nsets], x)
-    ev1.record()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    # the --steps long loop is timed `reps` times (CUDA events on the launching stream, barrier and synchronize on both
+    # sides of every repetition, max over ranks); the median repetition is the reported step time
+    rep_ms, windows = [], []
+    for rep in range(max(1, args.reps)):
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        ev0.record()
+        for t in range(args.steps):
+            step(gsets[(args.warmup + t) % nsets], x)
+        ev1.record()
+        torch.cuda.synchronize()
+        windows.append((t0, time.time()))
+        if world > 1:
+            dist.barrier()
+        rep_ms.append(reduce_max(ev0.elapsed_time(ev1), world, dev))
+    clocks = sampler.stop(windows) if rank == 0 else None
     opt.sync()
-    ms_total = reduce_max(ev0.elapsed_time(ev1), world, dev)
-    _, _, stage_launches = opt.timing()              # launch counts of the timed loop
+    ms_total = statistics.median(rep_ms)
+    _, _, stage_launches = opt.timing()              # launch counts of all timed repetitions
     launches = reduce_sum(float(sum(stage_launches)), world, dev)
     # per-stage times: the same steps once more with CUDA events around every stage (inside the library, on its stream)
     nsteps, stage_ms = 0, [0.0] * binding.NUM_STAGES
@@ -297,12 +402,16 @@ def main():
         k1_ms = stage_ms[2] / k1_launches
         k1_bytes = k1_bytes_step * args.steps / k1_launches
         achieved = k1_bytes / (k1_ms * 1e-3) / 1e9
-        sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2210_07454_b200", "csrc", "sk_sketch.cu"), "rb").read()).hexdigest()
+        windowed = bool(opt.get_option("window_lines")) and args.variant == "ga" and not args.sum_sketch
+        kernel = "k_moment_sketch_pa_v4" if args.variant != "ga" else ("k_moment_sketch_own" if windowed else "k_moment_sketch_v4")
         traffic = None
-        if NCU_TRAFFIC["sha256"] == sha and NCU_TRAFFIC["bytes_per_worker_coord"] and args.variant == "ga" \
-                and not args.grads_bf16 and not args.sum_sketch and args.P == 1 and not opt.get_option("window_lines"):
-            traffic = NCU_TRAFFIC["bytes_per_worker_coord"] * w.n * w.d * args.steps / k1_launches
-        roofline = {"bound": "hbm", "kernel": "k_moment_sketch_v4" if args.variant == "ga" else "k_moment_sketch_pa_v4", "achieved": achieved, "peak": peak,
+        rec = NCU_TRAFFIC.get(kernel)
+        if rec and rec["sha256"] and rec["bytes_per_worker_coord"] and not args.grads_bf16 and not args.sum_sketch \
+                and args.P == 1 and args.worker_sum <= 0:
+            path = os.path.join(ROOT, "paper_2210_07454_b200", "csrc", rec["file"])
+            if hashlib.sha256(open(path, "rb").read()).hexdigest() == rec["sha256"]:
+                traffic = rec["bytes_per_worker_coord"] * w.n * w.d * args.steps / k1_launches
+        roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                     "ms_per_launch": k1_ms, "launches_per_step": k1_launches / args.steps,
                     "algorithmic_bytes_per_launch": k1_bytes}
@@ -357,15 +466,28 @@ def main():
                       "ms_per_step": 1e3 * dt / args.e2e_steps, "steps": args.e2e_steps,
                       "api": "sk_step_host_sparse: parameters resident on the device, sparse update returned"}
 
+    fam = (opt.get_option("log2g"), opt.get_option("window_lines"))
+    hash_group, worker_chunk = 1 << fam[0], opt.get_option("worker_chunk")
+    # the other configurations of d >= 25.6M the roofline target covers, in short runs with the default options
+    others = None
+    if world == 1 and not args.no_other_workloads and args.workload == DEFAULT_WORKLOAD and args.scale == 1:
+        del opt, gsets, x
+        torch.cuda.empty_cache()
+        others = {name: quick_step_roofline(name, dev, peak) for name in ("C4", "C5")}
+
     if rank != 0:
         return
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
+        # the oracle as it stands, at the benchmark's own size: two steps on all host cores (the second is reported:
+        # from it on I_{t-1} is not empty), and one step on a single thread
         threads = os.cpu_count() or 1
-        scale = 4
-        ws, times, sample = cpu_oracle_rate(w, scale, 3, threads, args.variant, args.P)
-        cpu = {"value": ws.n * ws.d / (sum(times[1:]) / len(times[1:])) / 1e9, "unit": UNIT, "cores": threads,
-               "kind": "oracle", "sample": sample}
+        ws, times, sample = cpu_oracle_rate(w, 1, 2, threads, args.variant, args.P, family=fam)
+        _, times1, sample1 = cpu_oracle_rate(w, 1, 1, 1, args.variant, args.P, family=fam)
+        cpu = {"value": ws.n * ws.d / times[-1] / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+               "seconds_per_step": times[-1], "cpu": cpu_model(),
+               "single_thread": {"value": ws.n * ws.d / times1[-1] / 1e9, "unit": UNIT, "cores": 1,
+                                 "seconds_per_step": times1[-1], "sample": sample1}}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -374,21 +496,25 @@ def main():
             "config": {"sketches": "one, of the worker sum (linearity; not the headline path)" if args.sum_sketch
                        else "one per worker, then summed", "gradient_storage": "bf16" if args.grads_bf16 else "f32",
                        "workload": w.name, "d": w.d, "n": n_all, "r": w.r, "c": w.c, "k": w.k,
-                       "recipe": w.recipe, "variant": args.variant, "P": args.P, "hash_group": 1 << opt.get_option("log2g"),
-                       "window_lines": opt.get_option("window_lines"),
-                       "worker_chunk": opt.get_option("worker_chunk"),
+                       "recipe": w.recipe, "variant": args.variant, "P": args.P, "hash_group": hash_group,
+                       "window_lines": fam[1], "worker_chunk": worker_chunk,
                        "replicas": 1 if args.partition_workers else world,
                        "workers_per_process": w.n, "partitioned": bool(args.partition_workers),
                        "stage_times": "a second pass of the same steps with CUDA events around every stage; "
                                       "ms_per_step is from the pass without them",
-                       "l2": f"inputs larger than L2: {nsets} rotating gradient sets of {set_bytes / 1e9:.2f} GB"},
+                       "l2": f"inputs larger than L2: {nsets} rotating gradient sets of {set_bytes / 1e9:.2f} GB",
+                       "repetitions": len(rep_ms),
+                       "timing": "ms_per_step is the median over the repetitions of (time of --steps steps) / steps",
+                       "ms_per_step_min": min(rep_ms) / args.steps, "ms_per_step_max": max(rep_ms) / args.steps},
             "steps_per_s": 1e3 / ms_step,
             "step_roofline": {"algorithmic_bytes": b_alg, "achieved_gbs": b_alg / (ms_step * 1e-3) / 1e9,
                               "peak_gbs": peak, "peak_kind": f"of {peak_kind}",
                               "frac": b_alg / (ms_step * 1e-3) / 1e9 / peak},
             "roofline": roofline,
             "stage_ms_per_step": {nm: stage_ms[q] / max(1, nsteps) for q, nm in enumerate(binding.STAGE_NAMES)},
-            "cpu_baseline": cpu, "e2e": e2e, "e2e_sparse_return": e2e_sparse, "gpu_launches": int(launches), "clocks": clocks}
+            "cpu_baseline": cpu, "e2e": e2e, "e2e_sparse_return": e2e_sparse, "gpu_launches": int(launches),
+            "gpu_launches_per_step": launches / (world * args.steps * len(rep_ms)), "clocks": clocks,
+            "other_workloads": others}
     print(json.dumps(line), flush=True)
 
 

@@ -114,8 +114,33 @@ void sk_destroy(sk_state* state);
 
 /* stream: a cudaStream_t cast to void* (NULL = default stream).  The handle does not own it. */
 int sk_set_stream(sk_state* state, void* stream);
-/* Waits for everything enqueued on the handle's stream and reports the device status word. */
+/* Waits for everything enqueued on the handle's stream and reports the device status word: SK_EDEVICE with a
+ * message if it is not zero, after which the word is cleared (the handle stays usable).  Bit 0: a selection emitted a
+ * number of indices other than k.  Bits 1..5 exist in the debug build (compiled with -DSK_DEBUG=1, see
+ * paper_2210_07454_b200/build.py --debug), whose kernels compare every hashed table offset, coordinate index, list
+ * position, histogram bin and shared-memory window offset with the size of what it addresses, record a violation
+ * here and skip the access; nothing traps. */
 int sk_sync(sk_state* state);
+
+/* Per-step statistics of the last step's selection (Algorithm 2's Top-k) and the method's exchange volume, for
+ * logging: out[0] = the threshold key's leading 24 bits as an fp32 value (a lower bound of the k-th largest
+ * |estimate|, within 2^-16 relative), out[1] = coordinates whose key fell into the threshold's 4096-way bin,
+ * out[2] = coordinates sharing the threshold's leading 24 key bits (the tie group resolved exactly),
+ * out[3] = indices emitted (k unless the status word says otherwise), out[4] = floats one iteration puts on the wire
+ * by Section III-B's count, r*c + P*k + 2k (r*c + P*k + k for Algorithm 1), out[5] = the device status word.
+ * `out` is a HOST array of at least SK_NUM_STATS doubles.  Synchronises the stream. */
+#define SK_NUM_STATS 6
+int sk_get_stats(sk_state* state, double* out, uint32_t count);
+
+/* Test hooks (host side; neither touches the GPU's state).
+ * sk_test_fail_allocation(nth): the (nth+1)-th device allocation of the following sk_create calls fails as if the
+ * device were out of memory (sk_create then returns NULL with a message and frees what it had allocated); nth < 0
+ * switches the hook off.  Process-wide; not thread-safe.
+ * sk_debug_check(state, kind), kind 1..5: in the debug build a one-thread kernel runs the bounds check of that kind
+ * with a false condition (no access is made), so the next sk_sync must report bit `kind`; SK_ESTATE in the normal
+ * build, which has no device-side checks.  The paper has no counterpart for either. */
+int sk_test_fail_allocation(int64_t nth);
+int sk_debug_check(sk_state* state, uint32_t kind);
 
 /* Options (integers):
  *   "log2g"        hash group size g = 2^log2g, 0..5 (Section II-C fixes no hash family; see sk_hash).
@@ -173,6 +198,8 @@ int sk_hash(const sk_state* state, uint32_t row, uint64_t i0, uint64_t count,
  *   "v","vhat" d   second moments ("v" is brought up to date with the decay it is owed before export)
  *   "tables"  n*r*c  the worker sketches S_t^(w) of the last step;  "sum"  r*c  the aggregate S_t
  *   "est"     d    the estimates of the last step (recomputed on request from "sum" and "vhat"; get only)
+ *   "keys"    d uint32  the ranking keys the last step's selection ran on: the bit pattern of |median * rsqrt(vhat)|
+ *                  (of |median| for Algorithm 1), as the key pass stored them (get only, after the first step)
  *   "I"       k uint32  I_t of the last step, ascending (get);  set: installs I_{t-1} for the next step
  *   "vw","vhatw" n*d  per-worker second moments (parameter-averaging variant only; "v","vhat" are then unavailable)
  *   "cand"    P*k uint32  candidates of the last step's second round, ascending (get only; empty when P = 1)
@@ -207,10 +234,16 @@ int sk_get_timing(sk_state* state, double* ms, uint64_t* launches);
  * all its scratch (histograms, ranking keys, candidate lists; about 5 MB) lives in one file-scope device array
  * inside the library, which every GPU that loads the library holds until the process exits.
  *   - Limit: d <= SK_STATIC_MAX_D; larger handles are rejected with SK_EINVAL and a message naming the limit.
- *     SK_ESTATE if the handle has not taken a step yet, or runs a second round (P > 1), whose exact values
- *     this entry point does not fetch.
- *   - The first call on a device resolves the device address of the scratch array (once per device, with that
- *     device current).  Make that first call before starting any stream capture.
+ *     SK_ESTATE if the handle has not taken a step yet, is in the middle of a partitioned step, or runs a second
+ *     round (P > 1), whose exact values this entry point does not fetch.
+ *   - The device address of the scratch array is resolved once per device, with that device current: by sk_create
+ *     (which is allowed to allocate, and so absorbs whatever loading the array's module costs) for every handle
+ *     with d <= SK_STATIC_MAX_D, else by the first call of this entry point on the device -- make that first call
+ *     before starting any stream capture.  The call launches only kernels the handle's last step has already
+ *     launched, so nothing is loaded lazily either: it is allocation-free once a handle exists on the device and
+ *     has taken a step.
+ *   - What the selection finds wrong (a count other than k; in the debug build any out-of-range position) is
+ *     OR-ed into the handle's status word, which sk_sync reports.
  *   - Every call, from every handle and stream, shares the one array, and the array keeps the previous call's
  *     contents; the entry point clears the parts that must start at zero itself.  Two calls that overlap on the
  *     GPU (different streams or threads) race on the array: serialise them.

@@ -11,11 +11,15 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsketched_amsgrad.so")
+# SKETCHED_AMSGRAD_LIB selects another build of the same library (e.g. the bounds-checked one)
+LIB_PATH = os.environ.get("SKETCHED_AMSGRAD_LIB") or os.path.join(_HERE, "libsketched_amsgrad.so")
 
 EXPORTS = ["sk_create", "sk_step", "sk_set_lr", "sk_step_host", "sk_step_host_sparse", "sk_destroy", "sk_set_stream", "sk_sync", "sk_set_option",
            "sk_get_option", "sk_hash", "sk_get", "sk_set", "sk_algorithmic_bytes", "sk_get_timing", "sk_select_static",
-           "sk_exchange_floats", "sk_step_local", "sk_step_select", "sk_step_finish", "sk_last_error", "sk_version"]
+           "sk_exchange_floats", "sk_step_local", "sk_step_select", "sk_step_finish", "sk_last_error", "sk_version",
+           "sk_get_stats", "sk_test_fail_allocation", "sk_debug_check"]
+NUM_STATS = 6
+STAT_NAMES = ["threshold", "threshold_bin_count", "tie_group_count", "emitted", "floats_on_the_wire", "status"]
 STATIC_MAX_D = 262144
 NUM_STAGES = 8
 STAGE_NAMES = ["zero_tables", "second_moment", "moment_sketch", "sum_tables", "unsketch_hist",
@@ -54,6 +58,9 @@ def lib() -> C.CDLL:
         L.sk_get_timing.restype = C.c_int
         L.sk_get_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u64)]
         L.sk_select_static.restype = C.c_int; L.sk_select_static.argtypes = [vp, vp]
+        L.sk_get_stats.restype = C.c_int; L.sk_get_stats.argtypes = [vp, C.POINTER(C.c_double), u32]
+        L.sk_test_fail_allocation.restype = C.c_int; L.sk_test_fail_allocation.argtypes = [i64]
+        L.sk_debug_check.restype = C.c_int; L.sk_debug_check.argtypes = [vp, u32]
         L.sk_exchange_floats.restype = u64; L.sk_exchange_floats.argtypes = [vp, C.c_int]
         L.sk_step_local.restype = C.c_int; L.sk_step_local.argtypes = [vp, vp, vp]
         L.sk_step_select.restype = C.c_int; L.sk_step_select.argtypes = [vp, vp, vp]
@@ -91,6 +98,7 @@ class SketchedAMSGrad:
     def __init__(self, d, n, r, c, k, seed=0, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, log2g=None,
                  window_lines=None, variant="ga", P=1, workers_total=None):
         self.d, self.n, self.r, self.c, self.k = d, n, r, c, k
+        self.stream_ptr = 0               # the CUDA stream the handle launches on (0 = the default stream)
         self._h = lib().sk_create(d, n, r, c, k, seed, lr, beta1, beta2, eps)
         if not self._h:
             raise SkError(f"sk_create failed: {lib().sk_last_error().decode()}")
@@ -153,6 +161,7 @@ class SketchedAMSGrad:
 
     def set_stream(self, cuda_stream_ptr: int) -> None:
         _check(lib().sk_set_stream(self._h, cuda_stream_ptr))
+        self.stream_ptr = int(cuda_stream_ptr or 0)
 
     def set_option(self, key: str, value: int) -> None:
         _check(lib().sk_set_option(self._h, key.encode(), int(value)))
@@ -175,6 +184,8 @@ class SketchedAMSGrad:
                 out = np.empty(self.P * self.k if (self.P > 1 and self._count_I()) else 0, np.uint32)
             elif field == "t":
                 out = np.empty(1, np.uint64)
+            elif field == "keys":
+                out = np.empty(self.d, np.uint32)
             else:
                 if field not in self._FIELD_SHAPES:
                     raise SkError(f"unknown field '{field}'")
@@ -188,6 +199,16 @@ class SketchedAMSGrad:
 
     def set(self, field: str, value) -> None:
         _check(lib().sk_set(self._h, field.encode(), _ptr(value) if _nbytes(value) else 0, _nbytes(value)))
+
+    def stats(self) -> dict:
+        """Statistics of the last step's selection and the exchange volume (see sk_get_stats)."""
+        out = (C.c_double * NUM_STATS)()
+        _check(lib().sk_get_stats(self._h, out, NUM_STATS))
+        return dict(zip(STAT_NAMES, [float(v) for v in out]))
+
+    def debug_check(self, kind: int) -> None:
+        """Debug build: makes the device record a bounds violation of `kind` (1..5) without any access."""
+        _check(lib().sk_debug_check(self._h, kind))
 
     def select_static(self, idx_out) -> None:
         """Re-runs the last step's top-k selection into `idx_out` (CUDA tensor of k int32/uint32) without

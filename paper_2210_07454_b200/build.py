@@ -16,6 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsketched_amsgrad.so")
+LIB_DEBUG = os.path.join(HERE, "libsketched_amsgrad_debug.so")    # device-side bounds checks compiled in
 SOURCES = ["sk_api.cu", "sk_sketch.cu", "sk_sketch_own.cu", "sk_select.cu", "sk_static.cu", "sk_shard.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
@@ -28,8 +29,10 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def _flags(verbose: bool) -> list[str]:
+def _flags(verbose: bool, debug: bool = False) -> list[str]:
     flags = list(NVCC_FLAGS) + shlex.split(os.environ.get("SK_NVCC_EXTRA", ""))
+    if debug:
+        flags += ["-DSK_DEBUG=1"]
     if verbose:
         flags += ["-Xptxas", "-v"]
     return flags
@@ -57,8 +60,10 @@ def _compile(src: str, flags: list[str], force: bool) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    flags = _flags(verbose)
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Builds (if stale) and returns the library's path; debug=True builds the bounds-checked variant beside it."""
+    flags = _flags(verbose, debug)
+    LIB = LIB_DEBUG if debug else globals()["LIB"]
     os.makedirs(OBJ, exist_ok=True)
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 1)) as pool:
         objs = list(pool.map(lambda s: _compile(s, flags, force), SOURCES))
@@ -70,4 +75,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -16,6 +16,7 @@
 namespace {
 
 thread_local std::string g_err;
+int64_t g_fail_alloc_countdown = -1;     // >= 0: the (countdown+1)-th device allocation of sk_create fails (test hook)
 
 constexpr uint32_t kDefaultWindowLines = 8;
 
@@ -108,8 +109,14 @@ int check_status(sk_state* s) {
     sk::Select h{};
     SK_CUDA(cudaMemcpyAsync(&h, s->sel, sizeof h, cudaMemcpyDeviceToHost, s->stream));
     SK_CUDA(cudaStreamSynchronize(s->stream));
-    if (h.status) return fail(SK_EDEVICE, "device status word = %u (selection emitted %u of %u indices)", h.status,
-                              h.cnt_out, s->P.k);
+    if (h.status) {
+        // reported once: the word is cleared so that the handle stays usable
+        SK_CUDA(cudaMemsetAsync(&s->sel->status, 0, sizeof(uint32_t), s->stream));
+        SK_CUDA(cudaStreamSynchronize(s->stream));
+        return fail(SK_EDEVICE, "device status word = 0x%x (bit 0: selection emitted %u of %u indices; bits 1-5, debug "
+                    "build: table offset, index, list position, histogram bin, window offset out of range)", h.status,
+                    h.cnt_out, s->P.k);
+    }
     return SK_OK;
 }
 
@@ -162,7 +169,7 @@ int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, ui
     }
     if (sharded && s->k_prev && first) {      // I_{t-1} in ascending order, from its bitmap
         StageTimer tm(s, 0);
-        tm.done(sk::launch_list_from_bitmap(s->bitmap, s->bitmap_bytes / 4, s->scan, s->I_prev, st));
+        tm.done(sk::launch_list_from_bitmap(P, s->bitmap, s->bitmap_bytes / 4, s->scan, s->I_prev, P.k, st));
     }
     for (uint32_t w0 = wbeg; w0 < wend; w0 += wc) {
         const uint32_t nw = std::min(wc, wend - w0);
@@ -184,7 +191,7 @@ int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, ui
         StageTimer tm(s, 3);
         int l = s->sum_sketch ? 0 : sk::launch_sum_tables(P, s->tables, sum_out, st);
         if (sharded && s->variant == 0)      // h_t: this process's gradient sums on I_{t-1}, zero-padded to k
-            l += sk::launch_gather(s->I_prev, s->k_prev, P.k, s->gsum, x1 + tfloats, st);
+            l += sk::launch_gather(P, s->I_prev, s->k_prev, P.k, s->gsum, x1 + tfloats, st);
         tm.done(l);
     }
     SK_CUDA(cudaGetLastError());
@@ -206,7 +213,7 @@ int phase_select(sk_state* s, const float* x1, float* x2) {
         int l = 0;
         if (sharded) {                          // the summed exchange buffer: mean sketch, then gradient sums on I_{t-1}
             SK_CUDA(cudaMemcpyAsync(s->sum, x1, (uint64_t)P.r * P.cs * 4, cudaMemcpyDeviceToDevice, st));
-            if (s->variant == 0) l += sk::launch_scatter(s->I_prev, s->k_prev, x1 + (uint64_t)P.r * P.cs, s->gsum, st);
+            if (s->variant == 0) l += sk::launch_scatter(P, s->I_prev, s->k_prev, x1 + (uint64_t)P.r * P.cs, s->gsum, st);
         }
         // ranking keys; v and vhat on I_{t-1} are brought up to date on the way, from the sums in gsum
         l += sk::launch_unsketch_hist(P, A, s->sum, s->keys, s->hist, vec, s->sm_count, st);
@@ -222,7 +229,7 @@ int phase_select(sk_state* s, const float* x1, float* x2) {
         StageTimer tm(s, 6);
         int l = sk::launch_refine(Q, s->sel, s->cand, s->cand2, s->hist2, list, s->sm_count, st);
         if (sharded) {                          // candidates in ascending order, and this process's sums of a_t there
-            l += sk::launch_sort_list(list, Q.k, s->cbitmap, s->bitmap_bytes / 4, s->scan, st);
+            l += sk::launch_sort_list(P, list, Q.k, s->cbitmap, s->bitmap_bytes / 4, s->scan, st);
             l += sk::launch_gather_worker_sum(P, list, Q.k, s->e, x2, st);
         }
         tm.done(l);
@@ -241,7 +248,7 @@ int phase_finish(sk_state* s, const float* x2, float* x) {
     if (sharded) {                              // the summed exact values, placed at their coordinates
         StageTimer tm(s, 6);
         uint32_t* list = s->cand_mult > 1 ? s->Ic : s->I;
-        tm.done(sk::launch_scatter(list, (uint32_t)s->cand_mult * P.k, x2, s->asum, st));
+        tm.done(sk::launch_scatter(P, list, (uint32_t)s->cand_mult * P.k, x2, s->asum, st));
         asum = s->asum;
     }
     if (s->cand_mult > 1) {
@@ -291,15 +298,17 @@ int shard_buffers(sk_state* s) {
     return SK_OK;
 }
 
-enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_VW, F_VHATW, F_CAND, F_X, F_BAD };
+enum Field { F_M, F_E, F_V, F_VHAT, F_TABLES, F_SUM, F_EST, F_I, F_T, F_VW, F_VHATW, F_CAND, F_X, F_KEYS, F_BAD };
 
 Field field_of(const char* name) {
-    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t", "vw", "vhatw", "cand", "x"};
-    for (int q = 0; q < 13; ++q) if (!strcmp(name, names[q])) return (Field)q;
+    static const char* names[] = {"m", "e", "v", "vhat", "tables", "sum", "est", "I", "t", "vw", "vhatw", "cand", "x", "keys"};
+    for (int q = 0; q < 14; ++q) if (!strcmp(name, names[q])) return (Field)q;
     return F_BAD;
 }
 
 }  // namespace
+
+int sk_static_prepare(void);      // sk_static.cu
 
 // lets the library's other translation units report through sk_last_error()
 int sk_fail_message(int code, const char* message) { return fail(code, "%s", message); }
@@ -345,10 +354,14 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     const uint64_t nd = (uint64_t)n * d, tf = (uint64_t)r * P.cs;
     bool ok = true;
     auto alloc = [&](void** p, uint64_t bytes) {
-        if (ok && cudaMalloc(p, bytes ? bytes : 4) != cudaSuccess) {
+        if (!ok) return;
+        cudaError_t err = cudaErrorMemoryAllocation;               // what an injected failure looks like
+        if (g_fail_alloc_countdown < 0 || g_fail_alloc_countdown-- != 0) err = cudaMalloc(p, bytes ? bytes : 4);
+        if (err != cudaSuccess) {
             ok = false;
-            fail(SK_ENOMEM, "cudaMalloc of %llu bytes failed: %s", (unsigned long long)bytes,
-                 cudaGetErrorString(cudaGetLastError()));
+            *p = nullptr;
+            cudaGetLastError();
+            fail(SK_ENOMEM, "cudaMalloc of %llu bytes failed: %s", (unsigned long long)bytes, cudaGetErrorString(err));
         }
     };
     alloc((void**)&s->m, nd * 4); alloc((void**)&s->e, nd * 4);
@@ -363,13 +376,23 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     alloc((void**)&s->keys, d_pad * 4); alloc((void**)&s->gsum, d_pad * 4);
     alloc((void**)&s->bitmap, s->bitmap_bytes);
     if (!ok) { sk_destroy(s); return nullptr; }
-    cudaMemset(s->bitmap, 0, s->bitmap_bytes);                          // I_0 is empty
-    cudaMemset(s->m, 0, nd * 4); cudaMemset(s->e, 0, nd * 4);           // m_0 = e_0 = 0
-    cudaMemset(s->vstamp, 0, d * 4);
-    cudaMemset(s->gsum, 0, d_pad * 4);
-    cudaMemset(s->tables, 0, (uint64_t)n * tf * 4); cudaMemset(s->sum, 0, tf * 4);
-    cudaMemset(s->hist, 0, sk::kHistBins * 4); cudaMemset(s->hist2, 0, sk::kHistBins * 4);
-    cudaMemset(s->sel, 0, sizeof(sk::Select));
+    P.status = &s->sel->status;
+    if (d <= SK_STATIC_MAX_D) sk_static_prepare();   // so that sk_select_static finds its scratch resolved (it may not allocate)
+    cudaError_t init = cudaSuccess;
+    auto clear = [&](void* p, uint64_t bytes) { if (init == cudaSuccess) init = cudaMemset(p, 0, bytes); };
+    clear(s->bitmap, s->bitmap_bytes);                                  // I_0 is empty
+    clear(s->m, nd * 4); clear(s->e, nd * 4);                           // m_0 = e_0 = 0
+    clear(s->vstamp, d * 4);
+    clear(s->gsum, d_pad * 4);
+    clear(s->tables, (uint64_t)n * tf * 4); clear(s->sum, tf * 4);
+    clear(s->hist, sk::kHistBins * 4); clear(s->hist2, sk::kHistBins * 4);
+    clear(s->sel, sizeof(sk::Select));
+    if (init != cudaSuccess) {
+        fail(SK_ECUDA, "initialisation failed: %s", cudaGetErrorString(init));
+        cudaGetLastError();
+        sk_destroy(s);
+        return nullptr;
+    }
     uint32_t eps_bits;
     memcpy(&eps_bits, &eps, 4);
     sk::launch_fill_u32((uint32_t*)s->v, d, eps_bits, nullptr);         // v_0 = vhat_0 = eps
@@ -469,7 +492,7 @@ int sk_step_host_sparse(const void* grads_host, uint32_t* idx_host, float* value
     int rc = host_step(s, grads_host, nullptr);
     if (rc) return rc;
     const uint64_t kb = (uint64_t)s->P.k * 4;
-    sk::launch_gather(s->I_prev, s->P.k, s->P.k, s->stage_x, s->stage_vals, s->stream);   // I_prev holds I_t now
+    sk::launch_gather(s->P, s->I_prev, s->P.k, s->P.k, s->stage_x, s->stage_vals, s->stream);   // I_prev holds I_t now
     SK_CUDA(cudaMemcpyAsync(idx_host, s->I_prev, kb, cudaMemcpyDeviceToHost, s->stream));
     SK_CUDA(cudaMemcpyAsync(values_host, s->stage_vals, kb, cudaMemcpyDeviceToHost, s->stream));
     SK_CUDA(cudaStreamSynchronize(s->stream));
@@ -536,6 +559,43 @@ int sk_set_stream(sk_state* s, void* stream) {
 int sk_sync(sk_state* s) {
     if (!s) return fail(SK_EINVAL, "null handle");
     return check_status(s);
+}
+
+int sk_test_fail_allocation(int64_t nth) {
+    g_fail_alloc_countdown = nth;
+    return SK_OK;
+}
+
+int sk_debug_check(sk_state* s, uint32_t kind) {
+    if (!s) return fail(SK_EINVAL, "null handle");
+#ifdef SK_DEBUG
+    if (kind < 1 || kind > 5) return fail(SK_EINVAL, "kind must be in 1..5");
+    sk::launch_debug_violation(s->P, 1u << kind, s->stream);
+    SK_CUDA(cudaGetLastError());
+    return SK_OK;
+#else
+    (void)kind;
+    return fail(SK_ESTATE, "this build has no device-side checks (build with -DSK_DEBUG=1)");
+#endif
+}
+
+int sk_get_stats(sk_state* s, double* out, uint32_t count) {
+    if (!s || !out) return fail(SK_EINVAL, "null argument");
+    if (count < SK_NUM_STATS) return fail(SK_EINVAL, "sk_get_stats needs room for SK_NUM_STATS values");
+    if (s->t == 0) return fail(SK_ESTATE, "no step has been taken yet");
+    sk::Select h{};
+    SK_CUDA(cudaMemcpyAsync(&h, s->sel, sizeof h, cudaMemcpyDeviceToHost, s->stream));
+    SK_CUDA(cudaStreamSynchronize(s->stream));
+    const uint32_t lead = ((h.bin << sk::kHistBits) | h.bin2) << 7;      // the threshold key's leading 24 bits
+    float tau;
+    memcpy(&tau, &lead, 4);
+    out[0] = (double)tau;
+    out[1] = (double)h.cnt_cand;
+    out[2] = (double)h.cnt_cand2;
+    out[3] = (double)h.cnt_out;
+    out[4] = (double)s->P.r * s->P.c + (double)s->cand_mult * s->P.k + (s->variant == 0 ? 2.0 : 1.0) * s->P.k;
+    out[5] = (double)h.status;
+    return SK_OK;
 }
 
 int sk_set_option(sk_state* s, const char* key, int64_t value) {

@@ -8,6 +8,9 @@ namespace sk {
 
 constexpr uint64_t kGolden = 0x9E3779B97F4A7C15ULL;
 constexpr uint32_t kUnitShift = 10;     // windowed family: units of 1024 coordinates
+constexpr uint32_t kUnit = 1u << kUnitShift;
+constexpr uint32_t kQuadsPerUnit = kUnit / 4;         // 256
+constexpr uint32_t kGroupsPerUnit = kUnit / 32;       // 32
 
 __host__ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
@@ -104,6 +107,23 @@ __device__ __forceinline__ void quad_hashes(const Params& P, uint32_t r, uint32_
             if (row < r) h[row] = quad_from_draw(P, stream(P.row_key[row], (uint64_t)(i >> P.log2g) + 1), i, wbase);
     }
 }
+
+// The units in panel-major order: panel 0's units, then panel 1's, ...  Panel p owns the units p, p + panels,
+// p + 2 panels, ...; the first `rem` panels have `tbig` of them, the others tbig - 1.
+struct UnitWalk {
+    uint32_t panels, tbig, rem;
+    uint32_t panel, tu;
+    __device__ __forceinline__ void seek(uint32_t s) {
+        const uint32_t head = rem * tbig;
+        if (s < head) { panel = s / tbig; tu = s - panel * tbig; }
+        else { const uint32_t q = s - head; panel = rem + q / (tbig - 1u); tu = q - (panel - rem) * (tbig - 1u); }
+    }
+    __device__ __forceinline__ uint32_t unit() const { return panel + panels * tu; }
+    __device__ __forceinline__ void next() {
+        const uint32_t T = panel < rem ? tbig : tbig - 1u;
+        if (++tu >= T) { tu = 0; ++panel; }
+    }
+};
 
 __device__ __forceinline__ float flip(float a, uint32_t bit) {  // a * (bit ? -1 : +1)
     return __uint_as_float(__float_as_uint(a) ^ (bit << 31));

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cstdint>
+#include "sk_debug.cuh"
 
 namespace sk {
 
@@ -22,6 +23,7 @@ struct Params {
     uint32_t k;
     float beta1, beta2, lr;
     float rho;          // alpha_{t-1}/alpha_t, the weight of e_{t-1} in the sketched vector (1 for a constant step size)
+    uint32_t* status;   // the handle's device status word (bits: sk_debug.cuh); nullptr = none
     uint32_t n_all;     // workers the means are taken over: n, or the total over all processes when the workers are
                         // partitioned (the handle then holds n of them)
 };
@@ -62,9 +64,12 @@ struct MomentArgs {
 };
 
 // Launchers.  Each enqueues on `st` and returns the number of kernels it launched.
+int sm_count_of_device();
+// debug build only: one thread runs a bounds check with a false condition of the given kind (no access is made)
+int launch_debug_violation(const Params& P, uint32_t bit, cudaStream_t st);
 int launch_zero(void* p, uint64_t bytes, cudaStream_t st);
 int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st);
-int launch_set_bits(const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st);
+int launch_set_bits(const Params& P, const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st);
 int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,
                          cudaStream_t st);
 // windowed hash family, accumulation by ownership (one warp per worker, block-owned windows): at most kOwnMaxWorkers
@@ -104,14 +109,17 @@ int launch_masked_copy(const Params& P, const float* e, const uint32_t* bitmap, 
 constexpr uint32_t kScanWordsPerBlock = 1024;      // bitmap words one block of the compaction covers
 inline uint64_t scan_entries(uint64_t bitmap_words) { return (bitmap_words + kScanWordsPerBlock - 1) / kScanWordsPerBlock + 1; }
 // out <- the set bits of the bitmap as ascending coordinates; scan: scratch of scan_entries(words) uint32
-int launch_list_from_bitmap(const uint32_t* bitmap, uint64_t words, uint32_t* scan, uint32_t* out, cudaStream_t st);
+// cap: capacity of `out`; P: for the debug build's checks
+int launch_list_from_bitmap(const Params& P, const uint32_t* bitmap, uint64_t words, uint32_t* scan, uint32_t* out,
+                            uint32_t cap, cudaStream_t st);
 // sorts a list of distinct coordinates in place through a scratch bitmap of `words` words
-int launch_sort_list(uint32_t* list, uint32_t count, uint32_t* scratch_bitmap, uint64_t words, uint32_t* scan,
+int launch_sort_list(const Params& P, uint32_t* list, uint32_t count, uint32_t* scratch_bitmap, uint64_t words, uint32_t* scan,
                      cudaStream_t st);
 // out[q] = src[list[q]] for q < count, 0 for count <= q < padded
-int launch_gather(const uint32_t* list, uint32_t count, uint32_t padded, const float* src, float* out, cudaStream_t st);
+int launch_gather(const Params& P, const uint32_t* list, uint32_t count, uint32_t padded, const float* src, float* out,
+                  cudaStream_t st);
 // dst[list[q]] = vals[q]
-int launch_scatter(const uint32_t* list, uint32_t count, const float* vals, float* dst, cudaStream_t st);
+int launch_scatter(const Params& P, const uint32_t* list, uint32_t count, const float* vals, float* dst, cudaStream_t st);
 // out[q] = sum over this handle's workers (in order) of e[w][list[q]]
 int launch_gather_worker_sum(const Params& P, const uint32_t* list, uint32_t count, const float* e, float* out,
                              cudaStream_t st);

@@ -82,7 +82,8 @@ __device__ __forceinline__ float4 medians4(const Params& P, const float* __restr
 #pragma unroll
     for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
         if (row < r) {
-            float4 cch = __ldg((const float4*)(sum + (uint64_t)row * P.cs + h[row].off));
+            float4 cch = make_float4(0.f, 0.f, 0.f, 0.f);
+            SK_GUARD(h[row].off + 4u <= P.cs, kStatusBucket) cch = __ldg((const float4*)(sum + (uint64_t)row * P.cs + h[row].off));
             cch = quad_gather(h[row], cch);
             qx[row] = cch.x; qy[row] = cch.y; qz[row] = cch.z; qw[row] = cch.w;
         }
@@ -101,9 +102,15 @@ __device__ __forceinline__ float median1(const Params& P, const float* __restric
     for (uint32_t row = 0; row < P.r; ++row) {
         uint32_t b; float s;
         coord_hash(P, P.row_key[row], j, b, s);
-        q[row] = s * __ldg(sum + (uint64_t)row * P.cs + b);
+        q[row] = 0.0f;
+        SK_GUARD(b < P.c, kStatusBucket) q[row] = s * __ldg(sum + (uint64_t)row * P.cs + b);
     }
     return median_any(q, P.r);
+}
+
+// one count in a shared-memory histogram of kHistBins bins (the bin is checked in the debug build)
+__device__ __forceinline__ void hist_add(const Params& P, uint32_t* sh, uint32_t bin) {
+    SK_GUARD(bin < kHistBins, kStatusBin) atomicAdd(&sh[bin], 1u);
 }
 
 // ---- pass A: ranking keys of all coordinates (stored) + histogram of key bits 30..19 -----------------------------
@@ -136,8 +143,8 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
                 uint4 k4;
                 k4.x = key_of(med.x); k4.y = key_of(med.y); k4.z = key_of(med.z); k4.w = key_of(med.w);
                 ((uint4*)keys)[t] = k4;
-                atomicAdd(&sh[k4.x >> kHistShift], 1u); atomicAdd(&sh[k4.y >> kHistShift], 1u);
-                atomicAdd(&sh[k4.z >> kHistShift], 1u); atomicAdd(&sh[k4.w >> kHistShift], 1u);
+                hist_add(P, sh, k4.x >> kHistShift); hist_add(P, sh, k4.y >> kHistShift);
+                hist_add(P, sh, k4.z >> kHistShift); hist_add(P, sh, k4.w >> kHistShift);
             } else if (live) {
                 float4 vh = ((const float4*)A.vhat)[t];
                 const uint32_t mask = A.members ? ((__ldg(A.bitmap + (t >> 3)) >> ((t & 7u) * 4u)) & 0xFu) : 0u;
@@ -158,13 +165,13 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
                 k4.x = key_rank(med.x, vh.x); k4.y = key_rank(med.y, vh.y);
                 k4.z = key_rank(med.z, vh.z); k4.w = key_rank(med.w, vh.w);
                 ((uint4*)keys)[t] = k4;
-                atomicAdd(&sh[k4.x >> kHistShift], 1u); atomicAdd(&sh[k4.y >> kHistShift], 1u);
-                atomicAdd(&sh[k4.z >> kHistShift], 1u); atomicAdd(&sh[k4.w >> kHistShift], 1u);
+                hist_add(P, sh, k4.x >> kHistShift); hist_add(P, sh, k4.y >> kHistShift);
+                hist_add(P, sh, k4.z >> kHistShift); hist_add(P, sh, k4.w >> kHistShift);
             }
         } else if (live && A.variant == 1) {
             const uint32_t key = key_of(median1(P, sum, t));
             keys[t] = key;
-            atomicAdd(&sh[key >> kHistShift], 1u);
+            hist_add(P, sh, key >> kHistShift);
         } else if (live) {
             float vh = A.vhat[t];
             if (A.members && ((A.bitmap[t >> 5] >> (t & 31u)) & 1u)) {
@@ -176,11 +183,131 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
             }
             const uint32_t key = key_rank(median1(P, sum, t), vh);
             keys[t] = key;
-            atomicAdd(&sh[key >> kHistShift], 1u);
+            hist_add(P, sh, key >> kHistShift);
         }
     }
     __syncthreads();
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
+        if (sh[b]) atomicAdd(&hist[b], sh[b]);
+}
+
+// ---- pass A for the windowed hash family ---------------------------------------------------------------------------
+// A unit of 1024 coordinates reads, in every row, only its panel's window of the aggregate sketch.  A block walks a
+// run of units in panel-major order (the order the sketch kernel uses), keeps the current panel's windows (r x 32L
+// floats) and the unit's r x 32 group hashes in shared memory, and every thread takes one coordinate quad per unit:
+// r 16-byte shared-memory reads, sign and xor-permutation undone in registers, median, key, histogram.  Against the
+// general kernel this drops the per-quad hash exchange by shuffles and the L2 gathers.
+template <int R>
+__global__ void __launch_bounds__(kThreads)
+k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, const float* __restrict__ sum,
+                    uint32_t* keys, uint32_t* hist, uint32_t units_total, uint32_t tbig, uint32_t rem) {
+    extern __shared__ __align__(16) uint32_t dyn[];
+    constexpr int RMAX = R > 0 ? R : (int)kMaxRows;
+    const uint32_t r = R > 0 ? (uint32_t)R : P.r;
+    const uint32_t cw = P.win_cw;
+    uint32_t* sh = dyn;                                            // [4096] histogram
+    uint2* hsh = (uint2*)(sh + kHistBins);                         // [2][r][32]: x = line*32 | perm, y = sign bits
+    float* win = (float*)(hsh + 2u * r * kGroupsPerUnit);          // [r][cw]: the panel's window of every row
+    const uint32_t tid = threadIdx.x;
+    for (uint32_t b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
+    const uint32_t s_begin = (uint32_t)((uint64_t)units_total * blockIdx.x / gridDim.x);
+    const uint32_t s_end = (uint32_t)((uint64_t)units_total * (blockIdx.x + 1) / gridDim.x);
+    const uint32_t d4 = P.d >> 2;
+    const uint32_t sg = tid >> 3, o = (tid & 7u) * 4u;             // this thread's group inside the unit, offset inside it
+    const uint32_t sgn_mul = 1u << (28u - o);
+    const uint32_t bm_words = (P.d + 31u) >> 5;
+
+    auto fill_hashes = [&](uint32_t unit, uint32_t buf) {
+        for (uint32_t hq = tid; hq < r * kGroupsPerUnit; hq += kThreads) {
+            const uint32_t row = hq >> 5, s = hq & 31u;
+            const GroupHash gh = group_from_draw(P, stream(P.row_key[row & (kMaxRows - 1u)], (uint64_t)unit * kGroupsPerUnit + s + 1));
+            hsh[buf * r * kGroupsPerUnit + hq] = make_uint2(gh.base | gh.perm, gh.signs);
+        }
+    };
+    auto load_windows = [&](uint32_t panel) {
+        for (uint32_t q = tid; q < r * (cw >> 2); q += kThreads) {
+            const uint32_t row = q / (cw >> 2), c4 = q - row * (cw >> 2);
+            ((float4*)win)[q] = __ldg((const float4*)(sum + (uint64_t)row * P.cs + (uint64_t)panel * cw) + c4);
+        }
+    };
+
+    UnitWalk walk{P.win_panels, tbig, rem, 0u, 0u};
+    if (s_begin < s_end) {
+        walk.seek(s_begin);
+        fill_hashes(walk.unit(), 0u);
+        load_windows(walk.panel);
+    }
+    __syncthreads();
+    for (uint32_t s = s_begin; s < s_end; ++s) {
+        const uint32_t buf = (s - s_begin) & 1u;
+        const uint32_t unit = walk.unit(), panel = walk.panel;
+        const bool have_next = s + 1 < s_end;
+        walk.next();
+        if (have_next) fill_hashes(walk.unit(), buf ^ 1u);
+        const uint2* hs = hsh + buf * r * kGroupsPerUnit + sg;
+        const uint32_t t = unit * kQuadsPerUnit + tid;
+        if (t < d4) {
+            float qx[RMAX], qy[RMAX], qz[RMAX], qw[RMAX];
+#pragma unroll
+            for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
+                if (row < r) {
+                    const uint2 h = hs[row * kGroupsPerUnit];
+                    const uint32_t woff = (h.x ^ o) & ~3u;
+                    float4 cch = make_float4(0.f, 0.f, 0.f, 0.f);
+                    SK_GUARD(woff + 4u <= cw, kStatusWindow) cch = *(const float4*)(win + row * cw + woff);
+                    // coordinate l of the quad sits at element l xor p3 of the chunk, with sign bit o + l of h.y
+                    if (h.x & 1u) { float u = cch.x; cch.x = cch.y; cch.y = u; u = cch.z; cch.z = cch.w; cch.w = u; }
+                    if (h.x & 2u) { float u = cch.x; cch.x = cch.z; cch.z = u; u = cch.y; cch.y = cch.w; cch.w = u; }
+                    const uint32_t t3 = h.y * sgn_mul, t2 = t3 * 2u, t1 = t3 * 4u, t0 = t3 * 8u;
+                    qx[row] = __uint_as_float(__float_as_uint(cch.x) ^ (t0 & 0x80000000u));
+                    qy[row] = __uint_as_float(__float_as_uint(cch.y) ^ (t1 & 0x80000000u));
+                    qz[row] = __uint_as_float(__float_as_uint(cch.z) ^ (t2 & 0x80000000u));
+                    qw[row] = __uint_as_float(__float_as_uint(cch.w) ^ (t3 & 0x80000000u));
+                }
+            float4 med;
+            if constexpr (R > 0) {
+                med.x = median_fixed(qx); med.y = median_fixed(qy); med.z = median_fixed(qz); med.w = median_fixed(qw);
+            } else {
+                med.x = median_any(qx, r); med.y = median_any(qy, r); med.z = median_any(qz, r); med.w = median_any(qw, r);
+            }
+            uint4 k4;
+            if (A.variant == 1) {                                  // parameter averaging: U(S) takes no vhat (Algorithm 1)
+                k4.x = key_of(med.x); k4.y = key_of(med.y); k4.z = key_of(med.z); k4.w = key_of(med.w);
+            } else {
+                float4 vh = ((const float4*)A.vhat)[t];
+                uint32_t mask = 0;
+                if (A.members) {
+                    const uint32_t word = unit * kGroupsPerUnit + sg;
+                    if (word < bm_words) mask = (__ldg(A.bitmap + word) >> o) & 0xFu;
+                }
+                if (mask) {
+                    const float4 gs = ((const float4*)A.gsum)[t];
+                    float4 vv = ((const float4*)A.v)[t];
+                    uint4 vs = ((const uint4*)A.vstamp)[t];
+                    if (mask & 1u) update_member(P, A, gs.x, vv.x, vs.x, vh.x);
+                    if (mask & 2u) update_member(P, A, gs.y, vv.y, vs.y, vh.y);
+                    if (mask & 4u) update_member(P, A, gs.z, vv.z, vs.z, vh.z);
+                    if (mask & 8u) update_member(P, A, gs.w, vv.w, vs.w, vh.w);
+                    ((float4*)A.v)[t] = vv;
+                    ((uint4*)A.vstamp)[t] = vs;
+                    ((float4*)A.vhat)[t] = vh;
+                    ((float4*)A.gsum)[t] = make_float4(0.f, 0.f, 0.f, 0.f);   // consumed: the sums start from zero next step
+                }
+                k4.x = key_rank(med.x, vh.x); k4.y = key_rank(med.y, vh.y);
+                k4.z = key_rank(med.z, vh.z); k4.w = key_rank(med.w, vh.w);
+            }
+            ((uint4*)keys)[t] = k4;
+            hist_add(P, sh, k4.x >> kHistShift); hist_add(P, sh, k4.y >> kHistShift);
+            hist_add(P, sh, k4.z >> kHistShift); hist_add(P, sh, k4.w >> kHistShift);
+        }
+        __syncthreads();            // everyone is done with this unit's hashes (and with the windows, if the panel ends)
+        if (have_next && walk.panel != panel) {
+            load_windows(walk.panel);
+            __syncthreads();
+        }
+    }
+    __syncthreads();
+    for (uint32_t b = tid; b < kHistBins; b += kThreads)
         if (sh[b]) atomicAdd(&hist[b], sh[b]);
 }
 
@@ -258,29 +385,33 @@ __device__ __forceinline__ void block_append(uint32_t n_a, uint32_t n_b, uint32_
 constexpr uint32_t kWarpBuf = 128;
 
 template <typename T>
-__device__ __forceinline__ void warp_flush(T* buf, uint32_t& fill, uint32_t* counter, T* list) {
+__device__ __forceinline__ void warp_flush(const Params& P, T* buf, uint32_t& fill, uint32_t* counter, T* list, uint32_t cap) {
     __syncwarp();
     const uint32_t lane = threadIdx.x & 31u;
     uint32_t base = 0;
     if (lane == 0 && fill) base = atomicAdd(counter, fill);
     base = __shfl_sync(0xFFFFFFFFu, base, 0);
-    for (uint32_t q = lane; q < fill; q += 32) list[base + q] = buf[q];
+    for (uint32_t q = lane; q < fill; q += 32)
+        SK_GUARD(base + q < cap, kStatusListPos) list[base + q] = buf[q];
     __syncwarp();
     fill = 0;
 }
 
 // where this lane's `mine` entries of the warp's `total` go: into the staging buffer (flushed first if they do not
 // fit), or straight into the list when one tile yields more than a buffer holds
+// (a tile that yields more than a buffer holds goes straight into the list: the debug build checks the reserved
+// range against the capacity and diverts an overflowing warp into its staging buffer, whose flush is checked too)
 template <typename T>
-__device__ __forceinline__ T* warp_reserve(T* buf, uint32_t& fill, uint32_t* counter, T* list, uint32_t total,
-                                           uint32_t excl) {
+__device__ __forceinline__ T* warp_reserve(const Params& P, T* buf, uint32_t& fill, uint32_t* counter, T* list, uint32_t cap,
+                                           uint32_t total, uint32_t excl) {
     if (total == 0) return buf;
-    if (fill + total > kWarpBuf) warp_flush(buf, fill, counter, list);
+    if (fill + total > kWarpBuf) warp_flush(P, buf, fill, counter, list, cap);
     if (total > kWarpBuf) {
         uint32_t base = 0;
         if ((threadIdx.x & 31u) == 0) base = atomicAdd(counter, total);
         base = __shfl_sync(0xFFFFFFFFu, base, 0);
-        return list + base + excl;
+        if (in_bounds(base + total <= cap, P.status, kStatusListPos)) return list + base + excl;
+        return buf;          // debug build only: the entries of this tile are dropped (two lanes may share a slot)
     }
     T* dst = buf + fill + excl;
     fill += total;
@@ -289,8 +420,10 @@ __device__ __forceinline__ T* warp_reserve(T* buf, uint32_t& fill, uint32_t* cou
 
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
-k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx_map, Select* sel, uint32_t* I_out,
-       Cand* cand, uint32_t* hist2) {
+k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx_map, Select* sel,
+       uint32_t* I_out, Cand* cand, uint32_t* hist2) {
+    // P.d keys, the P.k largest wanted: I_out holds P.k entries, the candidate list P.d
+    const uint32_t d = P.d;
     // idx_map (scalar form only): keys[t] belongs to coordinate idx_map[t] instead of t (second round on a candidate list)
     __shared__ uint32_t sh2[kHistBins];
     __shared__ uint32_t wb_out[kThreads / 32][kWarpBuf];
@@ -347,8 +480,8 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
         const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
         if (total == 0) continue;
         const uint32_t excl = incl - packed;
-        uint32_t* po = warp_reserve(wb_out[wid], fill_out, &sel->cnt_out, I_out, total & 0xFFFFu, excl & 0xFFFFu);
-        Cand* pc = warp_reserve(wb_cand[wid], fill_cand, &sel->cnt_cand, cand, total >> 16, excl >> 16);
+        uint32_t* po = warp_reserve(P, wb_out[wid], fill_out, &sel->cnt_out, I_out, P.k, total & 0xFFFFu, excl & 0xFFFFu);
+        Cand* pc = warp_reserve(P, wb_cand[wid], fill_cand, &sel->cnt_cand, cand, P.d, total >> 16, excl >> 16);
         if (packed == 0) continue;                              // this lane has nothing to append
 #pragma unroll
         for (uint32_t u = 0; u < U; ++u) {
@@ -361,14 +494,14 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
                     const uint32_t key = kq[u][q];
                     if (key >= thr_hi) *po++ = idx0 + q;
                     else if (key >= thr_lo) {
-                        atomicAdd(&sh2[(key >> 7) & (kHistBins - 1u)], 1u);
+                        hist_add(P, sh2, (key >> 7) & (kHistBins - 1u));
                         pc->key = key; pc->idx = idx0 + q; ++pc;
                     }
                 }
         }
     }
-    warp_flush(wb_out[wid], fill_out, &sel->cnt_out, I_out);
-    warp_flush(wb_cand[wid], fill_cand, &sel->cnt_cand, cand);
+    warp_flush(P, wb_out[wid], fill_out, &sel->cnt_out, I_out, P.k);
+    warp_flush(P, wb_cand[wid], fill_cand, &sel->cnt_cand, cand, P.d);
     __syncthreads();
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
         if (sh2[b]) atomicAdd(&hist2[b], sh2[b]);
@@ -376,7 +509,7 @@ k_emit(uint32_t d, const uint32_t* __restrict__ keys, const uint32_t* __restrict
 
 // ---- pass C over the candidates: first 24 key bits above the threshold -> emit, equal -> second list ----------
 __global__ void __launch_bounds__(kThreads)
-k_split_candidates(Select* sel, const Cand* __restrict__ cand, uint32_t* I_out, Cand* cand2) {
+k_split_candidates(const __grid_constant__ Params P, Select* sel, const Cand* __restrict__ cand, uint32_t* I_out, Cand* cand2) {
     const uint32_t ncand = sel->cnt_cand;
     const uint32_t thr = (sel->bin << kHistBits) | sel->bin2;          // leading 24 bits of the threshold key
     const uint32_t trips = (ncand + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
@@ -392,16 +525,17 @@ k_split_candidates(Select* sel, const Cand* __restrict__ cand, uint32_t* I_out, 
         }
         uint32_t po, pc;
         block_append(n_out, n_eq, &sel->cnt_out, &sel->cnt_cand2, po, pc);
-        if (n_out) I_out[po] = cnd.idx;
-        if (n_eq) cand2[pc] = cnd;
+        if (n_out) SK_GUARD(po < P.k, kStatusListPos) I_out[po] = cnd.idx;
+        if (n_eq) SK_GUARD(pc < P.d, kStatusListPos) cand2[pc] = cnd;
     }
 }
 
 // ---- pass D: of the second list take the `need2` largest by (last 7 key bits, then smaller index) -------------
 // Radix select by one block on the 39-bit composite (key & 127, ~idx): all composites are distinct, so the
 // selection is exact and equal keys go to the smaller index.
-__global__ void __launch_bounds__(1024) k_resolve(uint32_t k, Select* sel, const Cand* __restrict__ cand2,
-                                                  uint32_t* I_out) {
+__global__ void __launch_bounds__(1024) k_resolve(const __grid_constant__ Params P, Select* sel,
+                                                  const Cand* __restrict__ cand2, uint32_t* I_out) {
+    const uint32_t k = P.k;
     constexpr uint32_t W = 11, BINS = 1u << W;
     __shared__ uint32_t hist[BINS];
     __shared__ uint32_t s_bin, s_need, s_done, s_pos;
@@ -459,7 +593,7 @@ __global__ void __launch_bounds__(1024) k_resolve(uint32_t k, Select* sel, const
             const uint64_t comp = ((uint64_t)(cnd.key & 127u) << 32) | (uint32_t)~cnd.idx;
             if (comp >= threshold) {
                 const uint32_t pos = atomicAdd(&s_pos, 1u);
-                if (pos < k) I_out[pos] = cnd.idx;
+                if (pos < k) I_out[pos] = cnd.idx;      // a surplus is not written; the count below reports it
             }
         }
     }
@@ -483,12 +617,13 @@ k_exact_keys(const __grid_constant__ Params P, const uint32_t* __restrict__ C, u
     for (uint32_t q = blockIdx.x * kThreads + threadIdx.x; q < count; q += gridDim.x * kThreads) {
         const uint32_t j = C[q];
         float abar = 0.0f;
+        if (!in_bounds(j < P.d, P.status, kStatusIndex)) continue;
         if (asum) abar = asum[j];
         else for (uint32_t w = 0; w < P.n; ++w) abar += e[(uint64_t)w * P.d + j];
         abar = abar / (float)P.n_all;
         const uint32_t key = key_of(vhat ? scale_est(abar, vhat[j]) : abar);
         keys2[q] = key;
-        atomicAdd(&sh[key >> kHistShift], 1u);
+        hist_add(P, sh, key >> kHistShift);
     }
     __syncthreads();
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads)
@@ -504,6 +639,7 @@ k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const 
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
     if (q >= P.k) return;
     const uint32_t j = I[q];
+    if (!in_bounds(j < P.d, P.status, kStatusIndex)) return;
     float abar = 0.0f;
     uint32_t w = asum ? P.n : 0;
     if (asum) abar = asum[j];
@@ -583,6 +719,33 @@ int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum,
         kfn<<<grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P, A, sum, keys, hist);
         return 1;
     }
+    if (P.win_cw != 0 && P.log2g == 5) {           // windowed family: shared-memory windows, panel-major walk
+        const uint32_t units_total = (P.d + kUnit - 1) / kUnit;
+        const uint32_t tbig = (units_total + P.win_panels - 1) / P.win_panels;
+        const uint32_t rem = units_total - (tbig - 1u) * P.win_panels;
+        const size_t smem = (size_t)kHistBins * 4 + (size_t)2 * P.r * kGroupsPerUnit * 8 + (size_t)P.r * P.win_cw * 4;
+#define SK_WIN_CASE(RR)                                                                                              \
+        {                                                                                                            \
+            auto kfn = k_unsketch_hist_win<RR>;                                                                      \
+            int nb = 0;                                                                                              \
+            if ((smem <= 48 * 1024 ||                                                                                \
+                 cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) && \
+                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kfn, kThreads, smem) == cudaSuccess && nb >= 1) { \
+                const uint64_t cap = (uint64_t)sm_count * nb;                                                        \
+                kfn<<<(int)(units_total < cap ? units_total : cap), kThreads, smem, st>>>(P, A, sum, keys, hist,     \
+                                                                                          units_total, tbig, rem);   \
+                return 1;                                                                                            \
+            }                                                                                                        \
+            cudaGetLastError();                                                                                      \
+        } break;
+        switch (P.r) {
+            case 5: SK_WIN_CASE(5)
+            case 7: SK_WIN_CASE(7)
+            case 10: SK_WIN_CASE(10)
+            default: SK_WIN_CASE(0)
+        }
+#undef SK_WIN_CASE
+    }
     const uint64_t items = P.d >> 2;
     SK_ROWS_SWITCH(k_unsketch_hist, P, A, sum, keys, hist)
     return 1;
@@ -597,11 +760,11 @@ int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, 
                 uint32_t* hist2, int sm_count, cudaStream_t st) {
     if (P.d % 4 == 0 && !idx_map) {
         auto kfn = k_emit<true>;
-        kfn<<<grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P.d, keys, nullptr, sel, I_out,
+        kfn<<<grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P, keys, nullptr, sel, I_out,
                                                                                                    cand, hist2);
     } else {
         auto kfn = k_emit<false>;
-        kfn<<<grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P.d, keys, idx_map, sel, I_out, cand, hist2);
+        kfn<<<grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P, keys, idx_map, sel, I_out, cand, hist2);
     }
     return 1;
 }
@@ -616,8 +779,8 @@ int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const 
 int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
                   int sm_count, cudaStream_t st) {
     k_pick_bin<<<1, 1024, 0, st>>>(P.k, hist2, sel, 1);
-    k_split_candidates<<<sm_count, kThreads, 0, st>>>(sel, cand, I_out, cand2);
-    k_resolve<<<1, 1024, 0, st>>>(P.k, sel, cand2, I_out);
+    k_split_candidates<<<sm_count, kThreads, 0, st>>>(P, sel, cand, I_out, cand2);
+    k_resolve<<<1, 1024, 0, st>>>(P, sel, cand2, I_out);
     return 3;
 }
 
@@ -628,13 +791,13 @@ int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const fl
 }
 
 int launch_estimates(const Params& P, const float* sum, const float* vhat, float* est, cudaStream_t st) {
-    k_estimates<<<grid_for(P.d, 148, 8), kThreads, 0, st>>>(P, sum, vhat, est);
+    k_estimates<<<grid_for(P.d, sm_count_of_device(), 8), kThreads, 0, st>>>(P, sum, vhat, est);
     return 1;
 }
 
 int launch_hash_export(const Params& P, uint32_t row, uint64_t i0, uint64_t count, uint32_t* idx, int8_t* sgn,
                        cudaStream_t st) {
-    k_hash_export<<<grid_for(count, 148, 8), kThreads, 0, st>>>(P, row, i0, count, idx, sgn);
+    k_hash_export<<<grid_for(count, sm_count_of_device(), 8), kThreads, 0, st>>>(P, row, i0, count, idx, sgn);
     return 1;
 }
 

@@ -71,7 +71,8 @@ k_scan_counts(uint32_t* counts, uint32_t n) {
 
 // the set bits of the block's words, written as ascending coordinates from offsets[block]
 __global__ void __launch_bounds__(kThreads)
-k_bits_emit(const uint32_t* __restrict__ bitmap, uint64_t words, const uint32_t* __restrict__ offsets, uint32_t* out) {
+k_bits_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ bitmap, uint64_t words,
+            const uint32_t* __restrict__ offsets, uint32_t* out, uint32_t cap) {
     const uint64_t w0 = (uint64_t)blockIdx.x * kScanWordsPerBlock + (uint64_t)threadIdx.x * kWordsPerThread;
     uint32_t w[kWordsPerThread];
     uint32_t c = 0;
@@ -87,28 +88,34 @@ k_bits_emit(const uint32_t* __restrict__ bitmap, uint64_t words, const uint32_t*
         uint32_t bits = w[q];
         const uint32_t first = (uint32_t)((w0 + q) << 5);
         while (bits) {
-            out[pos++] = first + (uint32_t)(__ffs((int)bits) - 1);
+            SK_GUARD(pos < cap, kStatusListPos) out[pos] = first + (uint32_t)(__ffs((int)bits) - 1);
+            ++pos;
             bits &= bits - 1u;
         }
     }
 }
 
 __global__ void __launch_bounds__(kThreads)
-k_list_set_bits(const uint32_t* __restrict__ list, uint32_t count, uint32_t* bitmap) {
+k_list_set_bits(const __grid_constant__ Params P, const uint32_t* __restrict__ list, uint32_t count, uint32_t* bitmap) {
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
-    if (q < count) atomicOr(&bitmap[list[q] >> 5], 1u << (list[q] & 31u));
+    if (q < count) SK_GUARD(list[q] < P.d, kStatusIndex) atomicOr(&bitmap[list[q] >> 5], 1u << (list[q] & 31u));
 }
 
 __global__ void __launch_bounds__(kThreads)
-k_gather(const uint32_t* __restrict__ list, uint32_t count, uint32_t padded, const float* __restrict__ src, float* out) {
+k_gather(const __grid_constant__ Params P, const uint32_t* __restrict__ list, uint32_t count, uint32_t padded,
+         const float* __restrict__ src, float* out) {
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
-    if (q < padded) out[q] = q < count ? src[list[q]] : 0.0f;
+    if (q >= padded) return;
+    float val = 0.0f;
+    if (q < count) SK_GUARD(list[q] < P.d, kStatusIndex) val = src[list[q]];
+    out[q] = val;
 }
 
 __global__ void __launch_bounds__(kThreads)
-k_scatter(const uint32_t* __restrict__ list, uint32_t count, const float* __restrict__ vals, float* dst) {
+k_scatter(const __grid_constant__ Params P, const uint32_t* __restrict__ list, uint32_t count, const float* __restrict__ vals,
+          float* dst) {
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
-    if (q < count) dst[list[q]] = vals[q];
+    if (q < count) SK_GUARD(list[q] < P.d, kStatusIndex) dst[list[q]] = vals[q];
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -118,7 +125,8 @@ k_gather_worker_sum(const __grid_constant__ Params P, const uint32_t* __restrict
     if (q >= count) return;
     const uint32_t j = list[q];
     float acc = 0.0f;
-    for (uint32_t w = 0; w < P.n; ++w) acc += e[(uint64_t)w * P.d + j];
+    SK_GUARD(j < P.d, kStatusIndex)
+        for (uint32_t w = 0; w < P.n; ++w) acc += e[(uint64_t)w * P.d + j];
     out[q] = acc;
 }
 
@@ -126,32 +134,34 @@ inline uint32_t blocks_for(uint64_t items) { return (uint32_t)((items + kThreads
 
 }  // namespace
 
-int launch_list_from_bitmap(const uint32_t* bitmap, uint64_t words, uint32_t* scan, uint32_t* out, cudaStream_t st) {
+int launch_list_from_bitmap(const Params& P, const uint32_t* bitmap, uint64_t words, uint32_t* scan, uint32_t* out,
+                            uint32_t cap, cudaStream_t st) {
     const uint32_t nblocks = (uint32_t)((words + kScanWordsPerBlock - 1) / kScanWordsPerBlock);
     if (nblocks == 0) return 0;
     k_bits_count<<<nblocks, kThreads, 0, st>>>(bitmap, words, scan);
     k_scan_counts<<<1, kThreads, 0, st>>>(scan, nblocks);
-    k_bits_emit<<<nblocks, kThreads, 0, st>>>(bitmap, words, scan, out);
+    k_bits_emit<<<nblocks, kThreads, 0, st>>>(P, bitmap, words, scan, out, cap);
     return 3;
 }
 
-int launch_sort_list(uint32_t* list, uint32_t count, uint32_t* scratch_bitmap, uint64_t words, uint32_t* scan,
+int launch_sort_list(const Params& P, uint32_t* list, uint32_t count, uint32_t* scratch_bitmap, uint64_t words, uint32_t* scan,
                      cudaStream_t st) {
     if (count == 0) return 0;
     int l = launch_zero(scratch_bitmap, words * 4, st);        // words * 4 is a multiple of 16 (the bitmap's padding)
-    k_list_set_bits<<<blocks_for(count), kThreads, 0, st>>>(list, count, scratch_bitmap);
-    return l + 1 + launch_list_from_bitmap(scratch_bitmap, words, scan, list, st);
+    k_list_set_bits<<<blocks_for(count), kThreads, 0, st>>>(P, list, count, scratch_bitmap);
+    return l + 1 + launch_list_from_bitmap(P, scratch_bitmap, words, scan, list, count, st);
 }
 
-int launch_gather(const uint32_t* list, uint32_t count, uint32_t padded, const float* src, float* out, cudaStream_t st) {
+int launch_gather(const Params& P, const uint32_t* list, uint32_t count, uint32_t padded, const float* src, float* out,
+                  cudaStream_t st) {
     if (padded == 0) return 0;
-    k_gather<<<blocks_for(padded), kThreads, 0, st>>>(list, count, padded, src, out);
+    k_gather<<<blocks_for(padded), kThreads, 0, st>>>(P, list, count, padded, src, out);
     return 1;
 }
 
-int launch_scatter(const uint32_t* list, uint32_t count, const float* vals, float* dst, cudaStream_t st) {
+int launch_scatter(const Params& P, const uint32_t* list, uint32_t count, const float* vals, float* dst, cudaStream_t st) {
     if (count == 0) return 0;
-    k_scatter<<<blocks_for(count), kThreads, 0, st>>>(list, count, vals, dst);
+    k_scatter<<<blocks_for(count), kThreads, 0, st>>>(P, list, count, vals, dst);
     return 1;
 }
 

@@ -17,6 +17,11 @@ __device__ __forceinline__ void red_add_v4(float* addr, float4 v) {
                  :: "l"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w));
 }
 
+// the reduction of one signed quad into row `row` of a table, at the chunk the hash gives (checked in the debug build)
+__device__ __forceinline__ void sketch_quad(const Params& P, float* table, uint32_t row, const Quad h, float4 a) {
+    SK_GUARD(h.off + 4u <= P.cs, kStatusBucket) red_add_v4(table + (uint64_t)row * P.cs + h.off, quad_scatter(h, a));
+}
+
 __global__ void __launch_bounds__(kThreads) k_zero(float4* p, uint64_t n4) {
     const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
     for (uint64_t t = blockIdx.x * (uint64_t)kThreads + threadIdx.x; t < n4; t += (uint64_t)gridDim.x * kThreads)
@@ -28,9 +33,10 @@ __global__ void __launch_bounds__(kThreads) k_fill_u32(uint32_t* p, uint64_t n, 
         p[t] = value;
 }
 
-__global__ void __launch_bounds__(kThreads) k_set_bits(const uint32_t* __restrict__ I, uint32_t count, uint32_t* bitmap) {
+__global__ void __launch_bounds__(kThreads)
+k_set_bits(const __grid_constant__ Params P, const uint32_t* __restrict__ I, uint32_t count, uint32_t* bitmap) {
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
-    if (q < count) atomicOr(&bitmap[I[q] >> 5], 1u << (I[q] & 31u));
+    if (q < count) SK_GUARD(I[q] < P.d, kStatusIndex) atomicOr(&bitmap[I[q] >> 5], 1u << (I[q] & 31u));
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -74,7 +80,7 @@ __device__ __forceinline__ void sketch_of_sum(const Params& P, const MomentArgs&
     as.x = as.x / fn; as.y = as.y / fn; as.z = as.z / fn; as.w = as.w / fn;
 #pragma unroll
     for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
-        if (row < r) red_add_v4(A.sum_table + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], as));
+        if (row < r) sketch_quad(P, A.sum_table, row, h[row], as);
 }
 
 // m = beta1 m + (1-beta1) g ; a = m + rho e (kept in the e buffer; e counts as 0 on I_{t-1}; rho = alpha_{t-1}/alpha_t,
@@ -125,8 +131,8 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
 #pragma unroll
                 for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
                     if (row < r) {
-                        red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
-                        red_add_v4(t1 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a1));
+                        sketch_quad(P, t0, row, h[row], a0);
+                        sketch_quad(P, t1, row, h[row], a1);
                     }
             }
         }
@@ -144,7 +150,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             if (!A.sum_table) {
 #pragma unroll
                 for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
-                    if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+                    if (row < r) sketch_quad(P, t0, row, h[row], a0);
             }
         }
         if (mask) ((float4*)A.gsum)[t] = gs;             // consumed by the key pass (or by the next launch)
@@ -198,7 +204,7 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
             if (!A.sum_table) {
 #pragma unroll
                 for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
-                    if (row < r) red_add_v4(t0 + (uint64_t)row * P.cs + h[row].off, quad_scatter(h[row], a0));
+                    if (row < r) sketch_quad(P, t0, row, h[row], a0);
             }
             as.x += a0.x; as.y += a0.y; as.z += a0.z; as.w += a0.w;
         }
@@ -236,7 +242,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
             for (uint32_t row = 0; row < P.r && !A.sum_table; ++row) {
                 uint32_t b; float s;
                 coord_hash(P, P.row_key[row], j, b, s);
-                atomicAdd(A.tables + (uint64_t)w * tstride + (uint64_t)row * P.cs + b, s * a);
+                SK_GUARD(b < P.c, kStatusBucket) atomicAdd(A.tables + (uint64_t)w * tstride + (uint64_t)row * P.cs + b, s * a);
             }
         }
         if (member && A.variant == 0) A.gsum[j] = gs;
@@ -246,7 +252,7 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
             for (uint32_t row = 0; row < P.r; ++row) {
                 uint32_t b; float s;
                 coord_hash(P, P.row_key[row], j, b, s);
-                atomicAdd(A.sum_table + (uint64_t)row * P.cs + b, s * share);
+                SK_GUARD(b < P.c, kStatusBucket) atomicAdd(A.sum_table + (uint64_t)row * P.cs + b, s * share);
             }
         }
     }
@@ -277,32 +283,63 @@ inline int grid_for(uint64_t items, int sm_count, int per_sm) {
 
 }  // namespace
 
+// multiprocessors of the current device (queried once per device), for the grids of the helper kernels
+int sm_count_of_device() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+#ifdef SK_DEBUG
+namespace {
+__global__ void k_debug_violation(const __grid_constant__ Params P, uint32_t bit) {
+    SK_GUARD(false, bit) { }
+}
+}  // namespace
+#endif
+
+int launch_debug_violation(const Params& P, uint32_t bit, cudaStream_t st) {
+#ifdef SK_DEBUG
+    k_debug_violation<<<1, 1, 0, st>>>(P, bit);
+    return 1;
+#else
+    (void)P; (void)bit; (void)st;
+    return 0;
+#endif
+}
+
 int launch_zero(void* p, uint64_t bytes, cudaStream_t st) {   // bytes must be a multiple of 16
-    k_zero<<<grid_for(bytes / 16, 148, 8), kThreads, 0, st>>>((float4*)p, bytes / 16);
+    k_zero<<<grid_for(bytes / 16, sm_count_of_device(), 8), kThreads, 0, st>>>((float4*)p, bytes / 16);
     return 1;
 }
 
 int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st) {
-    k_fill_u32<<<grid_for(n, 148, 8), kThreads, 0, st>>>(p, n, value);
+    k_fill_u32<<<grid_for(n, sm_count_of_device(), 8), kThreads, 0, st>>>(p, n, value);
     return 1;
 }
 
-int launch_set_bits(const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st) {
+int launch_set_bits(const Params& P, const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st) {
     if (count == 0) return 0;
-    k_set_bits<<<(count + kThreads - 1) / kThreads, kThreads, 0, st>>>(I, count, bitmap);
+    k_set_bits<<<(count + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, I, count, bitmap);
     return 1;
 }
 
 int launch_v_materialize(const Params& P, const float* v, const uint32_t* vstamp, uint32_t t, float* out,
                          cudaStream_t st) {
-    k_v_materialize<<<grid_for(P.d, 148, 8), kThreads, 0, st>>>(P, v, vstamp, t, out);
+    k_v_materialize<<<grid_for(P.d, sm_count_of_device(), 8), kThreads, 0, st>>>(P, v, vstamp, t, out);
     return 1;
 }
 
 int launch_masked_copy(const Params& P, const float* e, const uint32_t* bitmap, uint32_t workers, float* out,
                        cudaStream_t st) {
     const uint64_t total = (uint64_t)workers * P.d;
-    k_masked_copy<<<grid_for(total, 148, 16), kThreads, 0, st>>>(e, bitmap, P.d, total, out);
+    k_masked_copy<<<grid_for(total, sm_count_of_device(), 16), kThreads, 0, st>>>(e, bitmap, P.d, total, out);
     return 1;
 }
 
@@ -332,7 +369,7 @@ int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint
 }
 
 int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStream_t st) {
-    k_sum_tables<<<grid_for((P.r * P.cs) >> 2, 148, 8), kThreads, 0, st>>>(P, (const float4*)tables, (float4*)sum);
+    k_sum_tables<<<grid_for((P.r * P.cs) >> 2, sm_count_of_device(), 8), kThreads, 0, st>>>(P, (const float4*)tables, (float4*)sum);
     return 1;
 }
 

@@ -27,10 +27,7 @@ namespace sk {
 
 namespace {
 
-constexpr uint32_t kUnit = 1u << kUnitShift;          // 1024 coordinates
-constexpr uint32_t kQuadsPerUnit = kUnit / 4;         // 256
 constexpr uint32_t kChunksPerUnit = kUnit / 128;      // 8 warp-wide chunks of 128 coordinates
-constexpr uint32_t kGroupsPerUnit = kUnit / 32;       // 32
 
 __device__ __forceinline__ void red_add_v4(float* addr, float4 v) {
     asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
@@ -43,23 +40,6 @@ __device__ __forceinline__ void red_add_v4(float* addr, float4 v) {
     aa.x = fmaf(rho, (mask & 1u) ? 0.0f : aa.x, mm.x); aa.y = fmaf(rho, (mask & 2u) ? 0.0f : aa.y, mm.y); \
     aa.z = fmaf(rho, (mask & 4u) ? 0.0f : aa.z, mm.z); aa.w = fmaf(rho, (mask & 8u) ? 0.0f : aa.w, mm.w);
 
-// The units in panel-major order: panel 0's units, then panel 1's, ...  Panel p owns the units p, p + panels,
-// p + 2 panels, ...; the first `rem` panels have `tbig` of them, the others tbig - 1.
-struct UnitWalk {
-    uint32_t panels, tbig, rem;
-    uint32_t panel, tu;
-    __device__ __forceinline__ void seek(uint32_t s) {
-        const uint32_t head = rem * tbig;
-        if (s < head) { panel = s / tbig; tu = s - panel * tbig; }
-        else { const uint32_t q = s - head; panel = rem + q / (tbig - 1u); tu = q - (panel - rem) * (tbig - 1u); }
-    }
-    __device__ __forceinline__ uint32_t unit() const { return panel + panels * tu; }
-    __device__ __forceinline__ void next() {
-        const uint32_t T = panel < rem ? tbig : tbig - 1u;
-        if (++tu >= T) { tu = 0; ++panel; }
-    }
-};
-
 struct Chunk { float4 g, m, e; };
 
 // One read-add-write of this lane's four signed values into its worker's window of a row.
@@ -67,8 +47,9 @@ struct Chunk { float4 g, m, e; };
 // offset of the lane's first coordinate inside the group, sgn_mul = 2^(28 - o).
 // Shifts are written as multiplications so that they issue on the multiply-add pipe; the logic pipe, which this
 // kernel loads most, is left with one operation per sign and per select.
-__device__ __forceinline__ void window_add(float* wrow, const uint2 h, uint32_t o, uint32_t sgn_mul, float4 a) {
+__device__ __forceinline__ void window_add(const Params& P, float* wrow, const uint2 h, uint32_t o, uint32_t sgn_mul, float4 a) {
     const uint32_t off = (h.x ^ o) & ~3u;                          // line of the group, chunk after the xor permutation
+    if (!in_bounds(off + 4u <= P.win_cw, P.status, kStatusWindow)) return;
     const uint32_t t3 = h.y * sgn_mul;                             // sign bit of local coordinate 3 in bit 31
     const uint32_t t2 = t3 * 2u, t1 = t3 * 4u, t0 = t3 * 8u;       // ... of 2, 1, 0 in bit 31
     a.x = __uint_as_float(__float_as_uint(a.x) ^ (t0 & 0x80000000u));
@@ -172,14 +153,14 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
                     if (i < r) {
                         uint32_t row = i + grp;
                         if (row >= r) row -= r;
-                        window_add(mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, sgn_mul, aa);
+                        window_add(P, mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, sgn_mul, aa);
                         __syncwarp();                              // the next sub-step's lanes may read what these wrote
                     }
                 }
             } else {
                 for (uint32_t row = 0; row < r; ++row)
                     for (uint32_t q = 0; q < 4; ++q) {             // fewer rows than groups: the groups take turns
-                        if (grp == q) window_add(mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, sgn_mul, aa);
+                        if (grp == q) window_add(P, mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, sgn_mul, aa);
                         __syncwarp();
                     }
             }
@@ -212,7 +193,8 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
                 const uint32_t w = pr / r, row = pr - w * r;
                 const float4 val = ((float4*)win)[q];
                 ((float4*)win)[q] = zero4;
-                red_add_v4(A.tables + (uint64_t)(w0 + w) * tstride + (uint64_t)row * P.cs + (uint64_t)panel * cw + 4u * c4, val);
+                SK_GUARD((uint64_t)panel * cw + 4u * c4 + 4u <= P.cs && w0 + w < P.n, kStatusBucket)
+                    red_add_v4(A.tables + (uint64_t)(w0 + w) * tstride + (uint64_t)row * P.cs + (uint64_t)panel * cw + 4u * c4, val);
             }
         }
         if (A.asum || flush) __syncthreads();
@@ -313,8 +295,10 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
         __stcs(m4 + (tc_), mm); __stcs(e4 + (tc_), aa);                                                             \
         if (ASUM) sts128(ast_lane + (c_) * 512u, aa);                                                               \
         _Pragma("unroll") for (uint32_t i = 0; i < r; ++i) {                                   \
-            const uint32_t addr = wrow[i] + ((h[i].x ^ o) & ~3u) * 4u;                                              \
-            float4 cur = lds128(addr);                                                                              \
+            const uint32_t woff = (h[i].x ^ o) & ~3u;                                                               \
+            const uint32_t addr = wrow[i] + woff * 4u;                                                              \
+            const bool inside = in_bounds(woff + 4u <= cw, P.status, kStatusWindow);                                \
+            float4 cur = inside ? lds128(addr) : zero4;                                                             \
             const uint32_t t3 = h[i].y * sgn_mul, t2 = t3 * 2u, t1 = t3 * 4u, t0 = t3 * 8u;                         \
             float4 sa;                                                                                              \
             sa.x = __uint_as_float(__float_as_uint(aa.x) ^ (t0 & 0x80000000u));                                     \
@@ -324,7 +308,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
             if (h[i].x & 1u) { float t = sa.x; sa.x = sa.y; sa.y = t; t = sa.z; sa.z = sa.w; sa.w = t; }            \
             if (h[i].x & 2u) { float t = sa.x; sa.x = sa.z; sa.z = t; t = sa.y; sa.y = sa.w; sa.w = t; }            \
             cur.x += sa.x; cur.y += sa.y; cur.z += sa.z; cur.w += sa.w;                                             \
-            sts128(addr, cur);                                                                                      \
+            if (inside) sts128(addr, cur);                                                                          \
             __syncwarp();                        /* the next sub-step's lanes may read what these wrote */          \
         }                                                                                                           \
         /* gradient sums on I_{t-1}: every worker's warp adds its quad (gsum is zero between steps) */            \
@@ -376,7 +360,8 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
                 const uint32_t w = pr / r, row = pr - w * r;
                 const float4 val = ((float4*)win)[q];
                 ((float4*)win)[q] = zero4;
-                red_add_v4(A.tables + (uint64_t)(w0 + w) * tstride + (uint64_t)row * P.cs + (uint64_t)panel * cw + 4u * c4, val);
+                SK_GUARD((uint64_t)panel * cw + 4u * c4 + 4u <= P.cs && w0 + w < P.n, kStatusBucket)
+                    red_add_v4(A.tables + (uint64_t)(w0 + w) * tstride + (uint64_t)row * P.cs + (uint64_t)panel * cw + 4u * c4, val);
             }
         }
         if (ASUM || flush) __syncthreads();

@@ -52,8 +52,21 @@ int scratch_for_device(unsigned char** out, char* msg, size_t msg_len) {
 
 }  // namespace
 
+// what the static selection found wrong is OR-ed into the handle's own status word, which sk_sync reads
+__global__ void k_merge_status(const sk::Select* from, sk::Select* to) {
+    if (from->status) atomicOr(&to->status, from->status);
+}
+
 // defined in sk_api.cu: records the message for sk_last_error() and returns `code`
 int sk_fail_message(int code, const char* message);
+
+// Called by sk_create (which may allocate): resolves the scratch address on the current device, so that loading the
+// module that holds the array, whatever that costs, does not fall on the first sk_select_static call.
+int sk_static_prepare(void) {
+    char msg[200];
+    unsigned char* base = nullptr;
+    return scratch_for_device(&base, msg, sizeof msg);
+}
 
 extern "C" int sk_select_static(sk_state* s, uint32_t* idx_out) {
     if (!s || !idx_out) return sk_fail_message(SK_EINVAL, "sk_select_static: null argument");
@@ -66,6 +79,7 @@ extern "C" int sk_select_static(sk_state* s, uint32_t* idx_out) {
     }
     if (s->t == 0) return sk_fail_message(SK_ESTATE, "sk_select_static: no step has been taken yet");
     if (s->cand_mult > 1) return sk_fail_message(SK_ESTATE, "sk_select_static: not available with a second round (P > 1)");
+    if (s->phase != 0) return sk_fail_message(SK_ESTATE, "sk_select_static: a partitioned step is in progress");
     char msg[200];
     unsigned char* base = nullptr;
     int rc = scratch_for_device(&base, msg, sizeof msg);
@@ -78,17 +92,20 @@ extern "C" int sk_select_static(sk_state* s, uint32_t* idx_out) {
     sk::Cand* cand = (sk::Cand*)(base + kOffCand);
     sk::Cand* cand2 = (sk::Cand*)(base + kOffCand2);
     cudaStream_t st = s->stream;
-    const bool vec = (P.d % 4 == 0) && P.log2g >= 2;
+    const bool vec = s->step_vec;       // the kernels of the last step: already loaded, nothing new is instantiated
+    sk::Params Ps = P;
+    Ps.status = &sel->status;           // the debug build's checks report into the scratch's own record
 
     // the array is shared by all calls and keeps the last call's contents: clear what must start at zero
     sk::launch_zero(base + kOffHist, kOffKeys - kOffHist, st);
     sk::MomentArgs A{};                 // members = 0: read vhat only, the step's own update is not repeated
     A.vhat = s->vhat;
     A.variant = (uint32_t)s->variant;
-    sk::launch_unsketch_hist(P, A, s->sum, keys, hist, vec, s->sm_count, st);
-    sk::launch_pick_bin(P, hist, sel, 0, st);
-    sk::launch_emit(P, keys, nullptr, sel, idx_out, cand, hist2, s->sm_count, st);
-    sk::launch_refine(P, sel, cand, cand2, hist2, idx_out, s->sm_count, st);
+    sk::launch_unsketch_hist(Ps, A, s->sum, keys, hist, vec, s->sm_count, st);
+    sk::launch_pick_bin(Ps, hist, sel, 0, st);
+    sk::launch_emit(Ps, keys, nullptr, sel, idx_out, cand, hist2, s->sm_count, st);
+    sk::launch_refine(Ps, sel, cand, cand2, hist2, idx_out, s->sm_count, st);
+    k_merge_status<<<1, 1, 0, st>>>(sel, s->sel);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) {
         snprintf(msg, sizeof msg, "sk_select_static: launch failed: %s", cudaGetErrorString(err));

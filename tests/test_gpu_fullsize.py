@@ -1,7 +1,9 @@
 """Parity at the full benchmark sizes, in the launch configuration bench.py times (default options).
 
-C2 and C3: two teacher-forced steps against the full oracle.  C4 and C5: the first step against the full oracle
-(every stage, every element), then a second GPU step checked through properties that hold at any size.
+C2 and C3: five and four teacher-forced steps against the full oracle.  C4 and C5: three teacher-forced steps against the full
+oracle (every stage, every element): from the second step on I_{t-1} is not empty, so the membership bitmap, the
+gradient sums carried over the several launches these sizes need, the lazy second moments with decay owed and the
+masked residual are all compared element by element.
 """
 import numpy as np
 import pytest
@@ -34,27 +36,32 @@ def _one_step(w, src, gpu, ora, t, x_gpu, x_ref, variant="ga"):
     gpu.sync()
     del g
     exact = None
+    members = ora.field("I_prev").astype(np.int64).copy()
     if ora.P > 1:          # gradient averaging only: what the second round ranks by, mean_w(m_t + e_{t-1}) / sqrt(vhat_t)
         e_sum = ora.field("e").astype(np.float64).sum(axis=0)
     ora.step(g_host, x_ref)
     if ora.P > 1:
         exact = (ora.field("m").astype(np.float64).sum(axis=0) + e_sum) / w.n / np.sqrt(ora.field("vhat").astype(np.float64))
-    return compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, variant=variant, exact_ref=exact)
+    return compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, variant=variant, exact_ref=exact,
+                        grads=g_host, members=members, beta2=w.beta2)
 
 
-@pytest.mark.parametrize("name", ["C2", "C3"])
-def test_two_teacher_forced_steps(name):
+@pytest.mark.parametrize("name,steps", [("C2", 5), ("C3", 4)])
+def test_teacher_forced_steps(name, steps):
     w, src, gpu, ora = _setup(name)
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
-    _one_step(w, src, gpu, ora, 1, x_gpu, x_ref)
-    force_state(gpu, ora)
-    x_gpu.copy_(torch.from_numpy(x_ref))
-    _one_step(w, src, gpu, ora, 2, x_gpu, x_ref)
+    for t in range(1, steps + 1):
+        if t > 1:
+            force_state(gpu, ora)
+            x_gpu.copy_(torch.from_numpy(x_ref))
+        _one_step(w, src, gpu, ora, t, x_gpu, x_ref)
 
 
-def test_c3_windowed_family_first_step():
-    w, src, gpu, ora = _setup("C3", window_lines=4)
+def test_c3_plain_family_first_step():
+    # the plain hash family (any group lands anywhere in its row) runs the reduction kernel: the fallback of every
+    # configuration the shared-memory kernel does not cover
+    w, src, gpu, ora = _setup("C3", window_lines=0)
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
     _one_step(w, src, gpu, ora, 1, x_gpu, x_ref)
@@ -81,35 +88,16 @@ def test_c3_second_round_two_teacher_forced_steps():
 
 
 @pytest.mark.parametrize("name", ["C4", "C5"])
-def test_first_step_full_then_properties(name):
+def test_three_teacher_forced_steps(name):
     w, src, gpu, ora = _setup(name)
     x_gpu = src.x0()
     x_ref = x_gpu.cpu().numpy().copy()
-    _one_step(w, src, gpu, ora, 1, x_gpu, x_ref)
+    for t in (1, 2, 3):
+        if t > 1:
+            force_state(gpu, ora)
+            x_gpu.copy_(torch.from_numpy(x_ref))
+        _one_step(w, src, gpu, ora, t, x_gpu, x_ref)
     ora.close()
-    # second step on the GPU alone: invariants of Algorithm 2 that need no reference
-    I1 = gpu.get("I")
-    vhat1 = gpu.get("vhat")
-    x1 = x_gpu.cpu().numpy().copy()
-    g = src.grads(2)
-    gpu.step(g, x_gpu)
-    gpu.sync()
-    I2 = gpu.get("I")
-    assert len(I2) == w.k and np.all(np.diff(I2.astype(np.int64)) > 0) and I2[-1] < w.d
-    vhat2 = gpu.get("vhat")
-    assert np.all(vhat2 >= vhat1)                                   # vhat = max(vhat, v) never decreases
-    assert np.isin(np.flatnonzero(vhat2 != vhat1), I1).all()        # and changes only on I_{t-1}
-    x2 = x_gpu.cpu().numpy()
-    assert np.isin(np.flatnonzero(x2 != x1), I2).all()              # x moves only on I_t
-    # h_t on I_{t-1}: v there is beta2 v + (1-beta2) mean_w(g)^2, spot-checked on a sample in fp64
-    sample = I1[:: max(1, len(I1) // 2000)]
-    gs = g[:, torch.from_numpy(sample.astype(np.int64)).cuda()].double().mean(0).cpu().numpy()
-    b2 = np.float64(np.float32(w.beta2))
-    v_prev = np.float64(np.float32(w.eps)) * b2                      # after step 1: eps decayed once
-    want = b2 * v_prev + (1 - b2) * gs ** 2
-    np.testing.assert_allclose(gpu.get("v")[sample], want, rtol=1e-5)
-    e = gpu.get("e")
-    assert not e[:, I2].any()
 
 
 def test_c2_hundred_free_running_steps_keep_the_invariants():

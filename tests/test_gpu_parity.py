@@ -104,10 +104,12 @@ def _run_steps(w, steps, log2g=None, teacher=True, cfg_id=None, check_tables=Tru
         gpu.step(g, x_gpu)
         gpu.sync()
         e_before = ora.field("e").astype(np.float64) if P > 1 else None
+        members = ora.field("I_prev").astype(np.int64).copy()
         ora.step(g_host, x_ref)
         diff = compare_step(gpu, ora, x_gpu.cpu().numpy(), x_ref, x_before, w.lr, check_tables=check_tables,
                             x_gpu_before=x_gpu_before, variant=variant,
-                            exact_ref=_exact_values(ora, e_before, variant) if P > 1 else None)
+                            exact_ref=_exact_values(ora, e_before, variant) if P > 1 else None,
+                            grads=g_host, members=members, beta2=w.beta2)
         if diff.size and diverged_at is None:
             diverged_at = t
             if not teacher:

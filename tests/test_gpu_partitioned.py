@@ -262,3 +262,37 @@ def test_partitioned_driver_single_process():
     # one process, same worker order: the same sums in the same order, hence the same bits
     assert np.array_equal(a.get("I"), b.get("I"))
     assert torch.equal(xa, xb)
+
+
+def test_partitioned_driver_orders_a_side_stream_against_the_collective():
+    # The handle launches on a stream of its own; the all-reduce is enqueued on torch's current stream.  Two processes
+    # with identical workers are emulated: the sum over them is twice the local share (exact in fp32), and every
+    # mean divides by 2n, so the result must be the bits of the n-worker one-call step.  Delays on both streams
+    # widen the windows: a collective that starts before its phase has finished, or a phase that starts before the
+    # collective has, would lose or repeat the doubling.
+    from paper_2210_07454_b200 import binding
+    from paper_2210_07454_b200.partitioned import PartitionedStep
+    from paper_2210_07454_b200.synthetic import GradientSource
+    w = _workload()
+    side = torch.cuda.Stream()
+
+    def doubled(t):
+        torch.cuda._sleep(20_000_000)               # the collective is slow: the next phase has to wait for it
+        t.mul_(2.0)
+
+    a = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, eps=w.eps)
+    b = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, eps=w.eps, workers_total=2 * w.n)
+    drv = PartitionedStep(b, "cuda", all_reduce=doubled, stream=side)
+    src = GradientSource(w, device="cuda")
+    xa, xb = src.x0(), src.x0()
+    for t in (1, 2):
+        g = src.grads(t)
+        a.step(g, xa)
+        with torch.cuda.stream(side):
+            torch.cuda._sleep(20_000_000)           # the handle's stream is busy: the phases start late
+        drv.step(g, xb)
+        torch.cuda.synchronize()
+        a.sync(), b.sync()
+        assert np.array_equal(a.get("I"), b.get("I")), t
+        assert torch.equal(xa, xb), t
+    b.set_stream(0)
