@@ -110,13 +110,16 @@ def _run(w, split, steps, variant="ga", P=1, window_lines=None, cfg_id=None, lr_
         x_before = x_ref.astype(np.float64).copy()
         x_own = xs[0].cpu().numpy().copy()
         e_before = ora.field("e").astype(np.float64) if P > 1 else None
+        members = ora.field("I_prev").astype(np.int64).copy()
+        g_host = g.float().cpu().numpy()
         ranks.step(g, xs)
         ranks.sync()
-        ora.step(g.float().cpu().numpy(), x_ref)
+        ora.step(g_host, x_ref)
         for x in xs[1:]:
             assert torch.equal(x, xs[0]), "the replicas of x disagree"
         compare_step(ranks, ora, xs[0].cpu().numpy(), x_ref, x_before, w.lr, x_gpu_before=x_own, variant=variant,
-                     exact_ref=_exact_values(ora, e_before, variant) if P > 1 else None)
+                     exact_ref=_exact_values(ora, e_before, variant) if P > 1 else None,
+                     grads=g_host, members=members, beta2=w.beta2)
     return ranks
 
 
@@ -157,11 +160,13 @@ def test_c1_sketch_of_the_local_worker_sum():
         x_before = x_ref.astype(np.float64).copy()
         x_own = xs[0].cpu().numpy().copy()
         e_before = ora.field("e").astype(np.float64)
+        members = ora.field("I_prev").astype(np.int64).copy()
+        g_host = g.cpu().numpy()
         ranks.step(g, xs)
         ranks.sync()
-        ora.step(g.cpu().numpy(), x_ref)
+        ora.step(g_host, x_ref)
         compare_step(ranks, ora, xs[0].cpu().numpy(), x_ref, x_before, w.lr, check_tables=False, x_gpu_before=x_own,
-                     exact_ref=_exact_values(ora, e_before, "ga"))
+                     exact_ref=_exact_values(ora, e_before, "ga"), grads=g_host, members=members, beta2=w.beta2)
 
 
 def test_c1_schedule_and_bf16_gradients():
@@ -284,7 +289,7 @@ def test_partitioned_driver_orders_a_side_stream_against_the_collective():
     b = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k, seed=w.seed, lr=w.lr, eps=w.eps, workers_total=2 * w.n)
     drv = PartitionedStep(b, "cuda", all_reduce=doubled, stream=side)
     src = GradientSource(w, device="cuda")
-    xa, xb = src.x0(), src.x0()
+    xa, xb, x0 = src.x0(), src.x0(), src.x0()
     for t in (1, 2):
         g = src.grads(t)
         a.step(g, xa)
@@ -294,5 +299,8 @@ def test_partitioned_driver_orders_a_side_stream_against_the_collective():
         torch.cuda.synchronize()
         a.sync(), b.sync()
         assert np.array_equal(a.get("I"), b.get("I")), t
-        assert torch.equal(xa, xb), t
+        # equal up to the rounding of the gradient sums behind vhat, which both handles accumulate in arrival order;
+        # a lost or repeated doubling would be off by a factor of two
+        moved = float((xa - x0).abs().max())
+        assert float((xa - xb).abs().max()) <= 1e-5 * moved, t
     b.set_stream(0)
