@@ -247,6 +247,16 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
         const uint2* hs = hsh + buf * r * kGroupsPerUnit + sg;
         const uint32_t t = unit * kQuadsPerUnit + tid;
         if (t < d4) {
+            // issued first: the row work below hides the latency of these two global loads
+            float4 vh = make_float4(1.f, 1.f, 1.f, 1.f);
+            uint32_t mask = 0;
+            if (A.variant != 1) {
+                vh = __ldcs((const float4*)A.vhat + t);
+                if (A.members) {
+                    const uint32_t word = unit * kGroupsPerUnit + sg;
+                    if (word < bm_words) mask = (__ldg(A.bitmap + word) >> o) & 0xFu;
+                }
+            }
             float qx[RMAX], qy[RMAX], qz[RMAX], qw[RMAX];
 #pragma unroll
             for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
@@ -274,12 +284,6 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
             if (A.variant == 1) {                                  // parameter averaging: U(S) takes no vhat (Algorithm 1)
                 k4.x = key_of(med.x); k4.y = key_of(med.y); k4.z = key_of(med.z); k4.w = key_of(med.w);
             } else {
-                float4 vh = ((const float4*)A.vhat)[t];
-                uint32_t mask = 0;
-                if (A.members) {
-                    const uint32_t word = unit * kGroupsPerUnit + sg;
-                    if (word < bm_words) mask = (__ldg(A.bitmap + word) >> o) & 0xFu;
-                }
                 if (mask) {
                     const float4 gs = ((const float4*)A.gsum)[t];
                     float4 vv = ((const float4*)A.v)[t];
