@@ -168,8 +168,9 @@ int sk_debug_check(sk_state* state, uint32_t kind);
  *                  of the exact values on I_t.  Only before the first step; allocates 8*n*d bytes.
  *   "window_lines" L > 0 selects the windowed variant of the hash family (needs g = 32, 32*L <= c): units of
  *                  1024 coordinates map into one aligned window of 32*L buckets per row, which lets the sketch
- *                  kernel accumulate in shared memory, one warp per worker.  Default: 8 when g = 32 and c >= 256,
- *                  else 0 (plain family; also what "log2g" < 5 selects).  Only before the first step.
+ *                  kernel accumulate in shared memory, one warp per worker.  Default: 8 when g = 32 and c >= 256
+ *                  (Algorithm 2), else 0 (plain family; also what "log2g" < 5 and, unless set explicitly,
+ *                  "variant" = 1 select).  Only before the first step.
  *   "window_workers" (1..8) workers per launch of the shared-memory sketch kernel (one warp each); default 8.
  *   "worker_sum"   1: the sketch kernel also stores sum_w a^(w) per coordinate (4*d bytes more written, allocated
  *                  when first enabled), and the update of x reads one value per index of I_t instead of n.

@@ -614,6 +614,7 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         if (value > 0 && (s->P.log2g != 5 || 32ull * (uint64_t)value > s->P.c))
             return fail(SK_EINVAL, "window_lines needs a hash group of 32 and 32*window_lines <= c");
         s->window_lines = value;
+        s->window_explicit = true;
         refresh_hash(s);
         return SK_OK;
     }
@@ -669,6 +670,12 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
             SK_CUDA(cudaStreamSynchronize(s->stream));
         }
         s->variant = value;
+        // Algorithm 1 runs the reduction kernels, whose reductions spread best over the plain family: it becomes the
+        // default there (windows confine a tile's reductions to a few lines of every table)
+        if (!s->window_explicit) {
+            s->window_lines = (value == 0 && s->P.log2g == 5 && s->P.c >= 32u * kDefaultWindowLines) ? kDefaultWindowLines : 0;
+            refresh_hash(s);
+        }
         return SK_OK;
     }
     if (!strcmp(key, "window_workers")) {

@@ -44,6 +44,21 @@ __device__ __forceinline__ float4 load_grad4(const void* grads, uint64_t q, uint
     }
     return __ldcs((const float4*)grads + q);
 }
+// The same in two halves, for software pipelines: the load leaves bf16 entries unwidened (in .x and .y of the
+// result), and the widening happens where the values are consumed, so that nothing depends on the load at issue time.
+__device__ __forceinline__ float4 load_grad4_raw(const void* grads, uint64_t q, uint32_t bf16) {
+    if (bf16) {
+        const uint2 raw = __ldcs((const uint2*)grads + q);
+        return make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), 0.0f, 0.0f);
+    }
+    return __ldcs((const float4*)grads + q);
+}
+__device__ __forceinline__ float4 widen_grad4(float4 raw, uint32_t bf16) {
+    if (!bf16) return raw;
+    const uint32_t lo = __float_as_uint(raw.x), hi = __float_as_uint(raw.y);
+    return make_float4(__uint_as_float(lo << 16), __uint_as_float(lo & 0xFFFF0000u),
+                       __uint_as_float(hi << 16), __uint_as_float(hi & 0xFFFF0000u));
+}
 __device__ __forceinline__ float load_grad1(const void* grads, uint64_t q, uint32_t bf16) {
     if (bf16) return __uint_as_float((uint32_t)((const uint16_t*)grads)[q] << 16);
     return ((const float*)grads)[q];

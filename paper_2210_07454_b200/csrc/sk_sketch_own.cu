@@ -222,7 +222,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, float4 v) {
 // sub-step i, (i + group) mod r, is folded into per-lane address registers (the hash stage repeats its first three
 // rows after the last so that the lane's stage address is affine in i); the chunk loop is unrolled by two only, which
 // keeps the loop body inside the instruction cache.
-template <int R, bool ASUM>
+template <int R, bool ASUM, bool BF16>
 __global__ void __launch_bounds__(256, 3)
 k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw,
                     uint32_t s_lo, uint32_t s_hi, uint32_t tbig, uint32_t rem) {
@@ -241,7 +241,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
 
     const uint32_t d4 = P.d >> 2;
     const float b1 = P.beta1, omb1 = 1.0f - P.beta1, rho = P.rho;
-    const uint32_t gb = A.grad_bf16;
+    constexpr uint32_t gb = BF16 ? 1u : 0u;      // compile-time: the widening of bf16 entries costs the fp32 path nothing
     const uint64_t wbase = (uint64_t)(w0 + wid) * d4;
     float4* m4 = (float4*)A.m + wbase;
     float4* e4 = (float4*)A.e + wbase;
@@ -276,17 +276,17 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
     float4 G0, M0, E0, G1, M1, E1;
     {
         const uint32_t t = walk.unit() * kQuadsPerUnit + lane;
-        G0 = load_grad4(A.grads, wbase + t, gb); M0 = __ldcs(m4 + t); E0 = __ldcs(e4 + t);
-        G1 = load_grad4(A.grads, wbase + t + 32u, gb); M1 = __ldcs(m4 + t + 32u); E1 = __ldcs(e4 + t + 32u);
+        G0 = load_grad4_raw(A.grads, wbase + t, gb); M0 = __ldcs(m4 + t); E0 = __ldcs(e4 + t);
+        G1 = load_grad4_raw(A.grads, wbase + t + 32u, gb); M1 = __ldcs(m4 + t + 32u); E1 = __ldcs(e4 + t + 32u);
     }
     __syncthreads();
 
 // one chunk: consume ring slot (G_, M_, E_) holding quad tc, refill it with quad tp, sketch into the windows
 #define SK_OWN_CHUNK(G_, M_, E_, c_, tc_, tp_)                                                                      \
     {                                                                                                               \
-        const float4 gg = G_;                                                                                       \
+        const float4 gg = widen_grad4(G_, gb);                                                                      \
         float4 mm = M_, aa = E_;                                                                                    \
-        G_ = load_grad4(A.grads, wbase + (tp_), gb); M_ = __ldcs(m4 + (tp_)); E_ = __ldcs(e4 + (tp_));              \
+        G_ = load_grad4_raw(A.grads, wbase + (tp_), gb); M_ = __ldcs(m4 + (tp_)); E_ = __ldcs(e4 + (tp_));          \
         uint2 h[R];                                                                                                 \
         _Pragma("unroll") for (uint32_t i = 0; i < r; ++i) h[i] = lds64(hs_c + i * (kGroupsPerUnit * 8u));          \
         uint32_t mask = 0;                                                                                          \
@@ -411,8 +411,13 @@ int launch_own(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, i
     // whole units in the fast form; a partial last unit goes to the general form as a launch of its own
     const uint32_t units_total = (P.d + kUnit - 1) / kUnit, units_full = P.d / kUnit;
     const size_t smem = own_smem(P, nw, R + 3, A.asum != nullptr);
-    int l = A.asum ? launch_own_kernel(k_moment_sketch_own<R, true>, smem, P, A, w0, nw, units_full, sm_count, st)
-                   : launch_own_kernel(k_moment_sketch_own<R, false>, smem, P, A, w0, nw, units_full, sm_count, st);
+    int l;
+    if (A.grad_bf16)
+        l = A.asum ? launch_own_kernel(k_moment_sketch_own<R, true, true>, smem, P, A, w0, nw, units_full, sm_count, st)
+                   : launch_own_kernel(k_moment_sketch_own<R, false, true>, smem, P, A, w0, nw, units_full, sm_count, st);
+    else
+        l = A.asum ? launch_own_kernel(k_moment_sketch_own<R, true, false>, smem, P, A, w0, nw, units_full, sm_count, st)
+                   : launch_own_kernel(k_moment_sketch_own<R, false, false>, smem, P, A, w0, nw, units_full, sm_count, st);
     if (l < 0) return l;
     if (units_total > units_full) {
         const int l2 = launch_own_any(P, A, w0, nw, 1u, units_full, sm_count, st);

@@ -21,6 +21,7 @@ struct sk_state {
     size_t l2_bytes = 0;
     int64_t worker_chunk = 0;
     int64_t window_lines = 0;
+    bool window_explicit = false; // window_lines was set by the caller (else the default may follow the variant)
     int64_t cand_mult = 1;        // P of Section III-A: candidates of the second round = P * k (1 = no second round)
     uint32_t *Ic = nullptr, *keys2 = nullptr;   // the P*k candidates and their exact-value keys
     int64_t variant = 0;          // 0 = gradient averaging (Algorithm 2), 1 = parameter averaging (Algorithm 1)
