@@ -189,7 +189,8 @@ int sk_get_option(const sk_state* state, const char* key, int64_t* value);
  *   stream(s,t) = t-th output of splitmix64 started at s;  K_row = stream(seed, row+1);
  *   q = i div g, o = i mod g, G = c div g;  u = stream(K_row, q+1), hi = u div 2^32, lo = u mod 2^32;
  *   x = hi*G;  h_row(i) = g*(x div 2^32) + (o xor p), p = the leading log2(g) bits of (x mod 2^32);
- *   s_row(i) = +1 if bit o of lo is clear, else -1. */
+ *   s_row(i) = +1 if bit 0 of lo is clear, else -1: one sign per (row, group).  The coordinates of a group never
+ *   share a bucket, so their relative sign never enters a sum; coordinates of different groups carry independent signs. */
 int sk_hash(const sk_state* state, uint32_t row, uint64_t i0, uint64_t count,
             uint32_t* idx_out, int8_t* sign_out);
 

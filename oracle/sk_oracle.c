@@ -21,10 +21,12 @@
  *                                                                    leading b bits of the remainder of the
  *                                                                    range reduction (p = 0 when g = 1)
  *   h_j(i) = g*B + (o xor p)
- *   s_j(i) = +1 if bit o of lo is 0, else -1
+ *   s_j(i) = +1 if bit 0 of lo is 0, else -1:  ONE sign per (row, group)
  *
- * Two coordinates of one group never share a bucket; two coordinates of different groups share one
- * with probability 1/(G*g).  With g = 1 this is an ordinary per-coordinate hash.
+ * Two coordinates of one group never share a bucket, so their relative sign never enters a bucket's sum; two
+ * coordinates of different groups share one with probability 1/(G*g) and carry independent signs, which is all
+ * the second-moment argument behind the Count Sketch uses.  With g = 1 this is an ordinary per-coordinate hash
+ * and sign.
  * ------------------------------------------------------------------------------------------------ */
 static const uint64_t GOLDEN = 0x9E3779B97F4A7C15ULL;
 
@@ -66,7 +68,7 @@ void ora_hash_one_w(uint64_t seed, uint32_t log2g, uint32_t window_lines, uint32
         base = ((i / ORA_UNIT) % P) * cw;
     }
     *bucket = (uint32_t)(base + g * B + (o ^ p));
-    *sign = ((lo >> o) & 1ULL) ? -1 : 1;
+    *sign = (lo & 1ULL) ? -1 : 1;
 }
 
 void ora_hash_one(uint64_t seed, uint32_t log2g, uint32_t c, uint32_t row, uint64_t i,

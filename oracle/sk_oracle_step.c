@@ -132,7 +132,7 @@ static inline void hash_at(const ora_state* s, uint32_t j, uint64_t i, uint32_t*
     uint64_t x = (u >> 32) * G;
     uint64_t p = s->log2g ? ((x & 0xFFFFFFFFULL) >> (32 - s->log2g)) : 0;
     *b = (uint32_t)(base + g * (x >> 32) + (o ^ p));
-    *sg = (((u & 0xFFFFFFFFULL) >> o) & 1ULL) ? -1 : 1;
+    *sg = (u & 1ULL) ? -1 : 1;             /* one sign per (row, group) */
 }
 
 static int ora_step_pa(ora_state* s, const float* grads, float* x);

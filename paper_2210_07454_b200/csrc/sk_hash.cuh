@@ -34,17 +34,17 @@ __device__ __forceinline__ uint32_t window_base(const Params& P, uint32_t i) {
 struct GroupHash {
     uint32_t base;   // first bucket of the group's aligned block (relative to the window base, if any)
     uint32_t perm;   // xor permutation inside the block, in [0,g)
-    uint32_t signs;  // bit o set  <=>  coordinate with offset o carries sign -1
+    uint32_t sign;   // 1  <=>  the group's coordinates carry sign -1 in this row (one sign per row and group)
 };
 
 // from one 64-bit draw u: high word -> block by multiply-high range reduction over P.G choices, the leading
-// bits of the remainder -> xor permutation, low word -> sign bits
+// bits of the remainder -> xor permutation, bit 0 of the low word -> the group's sign
 __device__ __forceinline__ GroupHash group_from_draw(const Params& P, uint64_t u) {
     const uint32_t hi = (uint32_t)(u >> 32);
     GroupHash h;
     h.base = __umulhi(hi, P.G) << P.log2g;
     h.perm = P.log2g ? ((hi * P.G) >> (32u - P.log2g)) : 0u;
-    h.signs = (uint32_t)u;
+    h.sign = (uint32_t)u & 1u;
     return h;
 }
 
@@ -53,15 +53,15 @@ __device__ __forceinline__ void coord_hash(const Params& P, uint64_t key, uint32
     const uint32_t q = i >> P.log2g, o = i & ((1u << P.log2g) - 1u);
     const GroupHash h = group_from_draw(P, stream(key, (uint64_t)q + 1));
     bucket = window_base(P, i) + h.base + (o ^ h.perm);
-    sign = ((h.signs >> o) & 1u) ? -1.0f : 1.0f;
+    sign = h.sign ? -1.0f : 1.0f;
 }
 
 // Vector form for 4 consecutive coordinates i..i+3 (i % 4 == 0, g >= 4): they land in one aligned 16-byte
 // chunk of the row.  `off` is the element offset of that chunk inside the row; local coordinate l goes to
-// element (l xor p3) of the chunk; bit l of the sign field is its sign.
+// element (l xor p3) of the chunk; all four carry the group's sign.
 struct Quad {
     uint32_t off;
-    uint32_t p3sgn;  // bits 0..1: p3 ; bits 2..5: sign bits of local coordinates 0..3
+    uint32_t p3sgn;  // bits 0..1: p3 ; bit 2: the sign bit (1 = negative)
 };
 
 __device__ __forceinline__ Quad quad_from_draw(const Params& P, uint64_t u, uint32_t i, uint32_t wbase) {
@@ -69,7 +69,7 @@ __device__ __forceinline__ Quad quad_from_draw(const Params& P, uint64_t u, uint
     const GroupHash h = group_from_draw(P, u);
     Quad r;
     r.off = wbase + h.base + ((o ^ h.perm) & ~3u);
-    r.p3sgn = (h.perm & 3u) | (((h.signs >> o) & 0xFu) << 2);
+    r.p3sgn = (h.perm & 3u) | (h.sign << 2);
     return r;
 }
 
@@ -97,7 +97,7 @@ __device__ __forceinline__ void quad_hashes(const Params& P, uint32_t r, uint32_
                         // g = 32 written out: block = floor(hi * G / 2^32), permutation = the next 5 bits
                         const uint32_t o = i & 31u, perm = (ohi * P.G) >> 27;
                         h[k + j].off = wbase + (__umulhi(ohi, P.G) << 5) + ((o ^ perm) & ~3u);
-                        h[k + j].p3sgn = (perm & 3u) | (((olo >> o) & 0xFu) << 2);
+                        h[k + j].p3sgn = (perm & 3u) | ((olo & 1u) << 2);
                     }
             }
         }
@@ -131,11 +131,11 @@ __device__ __forceinline__ float flip(float a, uint32_t bit) {  // a * (bit ? -1
 
 // signed and permuted: out element e = s(l) * a_l with l = e xor p3
 __device__ __forceinline__ float4 quad_scatter(const Quad h, float4 a) {
-    const uint32_t s = h.p3sgn;                       // sign bit of local coordinate l is bit 2 + l
-    a.x = __uint_as_float(__float_as_uint(a.x) ^ ((s << 29) & 0x80000000u));
-    a.y = __uint_as_float(__float_as_uint(a.y) ^ ((s << 28) & 0x80000000u));
-    a.z = __uint_as_float(__float_as_uint(a.z) ^ ((s << 27) & 0x80000000u));
-    a.w = __uint_as_float(__float_as_uint(a.w) ^ ((s << 26) & 0x80000000u));
+    const uint32_t s = (h.p3sgn << 29) & 0x80000000u;  // the group's sign bit, in the sign position of a float
+    a.x = __uint_as_float(__float_as_uint(a.x) ^ s);
+    a.y = __uint_as_float(__float_as_uint(a.y) ^ s);
+    a.z = __uint_as_float(__float_as_uint(a.z) ^ s);
+    a.w = __uint_as_float(__float_as_uint(a.w) ^ s);
     if (h.p3sgn & 1u) { float t = a.x; a.x = a.y; a.y = t; t = a.z; a.z = a.w; a.w = t; }
     if (h.p3sgn & 2u) { float t = a.x; a.x = a.z; a.z = t; t = a.y; a.y = a.w; a.w = t; }
     return a;
@@ -145,11 +145,11 @@ __device__ __forceinline__ float4 quad_scatter(const Quad h, float4 a) {
 __device__ __forceinline__ float4 quad_gather(const Quad h, float4 cch) {
     if (h.p3sgn & 1u) { float t = cch.x; cch.x = cch.y; cch.y = t; t = cch.z; cch.z = cch.w; cch.w = t; }
     if (h.p3sgn & 2u) { float t = cch.x; cch.x = cch.z; cch.z = t; t = cch.y; cch.y = cch.w; cch.w = t; }
-    const uint32_t s = h.p3sgn;                       // sign bit of local coordinate l is bit 2 + l
-    cch.x = __uint_as_float(__float_as_uint(cch.x) ^ ((s << 29) & 0x80000000u));
-    cch.y = __uint_as_float(__float_as_uint(cch.y) ^ ((s << 28) & 0x80000000u));
-    cch.z = __uint_as_float(__float_as_uint(cch.z) ^ ((s << 27) & 0x80000000u));
-    cch.w = __uint_as_float(__float_as_uint(cch.w) ^ ((s << 26) & 0x80000000u));
+    const uint32_t s = (h.p3sgn << 29) & 0x80000000u;  // the group's sign bit, in the sign position of a float
+    cch.x = __uint_as_float(__float_as_uint(cch.x) ^ s);
+    cch.y = __uint_as_float(__float_as_uint(cch.y) ^ s);
+    cch.z = __uint_as_float(__float_as_uint(cch.z) ^ s);
+    cch.w = __uint_as_float(__float_as_uint(cch.w) ^ s);
     return cch;
 }
 

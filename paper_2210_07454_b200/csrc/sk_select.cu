@@ -206,7 +206,7 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
     const uint32_t cw = P.win_cw;
     uint32_t* sh = dyn;                                            // [4096] histogram
-    uint2* hsh = (uint2*)(sh + kHistBins);                         // [2][r][32]: x = line*32 | perm, y = sign bits
+    uint2* hsh = (uint2*)(sh + kHistBins);                         // [2][r][32]: x = line*32 | perm, y = sign as +-1.0f
     float* win = (float*)(hsh + 2u * r * kGroupsPerUnit);          // [r][cw]: the panel's window of every row
     const uint32_t tid = threadIdx.x;
     for (uint32_t b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
@@ -214,14 +214,13 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
     const uint32_t s_end = (uint32_t)((uint64_t)units_total * (blockIdx.x + 1) / gridDim.x);
     const uint32_t d4 = P.d >> 2;
     const uint32_t sg = tid >> 3, o = (tid & 7u) * 4u;             // this thread's group inside the unit, offset inside it
-    const uint32_t sgn_mul = 1u << (28u - o);
     const uint32_t bm_words = (P.d + 31u) >> 5;
 
     auto fill_hashes = [&](uint32_t unit, uint32_t buf) {
         for (uint32_t hq = tid; hq < r * kGroupsPerUnit; hq += kThreads) {
             const uint32_t row = hq >> 5, s = hq & 31u;
             const GroupHash gh = group_from_draw(P, stream(P.row_key[row & (kMaxRows - 1u)], (uint64_t)unit * kGroupsPerUnit + s + 1));
-            hsh[buf * r * kGroupsPerUnit + hq] = make_uint2(gh.base | gh.perm, gh.signs);
+            hsh[buf * r * kGroupsPerUnit + hq] = make_uint2(gh.base | gh.perm, 0x3F800000u | (gh.sign << 31));
         }
     };
     auto load_windows = [&](uint32_t panel) {
@@ -265,14 +264,11 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                     const uint32_t woff = (h.x ^ o) & ~3u;
                     float4 cch = make_float4(0.f, 0.f, 0.f, 0.f);
                     SK_GUARD(woff + 4u <= cw, kStatusWindow) cch = *(const float4*)(win + row * cw + woff);
-                    // coordinate l of the quad sits at element l xor p3 of the chunk, with sign bit o + l of h.y
+                    // coordinate l of the quad sits at element l xor p3 of the chunk; h.y is the group's sign (+-1.0f)
                     if (h.x & 1u) { float u = cch.x; cch.x = cch.y; cch.y = u; u = cch.z; cch.z = cch.w; cch.w = u; }
                     if (h.x & 2u) { float u = cch.x; cch.x = cch.z; cch.z = u; u = cch.y; cch.y = cch.w; cch.w = u; }
-                    const uint32_t t3 = h.y * sgn_mul, t2 = t3 * 2u, t1 = t3 * 4u, t0 = t3 * 8u;
-                    qx[row] = __uint_as_float(__float_as_uint(cch.x) ^ (t0 & 0x80000000u));
-                    qy[row] = __uint_as_float(__float_as_uint(cch.y) ^ (t1 & 0x80000000u));
-                    qz[row] = __uint_as_float(__float_as_uint(cch.z) ^ (t2 & 0x80000000u));
-                    qw[row] = __uint_as_float(__float_as_uint(cch.w) ^ (t3 & 0x80000000u));
+                    const float sg = __uint_as_float(h.y);
+                    qx[row] = sg * cch.x; qy[row] = sg * cch.y; qz[row] = sg * cch.z; qw[row] = sg * cch.w;
                 }
             float4 med;
             if constexpr (R > 0) {

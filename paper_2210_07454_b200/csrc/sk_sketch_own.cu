@@ -43,25 +43,20 @@ __device__ __forceinline__ void red_add_v4(float* addr, float4 v) {
 struct Chunk { float4 g, m, e; };
 
 // One read-add-write of this lane's four signed values into its worker's window of a row.
-// h.x = 32 * line + perm of the lane's group in that row, h.y = the group's 32 sign bits; o = 4 * (lane mod 8) is the
-// offset of the lane's first coordinate inside the group, sgn_mul = 2^(28 - o).
-// Shifts are written as multiplications so that they issue on the multiply-add pipe; the logic pipe, which this
-// kernel loads most, is left with one operation per sign and per select.
-__device__ __forceinline__ void window_add(const Params& P, float* wrow, const uint2 h, uint32_t o, uint32_t sgn_mul, float4 a) {
+// h.x = 32 * line + perm of the lane's group in that row, h.y = the group's sign in that row as the float +1 or -1;
+// o = 4 * (lane mod 8) is the offset of the lane's first coordinate inside the group.
+// The sign rides on the accumulation (one fused multiply-add per element); the logic pipe, which this kernel loads
+// most, is left with the selects of the xor-permutation.
+__device__ __forceinline__ void window_add(const Params& P, float* wrow, const uint2 h, uint32_t o, float4 a) {
     const uint32_t off = (h.x ^ o) & ~3u;                          // line of the group, chunk after the xor permutation
     if (!in_bounds(off + 4u <= P.win_cw, P.status, kStatusWindow)) return;
-    const uint32_t t3 = h.y * sgn_mul;                             // sign bit of local coordinate 3 in bit 31
-    const uint32_t t2 = t3 * 2u, t1 = t3 * 4u, t0 = t3 * 8u;       // ... of 2, 1, 0 in bit 31
-    a.x = __uint_as_float(__float_as_uint(a.x) ^ (t0 & 0x80000000u));
-    a.y = __uint_as_float(__float_as_uint(a.y) ^ (t1 & 0x80000000u));
-    a.z = __uint_as_float(__float_as_uint(a.z) ^ (t2 & 0x80000000u));
-    a.w = __uint_as_float(__float_as_uint(a.w) ^ (t3 & 0x80000000u));
+    const float sg = __uint_as_float(h.y);
     // element e of the chunk receives local coordinate e xor p3
     if (h.x & 1u) { float t = a.x; a.x = a.y; a.y = t; t = a.z; a.z = a.w; a.w = t; }
     if (h.x & 2u) { float t = a.x; a.x = a.z; a.z = t; t = a.y; a.y = a.w; a.w = t; }
     float4* dst = (float4*)(wrow + off);
     float4 cur = *dst;
-    cur.x += a.x; cur.y += a.y; cur.z += a.z; cur.w += a.w;
+    cur.x = fmaf(sg, a.x, cur.x); cur.y = fmaf(sg, a.y, cur.y); cur.z = fmaf(sg, a.z, cur.z); cur.w = fmaf(sg, a.w, cur.w);
     *dst = cur;
 }
 
@@ -75,7 +70,7 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
     const uint32_t cw = P.win_cw;
     float* win = smem;                                             // [nw][r][cw]
-    uint2* hsh = (uint2*)(win + (size_t)nw * r * cw);              // [2][r][32]: x = line*32 | perm, y = sign bits
+    uint2* hsh = (uint2*)(win + (size_t)nw * r * cw);              // [2][r][32]: x = line*32 | perm, y = sign as +-1.0f
     float4* ast = (float4*)(hsh + 2u * r * kGroupsPerUnit);        // [nw][256]: a_t of the unit (only with A.asum)
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, wid = tid >> 5;
@@ -94,14 +89,13 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
     const uint64_t tstride = (uint64_t)P.r * P.cs;
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
     const uint32_t grp = lane >> 3, o = (lane & 7u) * 4u;          // this lane's group in the chunk, offset inside it
-    const uint32_t sgn_mul = 1u << (28u - o);
     float* mywin = win + (size_t)wid * r * cw;
 
     auto fill_hashes = [&](uint32_t unit, uint32_t buf) {
         for (uint32_t hq = tid; hq < r * kGroupsPerUnit; hq += nthreads) {
             const uint32_t row = hq >> 5, s = hq & 31u;
             const GroupHash gh = group_from_draw(P, stream(P.row_key[row & (kMaxRows - 1u)], (uint64_t)unit * kGroupsPerUnit + s + 1));
-            hsh[buf * r * kGroupsPerUnit + hq] = make_uint2(gh.base | gh.perm, gh.signs);
+            hsh[buf * r * kGroupsPerUnit + hq] = make_uint2(gh.base | gh.perm, 0x3F800000u | (gh.sign << 31));
         }
     };
     auto issue = [&](uint32_t unit, uint32_t c, bool have, Chunk& k) {
@@ -153,14 +147,14 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
                     if (i < r) {
                         uint32_t row = i + grp;
                         if (row >= r) row -= r;
-                        window_add(P, mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, sgn_mul, aa);
+                        window_add(P, mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, aa);
                         __syncwarp();                              // the next sub-step's lanes may read what these wrote
                     }
                 }
             } else {
                 for (uint32_t row = 0; row < r; ++row)
                     for (uint32_t q = 0; q < 4; ++q) {             // fewer rows than groups: the groups take turns
-                        if (grp == q) window_add(P, mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, sgn_mul, aa);
+                        if (grp == q) window_add(P, mywin + row * cw, hs[row * kGroupsPerUnit + sg], o, aa);
                         __syncwarp();
                     }
             }
@@ -230,7 +224,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
     constexpr uint32_t r = (uint32_t)R, HR = (uint32_t)R + 3u;     // rows of the hash stage
     const uint32_t cw = P.win_cw;
     float* win = smem;                                             // [nw][r][cw]
-    uint2* hsh = (uint2*)(win + (size_t)nw * r * cw);              // [2][HR][32]: x = line*32 | perm, y = sign bits
+    uint2* hsh = (uint2*)(win + (size_t)nw * r * cw);              // [2][HR][32]: x = line*32 | perm, y = sign as +-1.0f
     float4* ast = (float4*)(hsh + 2u * HR * kGroupsPerUnit);       // [nw][256]: a_t of the unit (ASUM)
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, wid = tid >> 5;
@@ -248,7 +242,6 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
     const uint64_t tstride = (uint64_t)P.r * P.cs;
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
     const uint32_t grp = lane >> 3, o = (lane & 7u) * 4u;          // this lane's group in the chunk, offset inside it
-    const uint32_t sgn_mul = 1u << (28u - o);
     const uint32_t members = A.members, gsum_on = A.gsum_on;
 
     // per-lane shared addresses: the window row of sub-step i, and the stage entry of (row = group + i, group of chunk 0)
@@ -264,7 +257,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
             const uint32_t rowx = hq >> 5, s = hq & 31u;
             const uint32_t row = rowx < r ? rowx : rowx - r;
             const GroupHash gh = group_from_draw(P, stream(P.row_key[row & (kMaxRows - 1u)], (uint64_t)unit * kGroupsPerUnit + s + 1));
-            hsh[buf * HR * kGroupsPerUnit + hq] = make_uint2(gh.base | gh.perm, gh.signs);
+            hsh[buf * HR * kGroupsPerUnit + hq] = make_uint2(gh.base | gh.perm, 0x3F800000u | (gh.sign << 31));
         }
     };
 
@@ -299,15 +292,12 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
             const uint32_t addr = wrow[i] + woff * 4u;                                                              \
             const bool inside = in_bounds(woff + 4u <= cw, P.status, kStatusWindow);                                \
             float4 cur = inside ? lds128(addr) : zero4;                                                             \
-            const uint32_t t3 = h[i].y * sgn_mul, t2 = t3 * 2u, t1 = t3 * 4u, t0 = t3 * 8u;                         \
-            float4 sa;                                                                                              \
-            sa.x = __uint_as_float(__float_as_uint(aa.x) ^ (t0 & 0x80000000u));                                     \
-            sa.y = __uint_as_float(__float_as_uint(aa.y) ^ (t1 & 0x80000000u));                                     \
-            sa.z = __uint_as_float(__float_as_uint(aa.z) ^ (t2 & 0x80000000u));                                     \
-            sa.w = __uint_as_float(__float_as_uint(aa.w) ^ (t3 & 0x80000000u));                                     \
+            float4 sa = aa;                                                                                         \
+            const float sg = __uint_as_float(h[i].y);     /* the group's sign in this row, +1 or -1 */              \
             if (h[i].x & 1u) { float t = sa.x; sa.x = sa.y; sa.y = t; t = sa.z; sa.z = sa.w; sa.w = t; }            \
             if (h[i].x & 2u) { float t = sa.x; sa.x = sa.z; sa.z = t; t = sa.y; sa.y = sa.w; sa.w = t; }            \
-            cur.x += sa.x; cur.y += sa.y; cur.z += sa.z; cur.w += sa.w;                                             \
+            cur.x = fmaf(sg, sa.x, cur.x); cur.y = fmaf(sg, sa.y, cur.y);                                           \
+            cur.z = fmaf(sg, sa.z, cur.z); cur.w = fmaf(sg, sa.w, cur.w);                                           \
             if (inside) sts128(addr, cur);                                                                          \
             __syncwarp();                        /* the next sub-step's lanes may read what these wrote */          \
         }                                                                                                           \

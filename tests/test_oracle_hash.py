@@ -41,7 +41,7 @@ def _family(seed, log2g, c, row, i):
     hi, lo = divmod(u, 1 << 32)
     B, rem = divmod(hi * G, 1 << 32)
     p = (rem * g) >> 32                      # leading log2(g) bits of the 32-bit remainder
-    return g * B + (o ^ p), (-1 if (lo >> o) & 1 else 1)
+    return g * B + (o ^ p), (-1 if lo & 1 else 1)          # one sign per (row, group)
 
 
 @pytest.mark.parametrize("log2g", [0, 1, 2, 3, 4, 5])
@@ -111,10 +111,16 @@ def test_pair_collision_rate_and_sign_balance(log2g):
     c, N = 4096, 60_000
     g = 1 << log2g
     b, s = oracle.hash_family(3, log2g, c, 0, 0, N)
-    assert abs(s.astype(np.float64).mean()) < 5 / np.sqrt(N)
-    # sign pairs inside a group and across groups are uncorrelated
-    assert abs((s[:-1].astype(np.float64) * s[1:]).mean()) < 5 / np.sqrt(N)
-    assert abs((s[:-g].astype(np.float64) * s[g:]).mean()) < 5 / np.sqrt(N)
+    # one sign per (row, group): constant inside a group (whose coordinates never meet in a bucket), balanced and
+    # uncorrelated across groups (whose coordinates do), and uncorrelated across rows
+    sg = s[: (N // g) * g].reshape(-1, g).astype(np.float64)
+    assert np.all(sg == sg[:, :1])
+    n_groups = sg.shape[0]
+    assert abs(sg[:, 0].mean()) < 5 / np.sqrt(n_groups)
+    for lag in (1, 2, 7):
+        assert abs((sg[:-lag, 0] * sg[lag:, 0]).mean()) < 5 / np.sqrt(n_groups)
+    s_other = oracle.hash_family(3, log2g, c, 1, 0, N)[1][: (N // g) * g].reshape(-1, g)[:, 0].astype(np.float64)
+    assert abs((sg[:, 0] * s_other).mean()) < 5 / np.sqrt(n_groups)
     # collisions: count pairs sharing a bucket
     cnt = np.bincount(b, minlength=c).astype(np.float64)
     pairs_same_bucket = (cnt * (cnt - 1) / 2).sum()
@@ -143,7 +149,7 @@ def _family_w(seed, L, c, row, i):
     hi, lo = divmod(u, 1 << 32)
     line, rem = divmod(hi * L, 1 << 32)
     p = (rem * 32) >> 32
-    return ((i // 1024) % P) * cw + 32 * line + (o ^ p), (-1 if (lo >> o) & 1 else 1)
+    return ((i // 1024) % P) * cw + 32 * line + (o ^ p), (-1 if lo & 1 else 1)
 
 
 @pytest.mark.parametrize("L", [1, 4, 8, 16])

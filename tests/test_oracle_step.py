@@ -207,13 +207,18 @@ def test_frozen_second_moments():
         assert np.array_equal(a, b)
     assert np.array_equal(runs[1.0][2], runs[4.0][2])
     np.testing.assert_allclose(runs[4.0][1], runs[1.0][1] / 2, rtol=3e-7, atol=0)
-    # and the moving-vhat run differs (the switch does something)
-    o = oracle.Oracle(d, n, r, c, k, seed=3, log2g=3, lr=0.25, eps=1.0)
-    rng = np.random.default_rng(7)
-    x = np.zeros(d, np.float32)
-    for t in range(6):
-        o.step(rng.standard_normal((n, d)).astype(np.float32), x)
-    assert np.any(o.field("vhat") > 1.0) and not np.array_equal(x, runs[1.0][1])
+    # and the moving-vhat run differs (the switch does something): long enough for coordinates whose vhat has grown
+    # to be selected again
+    xs = {}
+    for frozen in (True, False):
+        o = oracle.Oracle(d, n, r, c, k, seed=3, log2g=3, lr=0.25, eps=1.0, freeze_v=frozen)
+        rng = np.random.default_rng(7)
+        x = np.zeros(d, np.float32)
+        for t in range(30):
+            o.step((3.0 * rng.standard_normal((n, d))).astype(np.float32), x)     # h^2 is often above v = 1
+        xs[frozen] = x
+        assert (np.count_nonzero(o.field("vhat") > 1.0) > 40) == (not frozen)
+    assert not np.array_equal(xs[True], xs[False])
 
 
 def test_no_compression_reduces_to_distributed_amsgrad():
