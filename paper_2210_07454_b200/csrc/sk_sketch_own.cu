@@ -217,7 +217,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, float4 v) {
 // rows after the last so that the lane's stage address is affine in i); the chunk loop is unrolled by two only, which
 // keeps the loop body inside the instruction cache.
 template <int R, bool ASUM, bool BF16>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, 3)      // 3 blocks = 24 warps per SM; 2 and 4 (spills) measured slower
 k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw,
                     uint32_t s_lo, uint32_t s_hi, uint32_t tbig, uint32_t rem) {
     extern __shared__ __align__(16) float smem[];
