@@ -119,7 +119,8 @@ int sk_set_stream(sk_state* state, void* stream);
  * number of indices other than k.  Bits 1..5 exist in the debug build (compiled with -DSK_DEBUG=1, see
  * paper_2210_07454_b200/build.py --debug), whose kernels compare every hashed table offset, coordinate index, list
  * position, histogram bin and shared-memory window offset with the size of what it addresses, record a violation
- * here and skip the access; nothing traps. */
+ * here and skip the access; nothing traps.  Bit 6 (debug build): a gradient entry was not finite -- inputs must be
+ * finite; the step is taken regardless and its results are then unspecified. */
 int sk_sync(sk_state* state);
 
 /* Per-step statistics of the last step's selection (Algorithm 2's Top-k) and the method's exchange volume, for
@@ -136,7 +137,7 @@ int sk_get_stats(sk_state* state, double* out, uint32_t count);
  * sk_test_fail_allocation(nth): the (nth+1)-th device allocation of the following sk_create calls fails as if the
  * device were out of memory (sk_create then returns NULL with a message and frees what it had allocated); nth < 0
  * switches the hook off.  Process-wide; not thread-safe.
- * sk_debug_check(state, kind), kind 1..5: in the debug build a one-thread kernel runs the bounds check of that kind
+ * sk_debug_check(state, kind), kind 1..6: in the debug build a one-thread kernel runs the bounds check of that kind
  * with a false condition (no access is made), so the next sk_sync must report bit `kind`; SK_ESTATE in the normal
  * build, which has no device-side checks.  The paper has no counterpart for either. */
 int sk_test_fail_allocation(int64_t nth);

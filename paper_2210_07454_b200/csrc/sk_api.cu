@@ -114,7 +114,8 @@ int check_status(sk_state* s) {
         SK_CUDA(cudaMemsetAsync(&s->sel->status, 0, sizeof(uint32_t), s->stream));
         SK_CUDA(cudaStreamSynchronize(s->stream));
         return fail(SK_EDEVICE, "device status word = 0x%x (bit 0: selection emitted %u of %u indices; bits 1-5, debug "
-                    "build: table offset, index, list position, histogram bin, window offset out of range)", h.status,
+                    "build: table offset, index, list position, histogram bin, window offset out of range; bit 6, debug "
+                    "build: a gradient entry was not finite)", h.status,
                     h.cnt_out, s->P.k);
     }
     return SK_OK;
@@ -569,7 +570,7 @@ int sk_test_fail_allocation(int64_t nth) {
 int sk_debug_check(sk_state* s, uint32_t kind) {
     if (!s) return fail(SK_EINVAL, "null handle");
 #ifdef SK_DEBUG
-    if (kind < 1 || kind > 5) return fail(SK_EINVAL, "kind must be in 1..5");
+    if (kind < 1 || kind > 6) return fail(SK_EINVAL, "kind must be in 1..6");
     sk::launch_debug_violation(s->P, 1u << kind, s->stream);
     SK_CUDA(cudaGetLastError());
     return SK_OK;

@@ -16,6 +16,7 @@ enum : uint32_t {
     kStatusListPos = 8u,    // an append position outside the list's capacity
     kStatusBin = 16u,       // a histogram bin outside the histogram
     kStatusWindow = 32u,    // a shared-memory window offset outside the window
+    kStatusNonFinite = 64u, // a gradient entry that is not finite (inputs must be finite; the step goes on regardless)
 };
 
 #ifdef SK_DEBUG
@@ -28,6 +29,14 @@ __device__ __forceinline__ bool in_bounds(bool, uint32_t*, uint32_t) { return tr
 #endif
 
 }  // namespace sk
+
+// debug build: a non-finite entry of a gradient quad is recorded (nothing is skipped: the arithmetic cannot fault)
+#ifdef SK_DEBUG
+#define SK_CHECK_FINITE4(g)                                                                                   \
+    sk::in_bounds(isfinite((g).x) && isfinite((g).y) && isfinite((g).z) && isfinite((g).w), P.status, sk::kStatusNonFinite)
+#else
+#define SK_CHECK_FINITE4(g) ((void)0)
+#endif
 
 // `statement` runs only if `cond` holds; in the debug build a failed `cond` is recorded in P.status
 #define SK_GUARD(cond, bit) if (sk::in_bounds((cond), P.status, (bit)))

@@ -117,6 +117,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             const float4 g0 = load_grad4(A.grads, q0, gb), g1 = load_grad4(A.grads, q1, gb);
             float4 m0 = __ldcs(m + q0), m1 = __ldcs(m + q1);
             float4 a0 = __ldcs(e + q0), a1 = __ldcs(e + q1);
+            SK_CHECK_FINITE4(g0); SK_CHECK_FINITE4(g1);
             SK_MOMENT(m0, a0, g0, mask)
             SK_MOMENT(m1, a1, g1, mask)
             gs.x = (gs.x + g0.x) + g1.x; gs.y = (gs.y + g0.y) + g1.y;
@@ -141,6 +142,7 @@ k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ Mom
             const float4 g0 = load_grad4(A.grads, q0, gb);
             float4 m0 = __ldcs(m + q0);
             float4 a0 = __ldcs(e + q0);
+            SK_CHECK_FINITE4(g0);
             SK_MOMENT(m0, a0, g0, mask)
             gs.x += g0.x; gs.y += g0.y; gs.z += g0.z; gs.w += g0.w;
             as.x += a0.x; as.y += a0.y; as.z += a0.z; as.w += a0.w;

@@ -137,6 +137,7 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
             const bool live = t < d4;
             const uint32_t mask = (__shfl_sync(0xFFFFFFFFu, bmw, c * 4u + grp) >> o) & 0xFu;
             float4 mm = k.m, aa = k.e;
+            if (live) SK_CHECK_FINITE4(k.g);
             SK_MOMENT(mm, aa, k.g, mask)
             if (live) { __stcs(m + wbase + t, mm); __stcs(e + wbase + t, aa); }
             if (A.asum) ast[wid * kQuadsPerUnit + c * 32u + lane] = aa;
@@ -284,6 +285,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
         _Pragma("unroll") for (uint32_t i = 0; i < r; ++i) h[i] = lds64(hs_c + i * (kGroupsPerUnit * 8u));          \
         uint32_t mask = 0;                                                                                          \
         if (members) mask = (__shfl_sync(0xFFFFFFFFu, bmw, (c_) * 4u + grp) >> o) & 0xFu;                           \
+        SK_CHECK_FINITE4(gg);                                                                                       \
         SK_MOMENT(mm, aa, gg, mask)                                                                                 \
         __stcs(m4 + (tc_), mm); __stcs(e4 + (tc_), aa);                                                             \
         if (ASUM) sts128(ast_lane + (c_) * 512u, aa);                                                               \

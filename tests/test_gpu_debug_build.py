@@ -43,7 +43,7 @@ opt = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k)
 x = src.x0()
 opt.step(src.grads(1), x); opt.sync()
 I1 = opt.get("I")
-for kind in (1, 2, 3, 4, 5):
+for kind in (1, 2, 3, 4, 5, 6):
     opt.debug_check(kind)                       # a failed check of this kind, with no access behind it
     try:
         opt.sync()
@@ -54,6 +54,16 @@ for kind in (1, 2, 3, 4, 5):
     opt.sync()                                  # reported once, then cleared: the handle stays usable
 opt.step(src.grads(2), x); opt.sync()
 assert len(opt.get("I")) == w.k and opt.stats()["status"] == 0.0
+# a non-finite gradient entry is an invalid input: the debug build's kernels notice it and the host gets an error
+fresh = binding.SketchedAMSGrad(w.d, w.n, w.r, w.c, w.k)
+bad = src.grads(3).clone(); bad[1, 12345] = float("nan")
+fresh.step(bad, src.x0())
+try:
+    fresh.sync()
+except binding.SkError as err:
+    assert "0x40" in str(err), str(err)
+else:
+    raise SystemExit("the non-finite entry was not reported")
 print("child ok")
 """
 
