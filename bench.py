@@ -13,6 +13,7 @@ from __future__ import annotations
 import argparse
 import hashlib
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -111,7 +112,13 @@ class ClockSampler:
             per_rep.append(statistics.median(v) if v else None)
         return {"sm_mhz": statistics.median([r[1] for r in use]) if use else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(rows), "samples_in_timed_region": len(inside),
-                "sm_mhz_per_repetition": per_rep}
+                "sm_mhz_per_repetition": per_rep if len(per_rep) <= 20 else self._spread(per_rep)}
+
+    @staticmethod
+    def _spread(per_rep):
+        seen = [v for v in per_rep if v is not None]
+        return {"repetitions_with_samples": len(seen), "min": min(seen) if seen else None,
+                "median": statistics.median(seen) if seen else None, "max": max(seen) if seen else None}
 
 
 def _dist():
@@ -273,7 +280,9 @@ def main():
     ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-scale", type=int, default=0, help="reference arm: 1/SCALE size per step (0 = full size if it fits the time budget)")
-    ap.add_argument("--reps", type=int, default=10, help="repetitions of the --steps long timed loop; the median is reported")
+    ap.add_argument("--reps", type=int, default=0,
+                    help="repetitions of the --steps long timed loop, the median is reported; 0 = as many as fill about "
+                         "one second (at least 10, at most 400), so that the clock sampler sees the timed region")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the short C4 and C5 runs reported beside the headline")
     ap.add_argument("--scale", type=int, default=1, help="run the workload at 1/SCALE size (profiling captures)")
     ap.add_argument("--grad-sets", type=int, default=0, help="rotating gradient sets (0 = as many as fit, 2..4)")
@@ -358,7 +367,9 @@ def main():
     # the --steps long loop is timed `reps` times (CUDA events on the launching stream, barrier and synchronize on both
     # sides of every repetition, max over ranks); the median repetition is the reported step time
     rep_ms, windows = [], []
-    for rep in range(max(1, args.reps)):
+    reps = args.reps if args.reps > 0 else 10
+    rep = 0
+    while rep < reps:
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
@@ -373,6 +384,9 @@ def main():
         if world > 1:
             dist.barrier()
         rep_ms.append(reduce_max(ev0.elapsed_time(ev1), world, dev))
+        rep += 1
+        if args.reps <= 0 and rep == 1:              # every rank derives the same count from the reduced time
+            reps = int(min(400, max(10, math.ceil(1000.0 / max(rep_ms[0], 1e-3)))))
     clocks = sampler.stop(windows) if rank == 0 else None
     opt.sync()
     ms_total = statistics.median(rep_ms)
