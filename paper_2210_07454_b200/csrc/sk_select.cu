@@ -108,6 +108,17 @@ __device__ __forceinline__ float median1(const Params& P, const float* __restric
     return median_any(q, P.r);
 }
 
+// a 16-byte global load that stays where it is written (the compiler would otherwise move it down to its first use)
+template <typename T4>
+__device__ __forceinline__ T4 ldg128_here(const T4* p) {
+    uint32_t a, b, c, d;
+    asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "l"(p) : "memory");
+    T4 out;
+    uint32_t* w = reinterpret_cast<uint32_t*>(&out);
+    w[0] = a; w[1] = b; w[2] = c; w[3] = d;
+    return out;
+}
+
 // one count in a shared-memory histogram of kHistBins bins (the bin is checked in the debug build)
 __device__ __forceinline__ void hist_add(const Params& P, uint32_t* sh, uint32_t bin) {
     SK_GUARD(bin < kHistBins, kStatusBin) atomicAdd(&sh[bin], 1u);
@@ -198,7 +209,7 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
 // r 16-byte shared-memory reads, sign and xor-permutation undone in registers, median, key, histogram.  Against the
 // general kernel this drops the per-quad hash exchange by shuffles and the L2 gathers.
 template <int R>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 5)
 k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, const float* __restrict__ sum,
                     uint32_t* keys, uint32_t* hist, uint32_t units_total, uint32_t tbig, uint32_t rem) {
     extern __shared__ __align__(16) uint32_t dyn[];
@@ -230,11 +241,20 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
         }
     };
 
+    // this thread's four membership bits of I_{t-1} in a unit (0 where the pass does not update v and vhat)
+    const bool members = A.variant != 1 && A.members;
+    auto member_bits = [&](uint32_t unit) -> uint32_t {
+        const uint32_t word = unit * kGroupsPerUnit + sg;
+        return (members && word < bm_words && unit * kQuadsPerUnit + tid < d4) ? (__ldg(A.bitmap + word) >> o) & 0xFu : 0u;
+    };
+
     UnitWalk walk{P.win_panels, tbig, rem, 0u, 0u};
+    uint32_t mask_ahead = 0;
     if (s_begin < s_end) {
         walk.seek(s_begin);
         fill_hashes(walk.unit(), 0u);
         load_windows(walk.panel);
+        mask_ahead = member_bits(walk.unit());
     }
     __syncthreads();
     for (uint32_t s = s_begin; s < s_end; ++s) {
@@ -242,20 +262,23 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
         const uint32_t unit = walk.unit(), panel = walk.panel;
         const bool have_next = s + 1 < s_end;
         walk.next();
+        // The membership word was fetched one unit ahead, so the loads of a member's gsum, v and stamp can be issued
+        // here, with the load of vhat, and the row work below hides their latency.
+        const uint32_t mask = mask_ahead;
+        const uint32_t t = unit * kQuadsPerUnit + tid;
+        float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), vv = gs;
+        uint4 vs = make_uint4(0u, 0u, 0u, 0u);
+        float4 vh = make_float4(1.f, 1.f, 1.f, 1.f);
+        if (t < d4 && A.variant != 1) vh = ldg128_here<float4>((const float4*)A.vhat + t);
+        if (mask) {
+            gs = ldg128_here<float4>((const float4*)A.gsum + t);
+            vv = ldg128_here<float4>((const float4*)A.v + t);
+            vs = ldg128_here<uint4>((const uint4*)A.vstamp + t);
+        }
+        mask_ahead = have_next ? member_bits(walk.unit()) : 0u;
         if (have_next) fill_hashes(walk.unit(), buf ^ 1u);
         const uint2* hs = hsh + buf * r * kGroupsPerUnit + sg;
-        const uint32_t t = unit * kQuadsPerUnit + tid;
         if (t < d4) {
-            // issued first: the row work below hides the latency of these two global loads
-            float4 vh = make_float4(1.f, 1.f, 1.f, 1.f);
-            uint32_t mask = 0;
-            if (A.variant != 1) {
-                vh = __ldcs((const float4*)A.vhat + t);
-                if (A.members) {
-                    const uint32_t word = unit * kGroupsPerUnit + sg;
-                    if (word < bm_words) mask = (__ldg(A.bitmap + word) >> o) & 0xFu;
-                }
-            }
             float qx[RMAX], qy[RMAX], qz[RMAX], qw[RMAX];
 #pragma unroll
             for (uint32_t row = 0; row < (uint32_t)RMAX; ++row)
@@ -281,9 +304,6 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                 k4.x = key_of(med.x); k4.y = key_of(med.y); k4.z = key_of(med.z); k4.w = key_of(med.w);
             } else {
                 if (mask) {
-                    const float4 gs = ((const float4*)A.gsum)[t];
-                    float4 vv = ((const float4*)A.v)[t];
-                    uint4 vs = ((const uint4*)A.vstamp)[t];
                     if (mask & 1u) update_member(P, A, gs.x, vv.x, vs.x, vh.x);
                     if (mask & 2u) update_member(P, A, gs.y, vv.y, vs.y, vh.y);
                     if (mask & 4u) update_member(P, A, gs.z, vv.z, vs.z, vh.z);
