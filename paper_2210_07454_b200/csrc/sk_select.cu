@@ -285,13 +285,17 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
                 if (row < r) {
                     const uint2 h = hs[row * kGroupsPerUnit];
                     const uint32_t woff = (h.x ^ o) & ~3u;
-                    float4 cch = make_float4(0.f, 0.f, 0.f, 0.f);
-                    SK_GUARD(woff + 4u <= cw, kStatusWindow) cch = *(const float4*)(win + row * cw + woff);
-                    // coordinate l of the quad sits at element l xor p3 of the chunk; h.y is the group's sign (+-1.0f)
-                    if (h.x & 1u) { float u = cch.x; cch.x = cch.y; cch.y = u; u = cch.z; cch.z = cch.w; cch.w = u; }
-                    if (h.x & 2u) { float u = cch.x; cch.x = cch.z; cch.z = u; u = cch.y; cch.y = cch.w; cch.w = u; }
+                    // coordinate l of the quad sits at element l xor p3 of the chunk: bit 1 of p3 is taken by the
+                    // address (which 8-byte half is read first), bit 0 by a swap; h.y is the group's sign (+-1.0f)
+                    float2 c01 = make_float2(0.f, 0.f), c23 = c01;
+                    SK_GUARD(woff + 4u <= cw, kStatusWindow) {
+                        const float* chunk = win + row * cw + woff;
+                        c01 = *(const float2*)(chunk + (h.x & 2u));
+                        c23 = *(const float2*)(chunk + ((h.x & 2u) ^ 2u));
+                    }
+                    if (h.x & 1u) { float u = c01.x; c01.x = c01.y; c01.y = u; u = c23.x; c23.x = c23.y; c23.y = u; }
                     const float sg = __uint_as_float(h.y);
-                    qx[row] = sg * cch.x; qy[row] = sg * cch.y; qz[row] = sg * cch.z; qw[row] = sg * cch.w;
+                    qx[row] = sg * c01.x; qy[row] = sg * c01.y; qz[row] = sg * c23.x; qw[row] = sg * c23.y;
                 }
             float4 med;
             if constexpr (R > 0) {
