@@ -275,6 +275,8 @@ def main():
                     help="ga = gradient averaging (Algorithm 2, the headline path); pa = parameter averaging (Algorithm 1)")
     ap.add_argument("--window-lines", type=int, default=None, help="windowed hash family: lines per window (0 = plain)")
     ap.add_argument("--window-workers", type=int, default=0, help="workers per launch of the windowed sketch kernel")
+    ap.add_argument("--chained-launches", type=int, default=-1,
+                    help="0: launch the step's kernels without programmatic dependent launch (the default is chained)")
     ap.add_argument("--worker-sum", type=int, default=-1, help="1: the sketch kernel leaves the worker sum of a_t for the update of x")
     ap.add_argument("--worker-chunk", type=int, default=0)
     ap.add_argument("--sketch-ctas", type=int, default=0, help="CTAs per SM of the sketch kernel (0 = default)")
@@ -342,6 +344,8 @@ def main():
         opt.set_option("sketch_ctas_per_sm", args.sketch_ctas)
     if args.worker_sum >= 0:
         opt.set_option("worker_sum", args.worker_sum)
+    if args.chained_launches >= 0:
+        opt.set_option("chained_launches", args.chained_launches)
     # gradient buffers rotate so that no step finds its inputs in L2 (each set is far larger than L2 anyway)
     free_b, _ = torch.cuda.mem_get_info()
     set_bytes = gbytes * w.n * w.d

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 #include "sk_debug.cuh"
+#include "sk_chain.cuh"
 
 namespace sk {
 
@@ -26,6 +27,7 @@ struct Params {
     uint32_t* status;   // the handle's device status word (bits: sk_debug.cuh); nullptr = none
     uint32_t n_all;     // workers the means are taken over: n, or the total over all processes when the workers are
                         // partitioned (the handle then holds n of them)
+    uint32_t chain;     // host side only: the step's kernels are launched chained (sk_chain.cuh)
 };
 
 // Device-resident selection state (one per handle).
@@ -67,7 +69,7 @@ struct MomentArgs {
 int sm_count_of_device();
 // debug build only: one thread runs a bounds check with a false condition of the given kind (no access is made)
 int launch_debug_violation(const Params& P, uint32_t bit, cudaStream_t st);
-int launch_zero(void* p, uint64_t bytes, cudaStream_t st);
+int launch_zero(void* p, uint64_t bytes, cudaStream_t st, bool chain = false);
 int launch_fill_u32(uint32_t* p, uint64_t n, uint32_t value, cudaStream_t st);
 int launch_set_bits(const Params& P, const uint32_t* I, uint32_t count, uint32_t* bitmap, cudaStream_t st);
 int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,

@@ -220,6 +220,7 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
     uint2* hsh = (uint2*)(sh + kHistBins);                         // [2][r][32]: x = line*32 | perm, y = sign as +-1.0f
     float* win = (float*)(hsh + 2u * r * kGroupsPerUnit);          // [r][cw]: the panel's window of every row
     const uint32_t tid = threadIdx.x;
+    chain_release();
     for (uint32_t b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
     const uint32_t s_begin = (uint32_t)((uint64_t)units_total * blockIdx.x / gridDim.x);
     const uint32_t s_end = (uint32_t)((uint64_t)units_total * (blockIdx.x + 1) / gridDim.x);
@@ -253,6 +254,9 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
     if (s_begin < s_end) {
         walk.seek(s_begin);
         fill_hashes(walk.unit(), 0u);
+    }
+    chain_acquire();                // nothing above touches global memory
+    if (s_begin < s_end) {
         load_windows(walk.panel);
         mask_ahead = member_bits(walk.unit());
     }
@@ -340,6 +344,8 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
 __global__ void __launch_bounds__(1024) k_pick_bin(uint32_t k, uint32_t* hist, Select* sel, int level) {
     __shared__ uint32_t part[1024];
     constexpr uint32_t per = kHistBins / 1024;
+    chain_release();
+    chain_acquire();
     const uint32_t need = level == 0 ? k : sel->need;
     uint32_t mine[per];
     uint32_t s = 0;
@@ -452,7 +458,9 @@ k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, cons
     __shared__ uint32_t sh2[kHistBins];
     __shared__ uint32_t wb_out[kThreads / 32][kWarpBuf];
     __shared__ Cand wb_cand[kThreads / 32][kWarpBuf];
+    chain_release();
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh2[b] = 0;
+    chain_acquire();                // nothing above touches global memory
     __syncthreads();
     const uint32_t bin = sel->bin;
     const uint32_t thr_lo = bin << kHistShift;                  // first key of the threshold bin
@@ -534,6 +542,8 @@ k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, cons
 // ---- pass C over the candidates: first 24 key bits above the threshold -> emit, equal -> second list ----------
 __global__ void __launch_bounds__(kThreads)
 k_split_candidates(const __grid_constant__ Params P, Select* sel, const Cand* __restrict__ cand, uint32_t* I_out, Cand* cand2) {
+    chain_release();
+    chain_acquire();
     const uint32_t ncand = sel->cnt_cand;
     const uint32_t thr = (sel->bin << kHistBits) | sel->bin2;          // leading 24 bits of the threshold key
     const uint32_t trips = (ncand + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
@@ -564,6 +574,8 @@ __global__ void __launch_bounds__(1024) k_resolve(const __grid_constant__ Params
     __shared__ uint32_t hist[BINS];
     __shared__ uint32_t s_bin, s_need, s_done, s_pos;
     __shared__ uint32_t s_wtot[32];
+    chain_release();
+    chain_acquire();
     const uint32_t ncand = sel->cnt_cand2;
     uint32_t need = sel->need2;
     uint64_t prefix = 0;        // composite >> shift must equal prefix for an element to be still undecided
@@ -660,6 +672,8 @@ __global__ void __launch_bounds__(kThreads)
 k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const float* __restrict__ vhat,
         const float* __restrict__ e, const float* __restrict__ asum, float* x, uint32_t* bitmap) {
     // asum != nullptr: the sketch kernel left sum_w a^(w) (added in worker order) there, one gather instead of n
+    chain_release();
+    chain_acquire();
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
     if (q >= P.k) return;
     const uint32_t j = I[q];
@@ -756,8 +770,8 @@ int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum,
                  cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) && \
                 cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kfn, kThreads, smem) == cudaSuccess && nb >= 1) { \
                 const uint64_t cap = (uint64_t)sm_count * nb;                                                        \
-                kfn<<<(int)(units_total < cap ? units_total : cap), kThreads, smem, st>>>(P, A, sum, keys, hist,     \
-                                                                                          units_total, tbig, rem);   \
+                launch_kernel(P.chain != 0, kfn, (int)(units_total < cap ? units_total : cap), kThreads, smem, st,   \
+                              P, A, sum, keys, hist, units_total, tbig, rem);                                        \
                 return 1;                                                                                            \
             }                                                                                                        \
             cudaGetLastError();                                                                                      \
@@ -776,7 +790,7 @@ int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum,
 }
 
 int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cudaStream_t st) {
-    k_pick_bin<<<1, 1024, 0, st>>>(P.k, hist, sel, level);
+    launch_kernel(P.chain != 0, k_pick_bin, 1, 1024, 0, st, P.k, hist, sel, level);
     return 1;
 }
 
@@ -784,11 +798,12 @@ int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, 
                 uint32_t* hist2, int sm_count, cudaStream_t st) {
     if (P.d % 4 == 0 && !idx_map) {
         auto kfn = k_emit<true>;
-        kfn<<<grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P, keys, nullptr, sel, I_out,
-                                                                                                   cand, hist2);
+        launch_kernel(P.chain != 0, kfn, grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P,
+                      keys, (const uint32_t*)nullptr, sel, I_out, cand, hist2);
     } else {
         auto kfn = k_emit<false>;
-        kfn<<<grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P, keys, idx_map, sel, I_out, cand, hist2);
+        launch_kernel(P.chain != 0, kfn, grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P, keys, idx_map,
+                      sel, I_out, cand, hist2);
     }
     return 1;
 }
@@ -802,15 +817,16 @@ int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const 
 
 int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
                   int sm_count, cudaStream_t st) {
-    k_pick_bin<<<1, 1024, 0, st>>>(P.k, hist2, sel, 1);
-    k_split_candidates<<<sm_count, kThreads, 0, st>>>(P, sel, cand, I_out, cand2);
-    k_resolve<<<1, 1024, 0, st>>>(P, sel, cand2, I_out);
+    const bool chain = P.chain != 0;
+    launch_kernel(chain, k_pick_bin, 1, 1024, 0, st, P.k, hist2, sel, 1);
+    launch_kernel(chain, k_split_candidates, sm_count, kThreads, 0, st, P, sel, cand, I_out, cand2);
+    launch_kernel(chain, k_resolve, 1, 1024, 0, st, P, sel, cand2, I_out);
     return 3;
 }
 
 int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, const float* asum, float* x,
                  uint32_t* bitmap, cudaStream_t st) {
-    k_apply<<<(P.k + kThreads - 1) / kThreads, kThreads, 0, st>>>(P, I, vhat, e, asum, x, bitmap);
+    launch_kernel(P.chain != 0, k_apply, (P.k + kThreads - 1) / kThreads, kThreads, 0, st, P, I, vhat, e, asum, x, bitmap);
     return 1;
 }
 

@@ -23,6 +23,8 @@ __device__ __forceinline__ void sketch_quad(const Params& P, float* table, uint3
 }
 
 __global__ void __launch_bounds__(kThreads) k_zero(float4* p, uint64_t n4) {
+    chain_release();
+    chain_acquire();
     const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
     for (uint64_t t = blockIdx.x * (uint64_t)kThreads + threadIdx.x; t < n4; t += (uint64_t)gridDim.x * kThreads)
         p[t] = z;
@@ -264,6 +266,8 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
 // workers partitioned over processes this is the process's share of the mean.
 __global__ void __launch_bounds__(kThreads)
 k_sum_tables(const __grid_constant__ Params P, const float4* __restrict__ tables, float4* sum) {
+    chain_release();
+    chain_acquire();
     const uint32_t q4 = (P.r * P.cs) >> 2;
     const float fn = (float)P.n_all;
     for (uint32_t t = blockIdx.x * kThreads + threadIdx.x; t < q4; t += gridDim.x * kThreads) {
@@ -316,8 +320,8 @@ int launch_debug_violation(const Params& P, uint32_t bit, cudaStream_t st) {
 #endif
 }
 
-int launch_zero(void* p, uint64_t bytes, cudaStream_t st) {   // bytes must be a multiple of 16
-    k_zero<<<grid_for(bytes / 16, sm_count_of_device(), 8), kThreads, 0, st>>>((float4*)p, bytes / 16);
+int launch_zero(void* p, uint64_t bytes, cudaStream_t st, bool chain) {   // bytes must be a multiple of 16
+    launch_kernel(chain, k_zero, grid_for(bytes / 16, sm_count_of_device(), 8), kThreads, 0, st, (float4*)p, bytes / 16);
     return 1;
 }
 
@@ -371,7 +375,8 @@ int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint
 }
 
 int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStream_t st) {
-    k_sum_tables<<<grid_for((P.r * P.cs) >> 2, sm_count_of_device(), 8), kThreads, 0, st>>>(P, (const float4*)tables, (float4*)sum);
+    launch_kernel(P.chain != 0, k_sum_tables, grid_for((P.r * P.cs) >> 2, sm_count_of_device(), 8), kThreads, 0, st, P,
+                  (const float4*)tables, (float4*)sum);
     return 1;
 }
 

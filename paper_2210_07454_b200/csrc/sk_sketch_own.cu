@@ -232,7 +232,8 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
     const uint32_t nthreads = blockDim.x;
     const uint32_t s_begin = s_lo + (uint32_t)((uint64_t)(s_hi - s_lo) * blockIdx.x / gridDim.x);
     const uint32_t s_end = s_lo + (uint32_t)((uint64_t)(s_hi - s_lo) * (blockIdx.x + 1) / gridDim.x);
-    if (s_begin >= s_end) return;                                  // the whole block leaves together
+    chain_release();
+    if (s_begin >= s_end) { chain_acquire(); return; }             // the whole block leaves together
 
     const uint32_t d4 = P.d >> 2;
     const float b1 = P.beta1, omb1 = 1.0f - P.beta1, rho = P.rho;
@@ -266,6 +267,7 @@ k_moment_sketch_own(const __grid_constant__ Params P, const __grid_constant__ Mo
     walk.seek(s_begin);
     for (uint32_t q = tid; q < nw * r * cw / 4u; q += nthreads) ((float4*)win)[q] = zero4;
     fill_hashes(walk.unit(), 0u);
+    chain_acquire();                // nothing above touches global memory
     // ring of two chunks in flight per lane
     float4 G0, M0, E0, G1, M1, E1;
     {
@@ -369,8 +371,8 @@ inline size_t own_smem(const Params& P, uint32_t nw, uint32_t stage_rows, bool a
 
 // grid and shared-memory set-up common to both forms; `units` = length of the unit sequence the launch enumerates
 template <typename K, typename... Extra>
-int launch_own_kernel(K kfn, size_t smem, const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, uint32_t units,
-                      int sm_count, cudaStream_t st, Extra... extra) {
+int launch_own_kernel(bool chain, K kfn, size_t smem, const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw,
+                      uint32_t units, int sm_count, cudaStream_t st, Extra... extra) {
     if (units == 0) return 0;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
@@ -388,13 +390,13 @@ int launch_own_kernel(K kfn, size_t smem, const Params& P, const MomentArgs& A, 
     const uint32_t rem = units - (tbig - 1u) * P.win_panels;
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const int grid = (int)(units < cap ? units : cap);
-    kfn<<<grid, threads, smem, st>>>(P, A, w0, nw, 0u, units, tbig, rem, extra...);
+    launch_kernel(chain, kfn, grid, threads, smem, st, P, A, w0, nw, 0u, units, tbig, rem, extra...);
     return 1;
 }
 
 int launch_own_any(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, uint32_t units, uint32_t single,
                    int sm_count, cudaStream_t st) {
-    return launch_own_kernel(k_moment_sketch_own_any<0>, own_smem(P, nw, P.r, A.asum != nullptr), P, A, w0, nw, units,
+    return launch_own_kernel(false, k_moment_sketch_own_any<0>, own_smem(P, nw, P.r, A.asum != nullptr), P, A, w0, nw, units,
                              sm_count, st, single);
 }
 
@@ -405,11 +407,11 @@ int launch_own(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, i
     const size_t smem = own_smem(P, nw, R + 3, A.asum != nullptr);
     int l;
     if (A.grad_bf16)
-        l = A.asum ? launch_own_kernel(k_moment_sketch_own<R, true, true>, smem, P, A, w0, nw, units_full, sm_count, st)
-                   : launch_own_kernel(k_moment_sketch_own<R, false, true>, smem, P, A, w0, nw, units_full, sm_count, st);
+        l = A.asum ? launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, true, true>, smem, P, A, w0, nw, units_full, sm_count, st)
+                   : launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, false, true>, smem, P, A, w0, nw, units_full, sm_count, st);
     else
-        l = A.asum ? launch_own_kernel(k_moment_sketch_own<R, true, false>, smem, P, A, w0, nw, units_full, sm_count, st)
-                   : launch_own_kernel(k_moment_sketch_own<R, false, false>, smem, P, A, w0, nw, units_full, sm_count, st);
+        l = A.asum ? launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, true, false>, smem, P, A, w0, nw, units_full, sm_count, st)
+                   : launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, false, false>, smem, P, A, w0, nw, units_full, sm_count, st);
     if (l < 0) return l;
     if (units_total > units_full) {
         const int l2 = launch_own_any(P, A, w0, nw, 1u, units_full, sm_count, st);
