@@ -33,12 +33,12 @@ DEFAULT_WORKLOAD = "C3"      # d = 25.6M: the size the headline metric is quoted
 # proportion to n*d, so the capture (C3 at half size, see profiles/) is scaled to the timed launch.
 NCU_TRAFFIC = {
     # shared-memory ownership kernel (windowed hash family, the default path)
-    # capture: 1.2653 GB read + 0.8009 GB written for 1.024e8 worker-coordinates (profiles/c3_half_moment_sketch_own_ncu_full.md)
-    "k_moment_sketch_own": {"file": "sk_sketch_own.cu", "sha256": "8cebeb0a9bfe70b1be8a44467615503b2c7a00a303a9c2c2893eb357493ebc7e",
-                            "bytes_per_worker_coord": 20.18},
-    # L2-reduction kernel (plain hash family): 1.2539 GB read + 0.7941 GB written for 1.024e8 worker-coordinates
-    "k_moment_sketch_v4": {"file": "sk_sketch.cu", "sha256": "0bdcf8570d0f285945aa41d187337492869ba658f80dc563b760b74395264035",
-                           "bytes_per_worker_coord": 20.00},
+    # capture: 1.2653 GB read + 0.8005 GB written for 1.024e8 worker-coordinates (profiles/c3_half_moment_sketch_own_ncu_full.md)
+    "k_moment_sketch_own": {"file": "sk_sketch_own.cu", "sha256": "943a8f79d4234ea88447d157741e7beb5e9bf7c32ab37ea428bc7c65e07cc04c",
+                            "bytes_per_worker_coord": 20.17},
+    # L2-reduction kernel (plain hash family): 1.2540 GB read + 0.7948 GB written for 1.024e8 worker-coordinates
+    "k_moment_sketch_v4": {"file": "sk_sketch.cu", "sha256": "22a40f26423a95e6b6fa606c5e4a3e3e111270585219b1883d76157e2977a1c0",
+                           "bytes_per_worker_coord": 20.01},
 }
 
 

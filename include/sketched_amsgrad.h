@@ -179,6 +179,11 @@ int sk_debug_check(sk_state* state, uint32_t kind);
  *   "worker_chunk" workers whose tables are accumulated concurrently by the sketch kernel (0 = automatic,
  *                  sized so that the concurrently updated tables stay resident in L2).
  *   "sketch_ctas_per_sm" grid size of the plain sketch kernel in blocks per SM (default 64: one tile per block).
+ *   "chained_launches" 1 (default): the kernels of a step are launched with the programmatic-serialization
+ *                  attribute: each may become resident while its predecessor in the stream still runs, does its
+ *                  shared-memory set-up, and waits for the predecessor's completion before it touches global
+ *                  memory.  Results do not depend on it; 0 launches them plainly (values 2..511 chain only some
+ *                  kinds of launch: a diagnostic mask, see csrc/sk_chain.cuh).  Any time between steps.
  *   "timing"       1 = record CUDA events around each stage (see sk_get_timing); 0 = off (default). */
 int sk_set_option(sk_state* state, const char* key, int64_t value);
 /* Also readable: "I_count" (entries "I" currently holds: 0 before the first step, else k unless sk_set installed

@@ -176,7 +176,7 @@ int phase_local(sk_state* s, const void* grads, float* x1, uint32_t wbeg = 0, ui
         const uint32_t nw = std::min(wc, wend - w0);
         if (!s->sum_sketch) {
             StageTimer tm(s, 0);
-            tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats * 4, st, P.chain != 0));
+            tm.done(sk::launch_zero(s->tables + (uint64_t)w0 * tfloats, (uint64_t)nw * tfloats * 4, st, (P.chain & sk::kChainZero) != 0));
         }
         StageTimer tm(s, 2);     // moments + sketch; also leaves the gradient sums on I_{t-1} in gsum
         if (windowed) {
@@ -267,7 +267,7 @@ int phase_finish(sk_state* s, const float* x2, float* x) {
     }
     {
         StageTimer tm(s, 7);     // the bitmap of I_{t-1} has served its purpose: clear it, then apply marks I_t
-        int l = sk::launch_zero(s->bitmap, s->bitmap_bytes, st, P.chain != 0);
+        int l = sk::launch_zero(s->bitmap, s->bitmap_bytes, st, (P.chain & sk::kChainZero) != 0);
         l += sk::launch_apply(P, s->I, vhat, s->e, asum, x, s->bitmap, st);
         tm.done(l);
     }
@@ -343,7 +343,7 @@ sk_state* sk_create(uint64_t d, uint32_t n, uint32_t r, uint32_t c, uint64_t k, 
     P.d = (uint32_t)d; P.n = n; P.n_all = n; P.r = r; P.c = c; P.k = (uint32_t)k;
     P.cs = (c + 31u) / 32u * 32u;
     P.beta1 = beta1; P.beta2 = beta2; P.lr = lr; P.rho = 1.0f;
-    P.chain = 1;                     // the step's kernels are launched chained (option "chained_launches")
+    P.chain = sk::kChainAll;                     // the step's kernels are launched chained (option "chained_launches")
     s->lr_prev = lr;
     uint32_t lg = 5;
     while ((1u << lg) > c) --lg;
@@ -704,8 +704,8 @@ int sk_set_option(sk_state* s, const char* key, int64_t value) {
         return SK_OK;
     }
     if (!strcmp(key, "chained_launches")) {
-        if (value != 0 && value != 1) return fail(SK_EINVAL, "chained_launches must be 0 or 1");
-        s->P.chain = (uint32_t)value;
+        if (value < 0 || value > (int64_t)sk::kChainAll) return fail(SK_EINVAL, "chained_launches must be 0, 1 or a mask below 512");
+        s->P.chain = value == 1 ? sk::kChainAll : (uint32_t)value;
         return SK_OK;
     }
     if (!strcmp(key, "timing")) {
@@ -731,7 +731,7 @@ int sk_get_option(const sk_state* s, const char* key, int64_t* value) {
     else if (!strcmp(key, "grads_bf16")) *value = s->grads_bf16;
     else if (!strcmp(key, "worker_chunk")) *value = chunk_of(s);
     else if (!strcmp(key, "timing")) *value = s->timing;
-    else if (!strcmp(key, "chained_launches")) *value = s->P.chain;
+    else if (!strcmp(key, "chained_launches")) *value = s->P.chain == sk::kChainAll ? 1 : s->P.chain;
     else if (!strcmp(key, "sketch_ctas_per_sm")) *value = s->sketch_ctas_per_sm;
     else if (!strcmp(key, "I_count")) *value = s->k_prev;
     else if (!strcmp(key, "vectorised")) *value = (s->P.d % 4 == 0) && s->P.log2g >= 2;

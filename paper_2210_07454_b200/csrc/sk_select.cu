@@ -141,6 +141,7 @@ k_unsketch_hist(const __grid_constant__ Params P, const __grid_constant__ Moment
                 uint32_t* keys, uint32_t* hist) {
     __shared__ uint32_t sh[kHistBins];
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh[b] = 0;
+    chain_acquire();                // nothing above touches global memory
     __syncthreads();
     const uint32_t items = VEC ? (P.d >> 2) : P.d;
     const uint32_t trips = (items + gridDim.x * kThreads - 1) / (gridDim.x * kThreads);
@@ -344,7 +345,6 @@ k_unsketch_hist_win(const __grid_constant__ Params P, const __grid_constant__ Mo
 __global__ void __launch_bounds__(1024) k_pick_bin(uint32_t k, uint32_t* hist, Select* sel, int level) {
     __shared__ uint32_t part[1024];
     constexpr uint32_t per = kHistBins / 1024;
-    chain_release();
     chain_acquire();
     const uint32_t need = level == 0 ? k : sel->need;
     uint32_t mine[per];
@@ -542,7 +542,6 @@ k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, cons
 // ---- pass C over the candidates: first 24 key bits above the threshold -> emit, equal -> second list ----------
 __global__ void __launch_bounds__(kThreads)
 k_split_candidates(const __grid_constant__ Params P, Select* sel, const Cand* __restrict__ cand, uint32_t* I_out, Cand* cand2) {
-    chain_release();
     chain_acquire();
     const uint32_t ncand = sel->cnt_cand;
     const uint32_t thr = (sel->bin << kHistBits) | sel->bin2;          // leading 24 bits of the threshold key
@@ -574,7 +573,6 @@ __global__ void __launch_bounds__(1024) k_resolve(const __grid_constant__ Params
     __shared__ uint32_t hist[BINS];
     __shared__ uint32_t s_bin, s_need, s_done, s_pos;
     __shared__ uint32_t s_wtot[32];
-    chain_release();
     chain_acquire();
     const uint32_t ncand = sel->cnt_cand2;
     uint32_t need = sel->need2;
@@ -649,6 +647,7 @@ k_exact_keys(const __grid_constant__ Params P, const uint32_t* __restrict__ C, u
              uint32_t* keys2, uint32_t* hist) {
     __shared__ uint32_t sh[kHistBins];
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh[b] = 0;
+    chain_acquire();                // nothing above touches global memory
     __syncthreads();
     for (uint32_t q = blockIdx.x * kThreads + threadIdx.x; q < count; q += gridDim.x * kThreads) {
         const uint32_t j = C[q];
@@ -672,7 +671,6 @@ __global__ void __launch_bounds__(kThreads)
 k_apply(const __grid_constant__ Params P, const uint32_t* __restrict__ I, const float* __restrict__ vhat,
         const float* __restrict__ e, const float* __restrict__ asum, float* x, uint32_t* bitmap) {
     // asum != nullptr: the sketch kernel left sum_w a^(w) (added in worker order) there, one gather instead of n
-    chain_release();
     chain_acquire();
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;
     if (q >= P.k) return;
@@ -735,7 +733,7 @@ int resident_per_sm(K kernel, int fallback) {
 
 #define SK_ROWS_CASE(KERNEL, RR, ...)                                                                      \
     { auto kfn = KERNEL<RR, true>;                                                                         \
-      kfn<<<grid_for(items, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(__VA_ARGS__); } break;
+      launch_kernel((P.chain & kChainKeys) != 0, kfn, grid_for(items, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, __VA_ARGS__); } break;
 #define SK_ROWS_SWITCH(KERNEL, ...)                                                                        \
     switch (P.r) {                                                                                         \
         case 1: SK_ROWS_CASE(KERNEL, 1, __VA_ARGS__)                                                       \
@@ -754,7 +752,7 @@ int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum,
                          bool vec, int sm_count, cudaStream_t st) {
     if (!vec) {
         auto kfn = k_unsketch_hist<0, false>;
-        kfn<<<grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st>>>(P, A, sum, keys, hist);
+        launch_kernel((P.chain & kChainKeys) != 0, kfn, grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P, A, sum, keys, hist);
         return 1;
     }
     if (P.win_cw != 0 && P.log2g == 5) {           // windowed family: shared-memory windows, panel-major walk
@@ -770,7 +768,7 @@ int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum,
                  cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) && \
                 cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kfn, kThreads, smem) == cudaSuccess && nb >= 1) { \
                 const uint64_t cap = (uint64_t)sm_count * nb;                                                        \
-                launch_kernel(P.chain != 0, kfn, (int)(units_total < cap ? units_total : cap), kThreads, smem, st,   \
+                launch_kernel((P.chain & kChainKeys) != 0, kfn, (int)(units_total < cap ? units_total : cap), kThreads, smem, st,   \
                               P, A, sum, keys, hist, units_total, tbig, rem);                                        \
                 return 1;                                                                                            \
             }                                                                                                        \
@@ -790,7 +788,7 @@ int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum,
 }
 
 int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cudaStream_t st) {
-    launch_kernel(P.chain != 0, k_pick_bin, 1, 1024, 0, st, P.k, hist, sel, level);
+    launch_kernel((P.chain & kChainPick) != 0, k_pick_bin, 1, 1024, 0, st, P.k, hist, sel, level);
     return 1;
 }
 
@@ -798,11 +796,11 @@ int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, 
                 uint32_t* hist2, int sm_count, cudaStream_t st) {
     if (P.d % 4 == 0 && !idx_map) {
         auto kfn = k_emit<true>;
-        launch_kernel(P.chain != 0, kfn, grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P,
+        launch_kernel((P.chain & kChainEmit) != 0, kfn, grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P,
                       keys, (const uint32_t*)nullptr, sel, I_out, cand, hist2);
     } else {
         auto kfn = k_emit<false>;
-        launch_kernel(P.chain != 0, kfn, grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P, keys, idx_map,
+        launch_kernel((P.chain & kChainEmit) != 0, kfn, grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P, keys, idx_map,
                       sel, I_out, cand, hist2);
     }
     return 1;
@@ -810,14 +808,14 @@ int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, 
 
 int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const float* vhat, const float* e,
                       const float* asum, uint32_t* keys2, uint32_t* hist, int sm_count, cudaStream_t st) {
-    k_exact_keys<<<grid_for(count, sm_count, resident_per_sm(k_exact_keys, 4)), kThreads, 0, st>>>(P, C, count, vhat, e, asum,
-                                                                                                  keys2, hist);
+    launch_kernel((P.chain & kChainExact) != 0, k_exact_keys, grid_for(count, sm_count, resident_per_sm(k_exact_keys, 4)), kThreads, 0, st, P, C,
+                  count, vhat, e, asum, keys2, hist);
     return 1;
 }
 
 int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, uint32_t* hist2, uint32_t* I_out,
                   int sm_count, cudaStream_t st) {
-    const bool chain = P.chain != 0;
+    const bool chain = (P.chain & kChainRefine) != 0;
     launch_kernel(chain, k_pick_bin, 1, 1024, 0, st, P.k, hist2, sel, 1);
     launch_kernel(chain, k_split_candidates, sm_count, kThreads, 0, st, P, sel, cand, I_out, cand2);
     launch_kernel(chain, k_resolve, 1, 1024, 0, st, P, sel, cand2, I_out);
@@ -826,7 +824,7 @@ int launch_refine(const Params& P, Select* sel, const Cand* cand, Cand* cand2, u
 
 int launch_apply(const Params& P, const uint32_t* I, const float* vhat, const float* e, const float* asum, float* x,
                  uint32_t* bitmap, cudaStream_t st) {
-    launch_kernel(P.chain != 0, k_apply, (P.k + kThreads - 1) / kThreads, kThreads, 0, st, P, I, vhat, e, asum, x, bitmap);
+    launch_kernel((P.chain & kChainApply) != 0, k_apply, (P.k + kThreads - 1) / kThreads, kThreads, 0, st, P, I, vhat, e, asum, x, bitmap);
     return 1;
 }
 

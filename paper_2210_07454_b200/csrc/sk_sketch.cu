@@ -23,7 +23,6 @@ __device__ __forceinline__ void sketch_quad(const Params& P, float* table, uint3
 }
 
 __global__ void __launch_bounds__(kThreads) k_zero(float4* p, uint64_t n4) {
-    chain_release();
     chain_acquire();
     const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
     for (uint64_t t = blockIdx.x * (uint64_t)kThreads + threadIdx.x; t < n4; t += (uint64_t)gridDim.x * kThreads)
@@ -94,6 +93,7 @@ __device__ __forceinline__ void sketch_of_sum(const Params& P, const MomentArgs&
 template <int R>
 __global__ void __launch_bounds__(kThreads, 3)
 k_moment_sketch_v4(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
+    chain_acquire();
     float4* m = (float4*)A.m;
     float4* e = (float4*)A.e;
     const uint32_t r = R > 0 ? (uint32_t)R : P.r;
@@ -177,6 +177,7 @@ __device__ __forceinline__ void pa_moment(float b1, float omb1, float b2, float 
 template <int R>
 __global__ void __launch_bounds__(kThreads, 3)
 k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
+    chain_acquire();
     float4* m = (float4*)A.m;
     float4* e = (float4*)A.e;
     float4* vw = (float4*)A.vw;
@@ -220,6 +221,7 @@ k_moment_sketch_pa_v4(const __grid_constant__ Params P, const __grid_constant__ 
 // Scalar form: any d, any alignment, any group size.  One thread per coordinate.
 __global__ void __launch_bounds__(kThreads)
 k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__ MomentArgs A, uint32_t w0, uint32_t nw) {
+    chain_acquire();
     const float b1 = P.beta1, omb1 = 1.0f - P.beta1, rho = P.rho;
     const uint64_t tstride = (uint64_t)P.r * P.cs;
     for (uint32_t j = blockIdx.x * kThreads + threadIdx.x; j < P.d; j += gridDim.x * kThreads) {
@@ -266,7 +268,6 @@ k_moment_sketch_scalar(const __grid_constant__ Params P, const __grid_constant__
 // workers partitioned over processes this is the process's share of the mean.
 __global__ void __launch_bounds__(kThreads)
 k_sum_tables(const __grid_constant__ Params P, const float4* __restrict__ tables, float4* sum) {
-    chain_release();
     chain_acquire();
     const uint32_t q4 = (P.r * P.cs) >> 2;
     const float fn = (float)P.n_all;
@@ -351,31 +352,32 @@ int launch_masked_copy(const Params& P, const float* e, const uint32_t* bitmap, 
 
 int launch_moment_sketch(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, bool vec, int sm_count,
                          cudaStream_t st) {
+    const bool chain = (P.chain & kChainSketch) != 0;
     if (!vec) {
-        k_moment_sketch_scalar<<<grid_for(P.d, sm_count, 1), kThreads, 0, st>>>(P, A, w0, nw);
+        launch_kernel(chain, k_moment_sketch_scalar, grid_for(P.d, sm_count, 1), kThreads, 0, st, P, A, w0, nw);
         return 1;
     }
     const int grid = grid_for(P.d >> 2, sm_count, 1);    // the caller passes SMs x CTAs per SM
     if (A.variant == 1) {
-#define SK_CASE(RR) case RR: k_moment_sketch_pa_v4<RR><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
+#define SK_CASE(RR) case RR: launch_kernel(chain, k_moment_sketch_pa_v4<RR>, grid, kThreads, 0, st, P, A, w0, nw); break;
         switch (P.r) {
             SK_CASE(1) SK_CASE(2) SK_CASE(3) SK_CASE(4) SK_CASE(5) SK_CASE(6) SK_CASE(7) SK_CASE(8) SK_CASE(10)
-            default: k_moment_sketch_pa_v4<0><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
+            default: launch_kernel(chain, k_moment_sketch_pa_v4<0>, grid, kThreads, 0, st, P, A, w0, nw); break;
         }
 #undef SK_CASE
         return 1;
     }
-#define SK_CASE(RR) case RR: k_moment_sketch_v4<RR><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
+#define SK_CASE(RR) case RR: launch_kernel(chain, k_moment_sketch_v4<RR>, grid, kThreads, 0, st, P, A, w0, nw); break;
     switch (P.r) {
         SK_CASE(1) SK_CASE(2) SK_CASE(3) SK_CASE(4) SK_CASE(5) SK_CASE(6) SK_CASE(7) SK_CASE(8) SK_CASE(10)
-        default: k_moment_sketch_v4<0><<<grid, kThreads, 0, st>>>(P, A, w0, nw); break;
+        default: launch_kernel(chain, k_moment_sketch_v4<0>, grid, kThreads, 0, st, P, A, w0, nw); break;
     }
 #undef SK_CASE
     return 1;
 }
 
 int launch_sum_tables(const Params& P, const float* tables, float* sum, cudaStream_t st) {
-    launch_kernel(P.chain != 0, k_sum_tables, grid_for((P.r * P.cs) >> 2, sm_count_of_device(), 8), kThreads, 0, st, P,
+    launch_kernel((P.chain & kChainSum) != 0, k_sum_tables, grid_for((P.r * P.cs) >> 2, sm_count_of_device(), 8), kThreads, 0, st, P,
                   (const float4*)tables, (float4*)sum);
     return 1;
 }

@@ -77,6 +77,7 @@ k_moment_sketch_own_any(const __grid_constant__ Params P, const __grid_constant_
     const uint32_t nthreads = blockDim.x;
     const uint32_t s_begin = s_lo + (uint32_t)((uint64_t)(s_hi - s_lo) * blockIdx.x / gridDim.x);
     const uint32_t s_end = s_lo + (uint32_t)((uint64_t)(s_hi - s_lo) * (blockIdx.x + 1) / gridDim.x);
+    chain_acquire();
     if (s_begin >= s_end) return;                                  // the whole block leaves together
 
     float4* m = (float4*)A.m;
@@ -396,7 +397,7 @@ int launch_own_kernel(bool chain, K kfn, size_t smem, const Params& P, const Mom
 
 int launch_own_any(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, uint32_t units, uint32_t single,
                    int sm_count, cudaStream_t st) {
-    return launch_own_kernel(false, k_moment_sketch_own_any<0>, own_smem(P, nw, P.r, A.asum != nullptr), P, A, w0, nw, units,
+    return launch_own_kernel((P.chain & kChainSketch) != 0, k_moment_sketch_own_any<0>, own_smem(P, nw, P.r, A.asum != nullptr), P, A, w0, nw, units,
                              sm_count, st, single);
 }
 
@@ -407,11 +408,11 @@ int launch_own(const Params& P, const MomentArgs& A, uint32_t w0, uint32_t nw, i
     const size_t smem = own_smem(P, nw, R + 3, A.asum != nullptr);
     int l;
     if (A.grad_bf16)
-        l = A.asum ? launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, true, true>, smem, P, A, w0, nw, units_full, sm_count, st)
-                   : launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, false, true>, smem, P, A, w0, nw, units_full, sm_count, st);
+        l = A.asum ? launch_own_kernel((P.chain & kChainSketch) != 0, k_moment_sketch_own<R, true, true>, smem, P, A, w0, nw, units_full, sm_count, st)
+                   : launch_own_kernel((P.chain & kChainSketch) != 0, k_moment_sketch_own<R, false, true>, smem, P, A, w0, nw, units_full, sm_count, st);
     else
-        l = A.asum ? launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, true, false>, smem, P, A, w0, nw, units_full, sm_count, st)
-                   : launch_own_kernel(P.chain != 0, k_moment_sketch_own<R, false, false>, smem, P, A, w0, nw, units_full, sm_count, st);
+        l = A.asum ? launch_own_kernel((P.chain & kChainSketch) != 0, k_moment_sketch_own<R, true, false>, smem, P, A, w0, nw, units_full, sm_count, st)
+                   : launch_own_kernel((P.chain & kChainSketch) != 0, k_moment_sketch_own<R, false, false>, smem, P, A, w0, nw, units_full, sm_count, st);
     if (l < 0) return l;
     if (units_total > units_full) {
         const int l2 = launch_own_any(P, A, w0, nw, 1u, units_full, sm_count, st);

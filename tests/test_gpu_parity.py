@@ -510,6 +510,41 @@ def test_integer_inputs_are_bit_exact():
     assert np.array_equal(x.cpu().numpy(), x_ref)
 
 
+@pytest.mark.parametrize("kw", [dict(), dict(window_lines=0), dict(variant="pa"), dict(P=4), dict(window_lines=0, P=2)],
+                         ids=["default", "plain_family", "parameter_averaging", "second_round", "plain_second_round"])
+def test_chained_and_plain_launches_give_the_same_bits(kw):
+    # The step's kernels are launched chained (each may become resident while its predecessor still runs and waits
+    # for it before touching global memory).  With integer gradients every sum is exact whatever the order of the
+    # atomic adds, so three steps with and without chaining must agree bit for bit; a kernel that read or wrote
+    # ahead of its predecessor would not.
+    d, n, r, c, k = 150_016, 4, 5, 4096, 800
+    b = _binding()
+    gen = torch.Generator(device="cuda").manual_seed(23)
+    grads = [torch.randint(-8, 9, (n, d), generator=gen, device="cuda").float() for _ in range(3)]
+    results = []
+    for chained in (1, 0):
+        gpu = b.SketchedAMSGrad(d, n, r, c, k, seed=4, lr=0.5, beta1=0.0, beta2=0.5, eps=1.0, **kw)
+        gpu.set_option("chained_launches", chained)
+        assert gpu.get_option("chained_launches") == chained
+        x = torch.zeros(d, device="cuda")
+        for g in grads:
+            gpu.step(g, x)
+        gpu.sync()
+        results.append({f: gpu.get(f) for f in ("tables", "sum", "m", "e", "I", "keys")} | {"x": x.cpu().numpy()})
+        if kw.get("variant") != "pa":
+            results[-1]["v"] = gpu.get("v")
+            results[-1]["vhat"] = gpu.get("vhat")
+    exact = kw.get("variant") != "pa"      # Algorithm 1 sketches m / sqrt(vhat): not integers, the add order shows
+    for f, a in results[0].items():
+        b_ = results[1][f]
+        if exact:
+            if f == "I":
+                a, b_ = np.sort(a), np.sort(b_)
+            assert np.array_equal(a, b_), f
+        elif f in ("tables", "sum", "m"):
+            assert np.allclose(a, b_, rtol=1e-5, atol=1e-5), f
+
+
 def test_all_zero_gradients_select_lowest_indices():
     d, n, r, c, k = 50_000, 2, 5, 1024, 77
     b = _binding()
