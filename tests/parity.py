@@ -29,12 +29,22 @@ def close(got, ref, what, groups_axis=None, rel=REL, scale=None):
                              f"got {got[q]!r} ref {ref[q]!r} err {err[q]:.3e} bound {np.broadcast_to(bound, err.shape)[q]:.3e}")
 
 
-def est_scale(S_ref, vhat_ref):
+def est_scale(S_ref, vhat_ref, tables_ref=None):
     """An estimate is one bucket of the aggregated sketch divided by sqrt(vhat): it inherits the bucket's absolute
-    error bound, rel * RMS(row), magnified by vhat^{-1/2}."""
+    error bound, rel * RMS(row), magnified by vhat^{-1/2}.  The aggregated bucket is the mean of the n workers'
+    buckets, each formed by fp32 additions whose rounding is relative to THAT worker's partial sums: where the
+    workers cancel (independent noise: the aggregate's RMS is 1/sqrt(n) of a worker's) the absolute error stays at
+    the workers' scale, so the row scale is the larger of the aggregate's RMS and the workers' (tables_ref given)."""
     S = np.asarray(S_ref, np.float64)
     row_rms = np.sqrt(np.mean(S * S, axis=1)).max()
+    if tables_ref is not None:
+        row_rms = max(row_rms, worker_row_rms(tables_ref).max())
     return row_rms / np.sqrt(np.asarray(vhat_ref, np.float64))
+
+
+def worker_row_rms(tables_ref):
+    """RMS of every (worker, row) of the worker sketches, computed worker by worker in fp64: shape (n, r)."""
+    return np.stack([np.sqrt(np.mean(np.asarray(t, np.float64) ** 2, axis=1)) for t in tables_ref])
 
 
 LAST_INDEX_DIFFERENCE = {}     # what the last index_sets_agree call saw: {"what", "count", "worst_offset_in_bands"}
@@ -129,7 +139,10 @@ def compare_step(gpu, ora, x_gpu, x_ref, x_before, lr, check_tables=True, x_gpu_
     d, n, k = ora.d, ora.n, ora.k
     if check_tables:
         close(gpu.get("tables"), ora.field("tables"), "worker sketches", groups_axis=1)
-    close(gpu.get("sum"), ora.field("sum"), "aggregated sketch", groups_axis=0)
+    # the aggregate is the mean of the workers' buckets: its error scale is a worker's row, not its own (est_scale)
+    tables_ref = ora.field("tables")
+    close(gpu.get("sum"), ora.field("sum"), "aggregated sketch", groups_axis=0,
+          scale=worker_row_rms(tables_ref).max(axis=0)[:, None])
     if variant == "ga":
         # v and vhat are sums of non-negative terms: the bound is relative to each ELEMENT, not to the array's scale
         v_ref = ora.field("v")
@@ -139,11 +152,11 @@ def compare_step(gpu, ora, x_gpu, x_ref, x_before, lr, check_tables=True, x_gpu_
             bad = err > vb
             assert not bad.any(), (f"{name}: {bad.sum()} of {bad.size} elements outside the element-relative bound; "
                                    f"worst ratio {np.max(err / np.maximum(vb, 1e-300)):.3f}")
-        sc = est_scale(ora.field("sum"), ora.field("vhat"))
+        sc = est_scale(ora.field("sum"), ora.field("vhat"), tables_ref)
     else:                       # Algorithm 1: per-worker second moments (sums of non-negative terms: element-relative),
         np.testing.assert_allclose(gpu.get("vw"), ora.field("vw"), rtol=REL, atol=0)       # and a plain unsketch
         np.testing.assert_allclose(gpu.get("vhatw"), ora.field("vhatw"), rtol=REL, atol=0)
-        sc = est_scale(ora.field("sum"), np.ones(d, np.float32))
+        sc = est_scale(ora.field("sum"), np.ones(d, np.float32), tables_ref)
     est_ref = ora.field("est")
     close(gpu.get("est"), est_ref, "estimates", scale=sc)
     # the keys the selection actually ran on (vector medians, hardware reciprocal square root), not the export path
