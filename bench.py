@@ -284,7 +284,7 @@ def main():
     ap.add_argument("--ref-scale", type=int, default=0, help="reference arm: 1/SCALE size per step (0 = full size if it fits the time budget)")
     ap.add_argument("--reps", type=int, default=0,
                     help="repetitions of the --steps long timed loop, the median is reported; 0 = as many as fill about "
-                         "one second (at least 10, at most 400), so that the clock sampler sees the timed region")
+                         "half a second (at least 10, at most 400), so that the clock sampler sees the timed region")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the short C4 and C5 runs reported beside the headline")
     ap.add_argument("--scale", type=int, default=1, help="run the workload at 1/SCALE size (profiling captures)")
     ap.add_argument("--grad-sets", type=int, default=0, help="rotating gradient sets (0 = as many as fit, 2..4)")
@@ -390,7 +390,7 @@ def main():
         rep_ms.append(reduce_max(ev0.elapsed_time(ev1), world, dev))
         rep += 1
         if args.reps <= 0 and rep == 1:              # every rank derives the same count from the reduced time
-            reps = int(min(400, max(10, math.ceil(1000.0 / max(rep_ms[0], 1e-3)))))
+            reps = int(min(400, max(10, math.ceil(500.0 / max(rep_ms[0], 1e-3)))))
     clocks = sampler.stop(windows) if rank == 0 else None
     opt.sync()
     ms_total = statistics.median(rep_ms)

@@ -352,15 +352,27 @@ __global__ void __launch_bounds__(1024) k_pick_bin(uint32_t k, uint32_t* hist, S
     const uint32_t top = kHistBins - 1 - threadIdx.x * per;   // thread i owns `per` bins in descending order
 #pragma unroll
     for (uint32_t q = 0; q < per; ++q) { mine[q] = hist[top - q]; hist[top - q] = 0; s += mine[q]; }
-    part[threadIdx.x] = s;
-    __syncthreads();
-    for (uint32_t off = 1; off < 1024; off <<= 1) {
-        const uint32_t add = threadIdx.x >= off ? part[threadIdx.x - off] : 0;
-        __syncthreads();
-        part[threadIdx.x] += add;
-        __syncthreads();
+    // inclusive scan of the 1024 per-thread counts: inside each warp by shuffles, then over the 32 warp totals
+    const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
+    uint32_t incl = s;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= (uint32_t)off) incl += o;
     }
-    uint32_t above = part[threadIdx.x] - s;
+    if (lane == 31u) part[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+        uint32_t w = part[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, w, off);
+            if (lane >= (uint32_t)off) w += o;
+        }
+        part[32u + lane] = w;                                 // inclusive totals of warps 0..lane
+    }
+    __syncthreads();
+    uint32_t above = incl - s + (wid ? part[32u + wid - 1u] : 0u);
 #pragma unroll
     for (uint32_t q = 0; q < per; ++q) {
         if (above < need && above + mine[q] >= need) {
