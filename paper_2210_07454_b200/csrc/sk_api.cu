@@ -224,7 +224,10 @@ int phase_select(sk_state* s, const float* x1, float* x2) {
     uint32_t* list = s->cand_mult > 1 ? s->Ic : s->I;
     {
         StageTimer tm(s, 5);
-        tm.done(sk::launch_emit(Q, s->keys, nullptr, s->sel, list, s->cand, s->hist2, s->sm_count, st));
+        // the pass also clears the bitmap of I_{t-1}, which has served its purpose once the key pass is through:
+        // the update of x then marks I_t in it
+        tm.done(sk::launch_emit(Q, s->keys, nullptr, s->sel, list, s->cand, s->hist2, s->sm_count, st, s->bitmap,
+                                s->bitmap_bytes));
     }
     {
         StageTimer tm(s, 6);
@@ -266,10 +269,8 @@ int phase_finish(sk_state* s, const float* x2, float* x) {
         tm.done(l);
     }
     {
-        StageTimer tm(s, 7);     // the bitmap of I_{t-1} has served its purpose: clear it, then apply marks I_t
-        int l = sk::launch_zero(s->bitmap, s->bitmap_bytes, st, (P.chain & sk::kChainZero) != 0);
-        l += sk::launch_apply(P, s->I, vhat, s->e, asum, x, s->bitmap, st);
-        tm.done(l);
+        StageTimer tm(s, 7);     // apply marks I_t in the bitmap, which the emit pass of the selection cleared
+        tm.done(sk::launch_apply(P, s->I, vhat, s->e, asum, x, s->bitmap, st));
     }
     SK_CUDA(cudaGetLastError());
     std::swap(s->I, s->I_prev);      // I_prev now holds I_t

@@ -85,8 +85,9 @@ int launch_unsketch_hist(const Params& P, const MomentArgs& A, const float* sum,
                          bool vec, int sm_count, cudaStream_t st);
 int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cudaStream_t st);
 // selection runs over P.d keys for the P.k largest; idx_map != nullptr: key t belongs to coordinate idx_map[t]
+// clear / clear_bytes (a multiple of 16, or nullptr / 0): a buffer the pass also zeroes (the bitmap of I_{t-1})
 int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, Select* sel, uint32_t* I_out, Cand* cand,
-                uint32_t* hist2, int sm_count, cudaStream_t st);
+                uint32_t* hist2, int sm_count, cudaStream_t st, void* clear = nullptr, uint64_t clear_bytes = 0);
 // second round: exact values of `count` candidate coordinates as ranking keys, with their first-level histogram
 // asum != nullptr: sum_w a^(w) per coordinate is read from there instead of gathering e for every worker
 int launch_exact_keys(const Params& P, const uint32_t* C, uint32_t count, const float* vhat, const float* e,

@@ -463,7 +463,9 @@ __device__ __forceinline__ T* warp_reserve(const Params& P, T* buf, uint32_t& fi
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx_map, Select* sel,
-       uint32_t* I_out, Cand* cand, uint32_t* hist2) {
+       uint32_t* I_out, Cand* cand, uint32_t* hist2, uint4* clear, uint32_t clear_n4) {
+    // clear (may be nullptr): clear_n4 16-byte words that this pass also sets to zero -- the membership bitmap of
+    // I_{t-1}, which the key pass was the last to read and the update of x will mark with I_t
     // P.d keys, the P.k largest wanted: I_out holds P.k entries, the candidate list P.d
     const uint32_t d = P.d;
     // idx_map (scalar form only): keys[t] belongs to coordinate idx_map[t] instead of t (second round on a candidate list)
@@ -474,6 +476,9 @@ k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, cons
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kThreads) sh2[b] = 0;
     chain_acquire();                // nothing above touches global memory
     __syncthreads();
+    if (clear)
+        for (uint32_t t = blockIdx.x * kThreads + threadIdx.x; t < clear_n4; t += gridDim.x * kThreads)
+            clear[t] = make_uint4(0u, 0u, 0u, 0u);
     const uint32_t bin = sel->bin;
     const uint32_t thr_lo = bin << kHistShift;                  // first key of the threshold bin
     const uint32_t thr_hi = (bin + 1u) << kHistShift;           // first key above it (2^31 for the last bin: no key)
@@ -805,15 +810,17 @@ int launch_pick_bin(const Params& P, uint32_t* hist, Select* sel, int level, cud
 }
 
 int launch_emit(const Params& P, const uint32_t* keys, const uint32_t* idx_map, Select* sel, uint32_t* I_out, Cand* cand,
-                uint32_t* hist2, int sm_count, cudaStream_t st) {
+                uint32_t* hist2, int sm_count, cudaStream_t st, void* clear, uint64_t clear_bytes) {
+    uint4* c4 = (uint4*)clear;
+    const uint32_t n4 = (uint32_t)(clear_bytes / 16);
     if (P.d % 4 == 0 && !idx_map) {
         auto kfn = k_emit<true>;
         launch_kernel((P.chain & kChainEmit) != 0, kfn, grid_for((P.d >> 2) / 4 + 1, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P,
-                      keys, (const uint32_t*)nullptr, sel, I_out, cand, hist2);
+                      keys, (const uint32_t*)nullptr, sel, I_out, cand, hist2, c4, n4);
     } else {
         auto kfn = k_emit<false>;
         launch_kernel((P.chain & kChainEmit) != 0, kfn, grid_for(P.d, sm_count, resident_per_sm(kfn, 4)), kThreads, 0, st, P, keys, idx_map,
-                      sel, I_out, cand, hist2);
+                      sel, I_out, cand, hist2, c4, n4);
     }
     return 1;
 }
