@@ -506,18 +506,23 @@ k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, cons
                 }
             }
         }
-        // counting is branch-free: almost every key is below the threshold bin
-        uint32_t n_out = 0, n_ge = 0;
+        // counting is branch-free: almost every key is below the threshold bin.  The vector form keeps the outcome
+        // of its sixteen comparisons as two bit masks (bit 4u+q), so that the append below visits the hits only.
+        uint32_t n_out = 0, n_ge = 0, m_out = 0, m_ge = 0;
 #pragma unroll
         for (uint32_t u = 0; u < U; ++u)
             if (nk[u]) {
 #pragma unroll
                 for (uint32_t q = 0; q < 4; ++q)
-                    if (VEC || q == 0) {
+                    if (VEC) {
+                        m_out |= (uint32_t)(kq[u][q] >= thr_hi) << (4u * u + q);
+                        m_ge |= (uint32_t)(kq[u][q] >= thr_lo) << (4u * u + q);
+                    } else if (q == 0) {
                         n_out += kq[u][q] >= thr_hi;
                         n_ge += kq[u][q] >= thr_lo;
                     }
             }
+        if (VEC) { n_out = (uint32_t)__popc(m_out); n_ge = (uint32_t)__popc(m_ge); }
         const uint32_t n_cand = n_ge - n_out;
         const uint32_t packed = n_out | (n_cand << 16);         // each <= 16 per thread, <= 512 per warp
         uint32_t incl = packed;
@@ -532,6 +537,22 @@ k_emit(const __grid_constant__ Params P, const uint32_t* __restrict__ keys, cons
         uint32_t* po = warp_reserve(P, wb_out[wid], fill_out, &sel->cnt_out, I_out, P.k, total & 0xFFFFu, excl & 0xFFFFu);
         Cand* pc = warp_reserve(P, wb_cand[wid], fill_cand, &sel->cnt_cand, cand, P.d, total >> 16, excl >> 16);
         if (packed == 0) continue;                              // this lane has nothing to append
+        if (VEC) {
+            // one iteration per hit, in the order of the bits (u-major): an index above the bin needs no key, a
+            // candidate reads its key back (keys[idx]: the vector form has no index map)
+            for (uint32_t m = m_ge; m; m &= m - 1u) {
+                const uint32_t b = (uint32_t)__ffs((int)m) - 1u;
+                const uint32_t idx = ((t0 + (b >> 2) * kThreads) << 2) + (b & 3u);
+                if ((m_out >> b) & 1u) {
+                    *po++ = idx;
+                } else {
+                    const uint32_t key = __ldg(keys + idx);
+                    hist_add(P, sh2, (key >> 7) & (kHistBins - 1u));
+                    pc->key = key; pc->idx = idx; ++pc;
+                }
+            }
+            continue;
+        }
 #pragma unroll
         for (uint32_t u = 0; u < U; ++u) {
             if (!nk[u]) continue;
