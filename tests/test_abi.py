@@ -54,3 +54,15 @@ def test_product_never_imports_the_oracle():
         if f.endswith((".py", ".c", ".h")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2210_07454_b200" not in text and "sketched_amsgrad.h" not in text, f
+
+
+def test_every_option_the_library_parses_is_documented_in_the_header():
+    # the option names are string literals on both sides: a name sk_set_option / sk_get_option compares against must
+    # appear, quoted, in the header's description of the options
+    import re
+    src = open(os.path.join(ROOT, "paper_2210_07454_b200", "csrc", "sk_api.cu")).read()
+    names = set(re.findall(r'strcmp\(key, "([A-Za-z_0-9]+)"\)', src))
+    assert {"log2g", "window_lines", "chained_launches", "timing"} <= names
+    header = open(os.path.join(ROOT, "include", "sketched_amsgrad.h")).read()
+    missing = sorted(n for n in names if f'"{n}"' not in header)
+    assert not missing, missing
